@@ -1,0 +1,119 @@
+/*
+ * torq.h -- C ABI of the B200 (sm_100a) hot path of TORQ's rotated-MXFP4 linear layer.
+ *
+ * The path is the paper's online inference procedure (Algorithm 3): a token's d features are
+ * viewed as d/32 blocks of 32 (step 1), multiplied by the inter-block rotation (step 2) and by
+ * the intra-block rotation of each block (step 3), quantized per block to MXFP4 (step 4, Eq. 1)
+ * and handed to the next linear layer whose weights already carry the inverse rotation and are
+ * themselves MXFP4 (step 5, option B "weight fusion").
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller; the library allocates nothing
+ *     and keeps no reference after the call returns.  `stream` is a cudaStream_t passed as
+ *     void* (NULL = the legacy default stream).  Calls only enqueue work; they never synchronise.
+ *   - Tokens are rows (row-vector convention): Z = X . R_inter, then per block Z_b . R_intra[b].
+ *   - bf16 = bfloat16, u8 = unsigned byte.  Matrices are row-major, densely packed.
+ *   - MXFP4 codes: 4 bits per element = sign<<3 | e2m1 magnitude index over
+ *     {0, 0.5, 1, 1.5, 2, 3, 4, 6}; two codes per byte, the even element in the low nibble.
+ *   - Scales: one E8M0 byte per (row, 32-element block), byte = e + 127 with
+ *     e = clamp(floor(log2 amax) - 2, -127, 127) (amax == 0 -> byte 0), stored in the tiled
+ *     layout the block-scaled tensor-core instruction reads (see torq_scale_offset).  A scale
+ *     buffer always has torq_scales_bytes(rows, k) bytes: rows are padded to a multiple of 128
+ *     and K-blocks to a multiple of 4.  Producers in this library write 0x00 (2^-127) into the
+ *     padding rows; consumers never let padding reach a stored output.
+ *   - Return value: TORQ_OK or a host-detected error; nothing is launched on error.  Conditions
+ *     only the device can see (a bounded wait that ran out) are latched in an error word read by
+ *     torq_last_device_error(); a kernel that hits one stops issuing work, drains and returns --
+ *     it never traps.  Non-finite inputs are outside the contract (results unspecified, no hang).
+ */
+#ifndef TORQ_H_
+#define TORQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TORQ_OK = 0,
+  TORQ_ERR_NULL = 1,       /* a required pointer is NULL */
+  TORQ_ERR_SHAPE = 2,      /* a size violates the stated divisibility / range rules */
+  TORQ_ERR_ALIGN = 3,      /* a pointer is not 16-byte aligned */
+  TORQ_ERR_ARCH = 4,       /* current device is not compute capability 10.x */
+  TORQ_ERR_LAUNCH = 5,     /* CUDA reported an error while encoding descriptors or launching */
+  TORQ_ERR_TIMEOUT = 6,    /* (device error word) a bounded wait inside a kernel ran out */
+  TORQ_ERR_WORKSPACE = 7   /* workspace missing or smaller than torq_workspace_bytes() */
+} torq_status;
+
+typedef enum { TORQ_F32 = 0, TORQ_BF16 = 1 } torq_dtype;
+
+/* Algorithm 3 steps 1-4 (rotation as in Section 5: R = inter then intra; quantizer Eq. 1).
+ *   X         [M, d]        bf16
+ *   R_inter   [d, d]        bf16, y[m,j] = sum_i x[m,i] R_inter[i,j]; NULL = identity
+ *   R_intra   [d/32,32,32]  bf16, z[m,32b+j] = sum_i y[m,32b+i] R_intra[b][i][j]; NULL = identity
+ *   out_codes [M, d/2]      u8
+ *   out_scales              torq_scales_bytes(M, d) bytes, tiled layout
+ * Requires M >= 1, d >= 32, d % 32 == 0, 16-byte aligned pointers.  Accumulation is fp32
+ * (inter: tensor cores with exact bf16 products; intra: fp32 FMAs in index order).
+ * When R_inter is NULL the call runs the quantize-only kernel (plus the intra step if given). */
+torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void* R_intra,
+                                 int64_t M, int64_t d, void* out_codes, void* out_scales,
+                                 void* stream);
+
+/* Algorithm 3 step 5 (option B): Y[m,n] = sum_k a^[m,k] w^[n,k], a^/w^ the dequantized MXFP4
+ * values (codeword x 2^e), fp32 accumulation on the block-scaled FP4 tensor cores.
+ *   Aq [M, K/2] u8, As scales of A (tiled, torq_scales_bytes(M, K))
+ *   Wq [N, K/2] u8 (the fused weight W' stored with K contiguous), Ws (tiled, (N, K))
+ *   Y  [M, N] row-major of y_dtype
+ * Requires M,N >= 1, K % 128 == 0, N % 8 == 0, 16-byte aligned pointers. */
+torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, const void* Ws,
+                            int64_t M, int64_t N, int64_t K, void* Y, torq_dtype y_dtype,
+                            void* stream);
+
+/* Algorithm 3 steps 1-5 in one call: rotate, quantize, multiply.  The quantized activations live
+ * in `workspace` (>= torq_workspace_bytes(M, d, N) bytes, 256-byte aligned), laid out as codes
+ * [M, d/2] followed (256-byte aligned) by the tiled scales; pass dbg_codes / dbg_scales non-NULL
+ * to also receive copies of them.  Requires d % 128 == 0 and N % 8 == 0. */
+torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* R_intra,
+                                const void* Wq, const void* Ws, int64_t M, int64_t d, int64_t N,
+                                void* Y, torq_dtype y_dtype, void* workspace,
+                                size_t workspace_bytes, void* dbg_codes, void* dbg_scales,
+                                void* stream);
+
+/* Eq. 1 alone: quantize Z [M, d] (fp32 or bf16) to MXFP4.  On fp32 input the result is defined
+ * bit for bit (round to nearest even on the e2m1 grid, saturation to +-6, sign bit kept). */
+torq_status torq_quantize_mxfp4(const void* Z, torq_dtype z_dtype, int64_t M, int64_t d,
+                                void* out_codes, void* out_scales, void* stream);
+
+/* Scale-factor layout (not in the paper; fixed by the FP4 tensor-core instruction): 512-byte tiles
+ * of 128 rows x 4 K-blocks, tiles ordered row-tile major; inside a tile
+ *   byte = (row % 32) * 16 + ((row % 128) / 32) * 4 + (kblock % 4).
+ * Host-side pure functions. */
+size_t torq_scales_bytes(int64_t rows, int64_t k);
+size_t torq_scale_offset(int64_t row, int64_t kblock, int64_t k);
+size_t torq_workspace_bytes(int64_t M, int64_t d, int64_t N);
+
+/* Re-tile a plain [rows, k/32] scale matrix into the layout above (padding bytes := 0x00). */
+torq_status torq_swizzle_scales(const void* linear_scales, int64_t rows, int64_t k, void* out,
+                                void* stream);
+
+/* Offline helper for the weight side of step 5 (W' = R~^T W, R~ = R_inter . blockdiag(R_intra)):
+ * writes R~ [d, d] as fp32 computed in fp32 from the bf16 inputs.  d % 32 == 0. */
+torq_status torq_merge_rotations(const void* R_inter, const void* R_intra, int64_t d,
+                                 void* R_merged_f32, void* stream);
+
+const char* torq_status_string(torq_status s);
+
+/* Synchronises `stream`, then returns and clears the device error word of the current device:
+ * 0, or TORQ_ERR_TIMEOUT in the low byte with the id of the wait that gave up in bits 8..15. */
+int torq_last_device_error(void* stream);
+
+/* Number of kernels this library has launched since load (all devices, all streams). */
+int64_t torq_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TORQ_H_ */

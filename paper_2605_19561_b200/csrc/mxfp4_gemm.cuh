@@ -1,0 +1,218 @@
+// Block-scaled MXFP4 x MXFP4 GEMM (Algorithm 3 step 5, option B) on the tcgen05 FP4 tensor
+// cores: Y[m,n] = sum_k a^[m,k] w^[n,k] with one E8M0 scale per 32 elements of K on each side.
+//
+// Persistent, warp-specialised, one CTA per SM:
+//   warp 0      TMA producer  : A / W tiles (128-byte swizzle) and their scale tiles into a
+//                               ring of shared-memory stages
+//   warp 1      MMA issuer    : copies the scale tiles shared -> tensor memory (tcgen05.cp),
+//                               issues tcgen05.mma kind::mxf4.block_scale, commits to barriers
+//   warps 2..5  epilogue      : tensor memory -> registers -> Y (fp32 or bf16), 32 rows per warp
+// Tile = 128 x BN x 256 (one stage = 128 bytes of K per row = one swizzle atom).  NACC
+// accumulator buffers in tensor memory let the epilogue of one tile overlap the next mainloop.
+#pragma once
+#include <cuda_bf16.h>
+#include "sm100_ptx.cuh"
+
+namespace torq {
+
+template <int BN, int NACC>
+struct GemmCfg {
+  static constexpr int BM = 128;
+  static constexpr int BK = 256;                       // elements of K per stage
+  static constexpr int A_BYTES = BM * BK / 2;          // 16 KiB
+  static constexpr int B_BYTES = BN * BK / 2;
+  static constexpr int SFA_BYTES = 1024;               // 128 rows x 8 K-blocks
+  static constexpr int SFB_BYTES = (BN / 128) * 1024;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
+  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+  static constexpr int BAR_BYTES = 256;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + align slack
+  static constexpr int ACC_COLS = NACC * BN;
+  static constexpr int SFA_COL = ACC_COLS;             // 2 K-chunks x 4 columns
+  static constexpr int SFB_COL = ACC_COLS + 8;         // 2 K-chunks x BN/32 columns
+  static constexpr int TMEM_COLS = 512;
+  static constexpr int THREADS = 192;
+  static_assert(SFB_COL + 2 * (BN / 32) <= TMEM_COLS, "tensor memory budget");
+  static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+};
+
+template <int BN, int NACC>
+__global__ void __launch_bounds__(192, 1)
+mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const uint8_t* __restrict__ As, const uint8_t* __restrict__ Ws,
+                  void* __restrict__ Y, int y_is_bf16, int M, int N, int K, int* err_word) {
+  using C = GemmCfg<BN, NACC>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + C::STAGES * C::STAGE_BYTES;
+  // barrier map (8 bytes each): full[s], empty[s], acc_full[a], acc_empty[a]
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };
+  auto accf_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + a); };
+  auto acce_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + NACC + a); };
+  volatile uint32_t* tmem_slot =
+      reinterpret_cast<volatile uint32_t*>(smem_gen + C::STAGES * C::STAGE_BYTES + 192);
+  volatile int* cta_abort =
+      reinterpret_cast<volatile int*>(smem_gen + C::STAGES * C::STAGE_BYTES + 200);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m_tiles = (M + C::BM - 1) / C::BM;
+  const int n_tiles = (N + BN - 1) / BN;
+  const int total_tiles = m_tiles * n_tiles;
+  const int k_tiles = (K + C::BK - 1) / C::BK;          // K % 128 == 0: last stage may be half
+  const int kb4 = K / 128;                              // scale K-chunks (4 K-blocks each) per row
+  const int n_rowtiles = (N + 127) / 128;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < NACC; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 4); }
+    *cta_abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS); tmem_relinquish(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tmA);
+      tma_prefetch_desc(&tmB);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int mt = tile % m_tiles, nt = tile / m_tiles;
+        const int rt0 = nt * (BN / 128);
+        const int n_sfb_tiles = min(BN / 128, n_rowtiles - rt0);
+        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+          const int s = it % C::STAGES;
+          if (!mbar_wait(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
+                         SITE_PRODUCER_EMPTY)) { ok = false; break; }
+          const int nchunk = min(2, kb4 - 2 * kt);
+          const uint32_t sf_bytes = 512u * nchunk;
+          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+          mbar_arrive_expect_tx(full_bar(s), C::A_BYTES + C::B_BYTES + sf_bytes * (1 + n_sfb_tiles));
+          tma_load_2d(st, &tmA, kt * 128, mt * C::BM, full_bar(s));
+          tma_load_2d(st + C::A_BYTES, &tmB, kt * 128, nt * BN, full_bar(s));
+          bulk_load_1d(st + C::A_BYTES + C::B_BYTES, As + ((size_t)mt * kb4 + 2 * kt) * 512, sf_bytes,
+                       full_bar(s));
+          for (int t = 0; t < n_sfb_tiles; ++t)
+            bulk_load_1d(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * 1024,
+                         Ws + ((size_t)(rt0 + t) * kb4 + 2 * kt) * 512, sf_bytes, full_bar(s));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+        const int a = tcount % NACC;
+        if (!mbar_wait(acce_bar(a), ((tcount / NACC) & 1) ^ 1, cta_abort, err_word,
+                       SITE_MMA_ACC_EMPTY)) { ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t acc = tmem_base + a * BN;
+        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+          const int s = it % C::STAGES;
+          if (!mbar_wait(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
+            ok = false; break;
+          }
+          tc_fence_after_sync();
+          const int nchunk = min(2, kb4 - 2 * kt);
+          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+          const uint32_t sfa = st + C::A_BYTES + C::B_BYTES, sfb = sfa + C::SFA_BYTES;
+          for (int c = 0; c < nchunk; ++c) {
+            tmem_cp_32x128b_warpx4(tmem_base + C::SFA_COL + 4 * c, make_desc(sfa + 512 * c, 0, 128, 0));
+#pragma unroll
+            for (int t = 0; t < BN / 128; ++t)
+              tmem_cp_32x128b_warpx4(tmem_base + C::SFB_COL + c * (BN / 32) + 4 * t,
+                                     make_desc(sfb + 1024 * t + 512 * c, 0, 128, 0));
+          }
+          const uint64_t adesc = make_desc(st, 16, 1024, kSwizzle128);
+          const uint64_t bdesc = make_desc(st + C::A_BYTES, 16, 1024, kSwizzle128);
+          for (int j = 0; j < 2 * nchunk; ++j) {        // 64 elements (32 bytes) of K each
+            const uint32_t id = (j & 1) * 2;
+            mma_mxf4(acc, adesc + 2 * j, bdesc + 2 * j, idesc_mxf4(128, BN, id, id),
+                     tmem_base + C::SFA_COL + 4 * (j >> 1),
+                     tmem_base + C::SFB_COL + (j >> 1) * (BN / 32), (kt | j) != 0);
+          }
+          tc_commit(empty_bar(s));
+        }
+        if (ok) tc_commit(accf_bar(a));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int q = warp & 3;                              // lane quarter this warp may read
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      const int mt = tile % m_tiles, nt = tile / m_tiles;
+      const int a = tcount % NACC;
+      ok = mbar_wait(accf_bar(a), (tcount / NACC) & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
+      ok = __all_sync(0xFFFFFFFFu, ok);                  // keep the warp together on the way out
+      if (!ok) break;
+      tc_fence_after_sync();
+      const int64_t row = (int64_t)mt * C::BM + q * 32 + lane;
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
+#pragma unroll 1
+      for (int cc = 0; cc < BN / 32; ++cc) {
+        uint32_t v[32];
+        tmem_ld_32x32(tacc + cc * 32, v);
+        tmem_ld_wait();
+        if (cc == BN / 32 - 1) {                         // accumulator fully read: hand it back
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acce_bar(a));
+        }
+        const int64_t col = (int64_t)nt * BN + cc * 32;
+        if (row < M && col < N) {
+          if (y_is_bf16) {
+            __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(Y) + row * N + col;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              if (col + 8 * g + 8 <= N) {
+                uint4 o;
+                uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                  __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[8 * g + 2 * p]),
+                                                           __uint_as_float(v[8 * g + 2 * p + 1]));
+                  ow[p] = *reinterpret_cast<uint32_t*>(&h);
+                }
+                *reinterpret_cast<uint4*>(yp + 8 * g) = o;
+              }
+            }
+          } else {
+            float* yp = reinterpret_cast<float*>(Y) + row * N + col;
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+              if (col + 4 * g + 4 <= N)
+                *reinterpret_cast<uint4*>(yp + 4 * g) =
+                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before_sync();
+  __syncthreads();
+  if (*cta_abort) {
+    // A wait gave up: give in-flight copies and MMAs time to land before the CTA's shared and
+    // tensor memory go away.
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+}
+
+}  // namespace torq

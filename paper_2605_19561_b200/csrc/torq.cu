@@ -1,0 +1,287 @@
+// C-ABI entry points of the library (see include/torq.h): argument validation, TMA descriptor
+// encoding, kernel selection and launch.  Nothing here computes on the host.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <atomic>
+#include <mutex>
+
+#include "../../include/torq.h"
+#include "mxfp4_gemm.cuh"
+#include "quantize.cuh"
+#include "rotate_quantize.cuh"
+#include "sm100_ptx.cuh"
+
+namespace torq {
+
+__device__ int g_error_word = 0;
+
+constexpr int kMaxDevices = 64;
+struct DeviceState {
+  bool ready = false;
+  bool arch_ok = false;
+  int sm_count = 0;
+  int* err_word = nullptr;
+};
+static DeviceState g_dev[kMaxDevices];
+static std::mutex g_mutex;
+static std::atomic<int64_t> g_launches{0};
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+
+template <typename K>
+static bool opt_in_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) ==
+         cudaSuccess;
+}
+
+// Per-device one-time set-up: architecture check, SM count, error-word address, shared-memory
+// opt-in of the tensor-core kernels.  Returns nullptr when CUDA itself fails.
+static DeviceState* device_state() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceState& st = g_dev[dev];
+  if (st.ready) return &st;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+    return nullptr;
+  if (cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return nullptr;
+  st.arch_ok = (major == 10);
+  if (st.arch_ok) {
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&st.err_word), g_error_word) != cudaSuccess)
+      return nullptr;
+    if (!g_encode) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) !=
+              cudaSuccess || qres != cudaDriverEntryPointSuccess || fn == nullptr)
+        return nullptr;
+      g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    bool ok = opt_in_smem(mxfp4_gemm_kernel<256, 1>, GemmCfg<256, 1>::SMEM_BYTES) &&
+              opt_in_smem(mxfp4_gemm_kernel<128, 2>, GemmCfg<128, 2>::SMEM_BYTES) &&
+              opt_in_smem(rotate_quantize_kernel<256>, RotCfg<256>::SMEM_BYTES) &&
+              opt_in_smem(rotate_quantize_kernel<128>, RotCfg<128>::SMEM_BYTES);
+    if (!ok) return nullptr;
+  }
+  st.ready = true;
+  return &st;
+}
+
+// 2-D row-major tensor [rows, cols] of `elem_bytes`-byte elements, box [box_rows, box_cols],
+// 128-byte swizzle, zero fill outside the tensor.
+static bool encode_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* base,
+                      uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return g_encode(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline int ew_grid(int64_t items, int per_block, int sm_count) {
+  int64_t blocks = (items + per_block - 1) / per_block;
+  int64_t cap = (int64_t)sm_count * 16;
+  return (int)(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
+}
+static inline torq_status launch_status() {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return cudaGetLastError() == cudaSuccess ? TORQ_OK : TORQ_ERR_LAUNCH;
+}
+
+static torq_status quantize_impl(DeviceState* st, const void* Z, torq_dtype dt, int64_t M, int64_t d,
+                                 void* codes, void* scales, cudaStream_t s) {
+  const int64_t kb4 = (d / 32 + 3) / 4;
+  const int64_t items = ((M + 127) / 128 * 128) * ((kb4 * 128 + 255) / 256);   // warps
+  const int grid = ew_grid(items, 8, st->sm_count);
+  if (dt == TORQ_F32)
+    quantize_kernel<float><<<grid, 256, 0, s>>>(static_cast<const float*>(Z), M, d,
+                                                static_cast<uint8_t*>(codes), static_cast<uint8_t*>(scales));
+  else
+    quantize_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(Z), M, d,
+                                                        static_cast<uint8_t*>(codes),
+                                                        static_cast<uint8_t*>(scales));
+  return launch_status();
+}
+
+}  // namespace torq
+
+using namespace torq;
+
+extern "C" {
+
+size_t torq_scales_bytes(int64_t rows, int64_t k) {
+  if (rows <= 0 || k <= 0) return 0;
+  return (size_t)((rows + 127) / 128) * (size_t)((k / 32 + 3) / 4) * 512;
+}
+
+size_t torq_scale_offset(int64_t row, int64_t kblock, int64_t k) {
+  return scale_offset(row, kblock, (k / 32 + 3) / 4);
+}
+
+size_t torq_workspace_bytes(int64_t M, int64_t d, int64_t N) {
+  (void)N;
+  if (M <= 0 || d <= 0) return 0;
+  size_t codes = ((size_t)M * (size_t)(d / 2) + 255) / 256 * 256;
+  return codes + torq_scales_bytes(M, d);
+}
+
+const char* torq_status_string(torq_status s) {
+  switch (s) {
+    case TORQ_OK: return "ok";
+    case TORQ_ERR_NULL: return "null pointer";
+    case TORQ_ERR_SHAPE: return "unsupported shape";
+    case TORQ_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case TORQ_ERR_ARCH: return "device is not compute capability 10.x";
+    case TORQ_ERR_LAUNCH: return "CUDA launch or descriptor error";
+    case TORQ_ERR_TIMEOUT: return "a bounded device wait ran out";
+    case TORQ_ERR_WORKSPACE: return "workspace missing or too small";
+  }
+  return "unknown";
+}
+
+int64_t torq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int torq_last_device_error(void* stream) {
+  DeviceState* st = device_state();
+  if (!st || !st->arch_ok) return 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(s) != cudaSuccess) return TORQ_ERR_LAUNCH;
+  int v = 0, zero = 0;
+  if (cudaMemcpy(&v, st->err_word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return TORQ_ERR_LAUNCH;
+  if (v != 0) cudaMemcpy(st->err_word, &zero, sizeof(int), cudaMemcpyHostToDevice);
+  return v;
+}
+
+torq_status torq_quantize_mxfp4(const void* Z, torq_dtype z_dtype, int64_t M, int64_t d,
+                                void* out_codes, void* out_scales, void* stream) {
+  if (!Z || !out_codes || !out_scales) return TORQ_ERR_NULL;
+  if (M < 1 || d < 32 || d % 32 != 0 || M > (1 << 30) || d > (1 << 30)) return TORQ_ERR_SHAPE;
+  if (z_dtype != TORQ_F32 && z_dtype != TORQ_BF16) return TORQ_ERR_SHAPE;
+  if (!aligned16(Z) || !aligned16(out_codes) || !aligned16(out_scales)) return TORQ_ERR_ALIGN;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  return quantize_impl(st, Z, z_dtype, M, d, out_codes, out_scales, static_cast<cudaStream_t>(stream));
+}
+
+torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void* R_intra, int64_t M,
+                                 int64_t d, void* out_codes, void* out_scales, void* stream) {
+  if (!X || !out_codes || !out_scales) return TORQ_ERR_NULL;
+  if (M < 1 || d < 32 || d % 32 != 0 || M > (1 << 30) || d > (1 << 24)) return TORQ_ERR_SHAPE;
+  if (!aligned16(X) || !aligned16(out_codes) || !aligned16(out_scales) ||
+      (R_inter && !aligned16(R_inter)) || (R_intra && !aligned16(R_intra)))
+    return TORQ_ERR_ALIGN;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* codes = static_cast<uint8_t*>(out_codes);
+  uint8_t* scales = static_cast<uint8_t*>(out_scales);
+  if (!R_inter) {
+    if (!R_intra) return quantize_impl(st, X, TORQ_BF16, M, d, codes, scales, s);
+    const int64_t items = ((M + 127) / 128 * 128) * (((d / 32 + 3) / 4) * 4);
+    intra_quantize_kernel<<<ew_grid(items, 128, st->sm_count), 128, 0, s>>>(
+        static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(R_intra), M, d, codes,
+        scales);
+    return launch_status();
+  }
+  CUtensorMap tmX, tmR;
+  if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d, 128, 64) ||
+      !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
+    return TORQ_ERR_LAUNCH;
+  const int m_tiles = (int)((M + 127) / 128);
+  const int tiles = m_tiles * (int)((d + 255) / 256);
+  const int grid = tiles < st->sm_count ? tiles : st->sm_count;
+  rotate_quantize_kernel<256><<<grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s>>>(
+      tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, st->err_word);
+  return launch_status();
+}
+
+torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, const void* Ws, int64_t M,
+                            int64_t N, int64_t K, void* Y, torq_dtype y_dtype, void* stream) {
+  if (!Aq || !As || !Wq || !Ws || !Y) return TORQ_ERR_NULL;
+  if (M < 1 || N < 8 || K < 128 || K % 128 != 0 || N % 8 != 0 || M > (1 << 30) || N > (1 << 30) ||
+      K > (1 << 24))
+    return TORQ_ERR_SHAPE;
+  if (y_dtype != TORQ_F32 && y_dtype != TORQ_BF16) return TORQ_ERR_SHAPE;
+  if (!aligned16(Aq) || !aligned16(As) || !aligned16(Wq) || !aligned16(Ws) || !aligned16(Y))
+    return TORQ_ERR_ALIGN;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  constexpr int BN = 256;
+  CUtensorMap tmA, tmB;
+  if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, (uint64_t)(K / 2), 128, 128) ||
+      !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)(K / 2), BN, 128))
+    return TORQ_ERR_LAUNCH;
+  const int tiles = (int)((M + 127) / 128) * (int)((N + BN - 1) / BN);
+  const int grid = tiles < st->sm_count ? tiles : st->sm_count;
+  mxfp4_gemm_kernel<BN, 1><<<grid, GemmCfg<BN, 1>::THREADS, GemmCfg<BN, 1>::SMEM_BYTES, s>>>(
+      tmA, tmB, static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y,
+      y_dtype == TORQ_BF16 ? 1 : 0, (int)M, (int)N, (int)K, st->err_word);
+  return launch_status();
+}
+
+torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* R_intra, const void* Wq,
+                                const void* Ws, int64_t M, int64_t d, int64_t N, void* Y,
+                                torq_dtype y_dtype, void* workspace, size_t workspace_bytes,
+                                void* dbg_codes, void* dbg_scales, void* stream) {
+  if (!X || !Wq || !Ws || !Y) return TORQ_ERR_NULL;
+  if (M < 1 || d < 128 || d % 128 != 0 || N < 8 || N % 8 != 0) return TORQ_ERR_SHAPE;
+  if (!workspace || workspace_bytes < torq_workspace_bytes(M, d, N)) return TORQ_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return TORQ_ERR_ALIGN;
+  uint8_t* codes = static_cast<uint8_t*>(workspace);
+  const size_t codes_bytes = (size_t)M * (size_t)(d / 2);
+  uint8_t* scales = codes + (codes_bytes + 255) / 256 * 256;
+  torq_status rc = torq_rotate_quantize(X, R_inter, R_intra, M, d, codes, scales, stream);
+  if (rc != TORQ_OK) return rc;
+  rc = torq_mxfp4_gemm(codes, scales, Wq, Ws, M, N, d, Y, y_dtype, stream);
+  if (rc != TORQ_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dbg_codes &&
+      cudaMemcpyAsync(dbg_codes, codes, codes_bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return TORQ_ERR_LAUNCH;
+  if (dbg_scales && cudaMemcpyAsync(dbg_scales, scales, torq_scales_bytes(M, d),
+                                    cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return TORQ_ERR_LAUNCH;
+  return TORQ_OK;
+}
+
+torq_status torq_swizzle_scales(const void* linear_scales, int64_t rows, int64_t k, void* out,
+                                void* stream) {
+  if (!linear_scales || !out) return TORQ_ERR_NULL;
+  if (rows < 1 || k < 32 || k % 32 != 0) return TORQ_ERR_SHAPE;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  const int64_t items = ((rows + 127) / 128 * 128) * (((k / 32 + 3) / 4) * 4);
+  swizzle_scales_kernel<<<ew_grid(items, 256, st->sm_count), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint8_t*>(linear_scales), rows, k / 32, static_cast<uint8_t*>(out));
+  return launch_status();
+}
+
+torq_status torq_merge_rotations(const void* R_inter, const void* R_intra, int64_t d, void* R_merged_f32,
+                                 void* stream) {
+  if (!R_inter || !R_intra || !R_merged_f32) return TORQ_ERR_NULL;
+  if (d < 32 || d % 32 != 0 || d > (1 << 24)) return TORQ_ERR_SHAPE;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  merge_rotations_kernel<<<ew_grid(d * d, 256, st->sm_count), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(R_inter), static_cast<const __nv_bfloat16*>(R_intra), d,
+      static_cast<float*>(R_merged_f32));
+  return launch_status();
+}
+
+}  // extern "C"

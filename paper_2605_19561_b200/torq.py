@@ -1,0 +1,200 @@
+"""Thin ctypes binding over the C-ABI library (include/torq.h).  Argument marshalling only:
+every step of the path runs in the CUDA kernels; PyTorch provides device memory and streams.
+There is no fallback: a missing library or a non-zero status raises."""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+TORQ_F32, TORQ_BF16 = 0, 1
+_STATUS = {0: "TORQ_OK", 1: "TORQ_ERR_NULL", 2: "TORQ_ERR_SHAPE", 3: "TORQ_ERR_ALIGN", 4: "TORQ_ERR_ARCH",
+           5: "TORQ_ERR_LAUNCH", 6: "TORQ_ERR_TIMEOUT", 7: "TORQ_ERR_WORKSPACE"}
+_lib_handle = None
+
+
+class TorqError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {_STATUS.get(code, code)}")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads (building first if the binary is absent or stale and nvcc is available)."""
+    global _lib_handle
+    if _lib_handle is not None:
+        return _lib_handle
+    path = _build.LIB_PATH
+    if _build.needs_build():
+        _build.build_library()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing; run paper_2605_19561_b200/build.py")
+    L = ctypes.CDLL(path)
+    vp, i64, sz, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_int
+    L.torq_rotate_quantize.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp]
+    L.torq_rotate_quantize.restype = ci
+    L.torq_mxfp4_gemm.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, ci, vp]
+    L.torq_mxfp4_gemm.restype = ci
+    L.torq_rotated_linear.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, vp, sz, vp, vp, vp]
+    L.torq_rotated_linear.restype = ci
+    L.torq_quantize_mxfp4.argtypes = [vp, ci, i64, i64, vp, vp, vp]
+    L.torq_quantize_mxfp4.restype = ci
+    L.torq_scales_bytes.argtypes = [i64, i64]
+    L.torq_scales_bytes.restype = sz
+    L.torq_scale_offset.argtypes = [i64, i64, i64]
+    L.torq_scale_offset.restype = sz
+    L.torq_workspace_bytes.argtypes = [i64, i64, i64]
+    L.torq_workspace_bytes.restype = sz
+    L.torq_swizzle_scales.argtypes = [vp, i64, i64, vp, vp]
+    L.torq_swizzle_scales.restype = ci
+    L.torq_merge_rotations.argtypes = [vp, vp, i64, vp, vp]
+    L.torq_merge_rotations.restype = ci
+    L.torq_status_string.argtypes = [ci]
+    L.torq_status_string.restype = ctypes.c_char_p
+    L.torq_last_device_error.argtypes = [vp]
+    L.torq_last_device_error.restype = ci
+    L.torq_launch_count.argtypes = []
+    L.torq_launch_count.restype = i64
+    _lib_handle = L
+    return L
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(t, dtype, name):
+    if t is None:
+        return
+    if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise ValueError(f"{name}: expected a contiguous CUDA tensor of {dtype}, got {t.dtype} on {t.device}")
+
+
+def _raise(code, where):
+    if code != 0:
+        raise TorqError(code, where)
+
+
+def torq_scales_bytes(rows: int, k: int) -> int:
+    return lib().torq_scales_bytes(rows, k)
+
+
+def torq_scale_offset(row: int, kblock: int, k: int) -> int:
+    return lib().torq_scale_offset(row, kblock, k)
+
+
+def torq_workspace_bytes(M: int, d: int, N: int) -> int:
+    return lib().torq_workspace_bytes(M, d, N)
+
+
+def torq_launch_count() -> int:
+    return lib().torq_launch_count()
+
+
+def torq_last_device_error(stream=None) -> int:
+    return lib().torq_last_device_error(_stream(stream))
+
+
+def torq_quantize_mxfp4(Z, out_codes=None, out_scales=None, stream=None):
+    """Z [M,d] float32 or bfloat16 -> (codes [M,d/2] uint8, tiled scale bytes uint8)."""
+    M, d = Z.shape
+    dt = TORQ_F32 if Z.dtype == torch.float32 else TORQ_BF16
+    _check(Z, torch.float32 if dt == TORQ_F32 else torch.bfloat16, "Z")
+    if out_codes is None:
+        out_codes = torch.empty((M, d // 2), dtype=torch.uint8, device=Z.device)
+    if out_scales is None:
+        out_scales = torch.empty(torq_scales_bytes(M, d), dtype=torch.uint8, device=Z.device)
+    _raise(lib().torq_quantize_mxfp4(_ptr(Z), dt, M, d, _ptr(out_codes), _ptr(out_scales), _stream(stream)),
+           "torq_quantize_mxfp4")
+    return out_codes, out_scales
+
+
+def torq_rotate_quantize(X, R_inter, R_intra, out_codes=None, out_scales=None, stream=None):
+    """X [M,d] bf16, R_inter [d,d] bf16 or None, R_intra [d/32,32,32] bf16 or None."""
+    M, d = X.shape
+    for t, n in ((X, "X"), (R_inter, "R_inter"), (R_intra, "R_intra")):
+        _check(t, torch.bfloat16, n)
+    if out_codes is None:
+        out_codes = torch.empty((M, d // 2), dtype=torch.uint8, device=X.device)
+    if out_scales is None:
+        out_scales = torch.empty(torq_scales_bytes(M, d), dtype=torch.uint8, device=X.device)
+    _raise(lib().torq_rotate_quantize(_ptr(X), _ptr(R_inter), _ptr(R_intra), M, d, _ptr(out_codes),
+                                      _ptr(out_scales), _stream(stream)), "torq_rotate_quantize")
+    return out_codes, out_scales
+
+
+def torq_mxfp4_gemm(Aq, As, Wq, Ws, out_dtype=torch.bfloat16, Y=None, stream=None):
+    """Aq [M,K/2], Wq [N,K/2] uint8 codes; As, Ws tiled scale bytes -> Y [M,N]."""
+    M, K2 = Aq.shape
+    N = Wq.shape[0]
+    for t, n in ((Aq, "Aq"), (As, "As"), (Wq, "Wq"), (Ws, "Ws")):
+        _check(t, torch.uint8, n)
+    if Y is None:
+        Y = torch.empty((M, N), dtype=out_dtype, device=Aq.device)
+    _check(Y, Y.dtype, "Y")
+    dt = TORQ_F32 if Y.dtype == torch.float32 else TORQ_BF16
+    _raise(lib().torq_mxfp4_gemm(_ptr(Aq), _ptr(As), _ptr(Wq), _ptr(Ws), M, N, 2 * K2, _ptr(Y), dt,
+                                 _stream(stream)), "torq_mxfp4_gemm")
+    return Y
+
+
+def torq_rotated_linear(X, R_inter, R_intra, Wq, Ws, out_dtype=torch.bfloat16, Y=None, workspace=None,
+                        dbg_codes=None, dbg_scales=None, stream=None):
+    """Rotate, quantize and multiply in one call.  Returns Y [M,N]."""
+    M, d = X.shape
+    N = Wq.shape[0]
+    for t, n in ((X, "X"), (R_inter, "R_inter"), (R_intra, "R_intra")):
+        _check(t, torch.bfloat16, n)
+    for t, n in ((Wq, "Wq"), (Ws, "Ws"), (dbg_codes, "dbg_codes"), (dbg_scales, "dbg_scales")):
+        _check(t, torch.uint8, n)
+    if Y is None:
+        Y = torch.empty((M, N), dtype=out_dtype, device=X.device)
+    if workspace is None:
+        workspace = torch.empty(torq_workspace_bytes(M, d, N), dtype=torch.uint8, device=X.device)
+    dt = TORQ_F32 if Y.dtype == torch.float32 else TORQ_BF16
+    _raise(lib().torq_rotated_linear(_ptr(X), _ptr(R_inter), _ptr(R_intra), _ptr(Wq), _ptr(Ws), M, d, N,
+                                     _ptr(Y), dt, _ptr(workspace), workspace.numel(), _ptr(dbg_codes),
+                                     _ptr(dbg_scales), _stream(stream)), "torq_rotated_linear")
+    return Y
+
+
+def torq_swizzle_scales(linear, k: int, out=None, stream=None):
+    rows = linear.shape[0]
+    _check(linear, torch.uint8, "linear")
+    if out is None:
+        out = torch.empty(torq_scales_bytes(rows, k), dtype=torch.uint8, device=linear.device)
+    _raise(lib().torq_swizzle_scales(_ptr(linear), rows, k, _ptr(out), _stream(stream)), "torq_swizzle_scales")
+    return out
+
+
+def torq_merge_rotations(R_inter, R_intra, out=None, stream=None):
+    d = R_inter.shape[0]
+    _check(R_inter, torch.bfloat16, "R_inter")
+    _check(R_intra, torch.bfloat16, "R_intra")
+    if out is None:
+        out = torch.empty((d, d), dtype=torch.float32, device=R_inter.device)
+    _raise(lib().torq_merge_rotations(_ptr(R_inter), _ptr(R_intra), d, _ptr(out), _stream(stream)),
+           "torq_merge_rotations")
+    return out
+
+
+def prepare_weights(R_inter, R_intra, W):
+    """Offline weight side of the layer (not on the timed path): W' = R~^T W for W [d,N] float32,
+    stored [N,d], MXFP4-quantized along K by torq_quantize_mxfp4.  The matrix product is a library
+    call (torch.matmul, fp32); returns (Wq [N,d/2], Ws tiled)."""
+    Rm = torq_merge_rotations(R_inter, R_intra)
+    prev = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = False
+    try:
+        Wp = torch.matmul(W.t().contiguous().to(torch.float32), Rm).contiguous()   # [N,d] = (R~^T W)^T
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = prev
+    return torq_quantize_mxfp4(Wp)

@@ -1,0 +1,65 @@
+"""Host-side checks that need no GPU: the shared library builds, loads, exports every symbol the
+header declares, its pure host functions agree with the layout the oracle states, and argument
+errors are reported as status codes before anything touches a device."""
+import ctypes
+import os
+import re
+
+import numpy as np
+
+import oracle as O
+from paper_2605_19561_b200 import torq
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "torq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(torq_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    L = torq.lib()
+    names = _declared_symbols()
+    assert {"torq_rotate_quantize", "torq_mxfp4_gemm", "torq_rotated_linear", "torq_quantize_mxfp4"} <= set(names)
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_scale_layout_functions_match_the_oracle_statement():
+    for rows, k in [(1, 32), (64, 256), (129, 4096), (2048, 14336), (200, 96)]:
+        assert torq.torq_scales_bytes(rows, k) == O.scale_layout_bytes(rows, k)
+    g = np.random.default_rng(0)
+    for _ in range(2000):
+        k = int(g.integers(1, 500)) * 32
+        r = int(g.integers(0, 5000))
+        c = int(g.integers(0, k // 32))
+        assert torq.torq_scale_offset(r, c, k) == int(O.scale_layout_offset(r, c, k))
+
+
+def test_workspace_holds_codes_and_scales():
+    M, d, N = 130, 256, 64
+    need = torq.torq_workspace_bytes(M, d, N)
+    assert need >= M * d // 2 + torq.torq_scales_bytes(M, d)
+    assert need % 256 == 0
+
+
+def test_argument_errors_are_status_codes():
+    L = torq.lib()
+    one = ctypes.c_void_p(16)      # non-null, 16-byte aligned, never dereferenced on these paths
+    odd = ctypes.c_void_p(24)
+    assert L.torq_rotate_quantize(None, None, None, 4, 64, one, one, None) == 1
+    assert L.torq_rotate_quantize(one, None, None, 4, 48, one, one, None) == 2      # d % 32 != 0
+    assert L.torq_rotate_quantize(one, None, None, 0, 64, one, one, None) == 2      # M < 1
+    assert L.torq_rotate_quantize(odd, None, None, 4, 64, one, one, None) == 3
+    assert L.torq_mxfp4_gemm(one, one, one, None, 4, 8, 128, one, 0, None) == 1
+    assert L.torq_mxfp4_gemm(one, one, one, one, 4, 8, 96, one, 0, None) == 2       # K % 128 != 0
+    assert L.torq_mxfp4_gemm(one, one, one, one, 4, 12, 128, one, 0, None) == 2     # N % 8 != 0
+    assert L.torq_mxfp4_gemm(one, one, one, one, 4, 8, 128, one, 5, None) == 2      # bad dtype
+    assert L.torq_quantize_mxfp4(one, 0, 4, 64, None, one, None) == 1
+    assert L.torq_quantize_mxfp4(one, 0, 4, 33, one, one, None) == 2
+    assert L.torq_rotated_linear(one, one, one, one, one, 4, 128, 8, one, 0, None, 0, None, None, None) == 7
+    assert L.torq_rotated_linear(one, one, one, one, one, 4, 128, 8, one, 0, one, 16, None, None, None) == 7
+    assert L.torq_rotated_linear(one, one, one, one, one, 4, 96, 8, one, 0, one, 1 << 20, None, None, None) == 2
+    assert L.torq_status_string(0) == b"ok" and L.torq_status_string(6)

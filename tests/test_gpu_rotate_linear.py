@@ -1,0 +1,135 @@
+"""GPU parity: rotate + quantize (Algorithm 3 steps 1-4) and the fused rotated linear layer
+(steps 1-5) against the oracle.
+
+Bounds (the fp32 tensor-core accumulation order differs from the oracle's fp64): at most 1e-4 of
+the elements may differ, each by one step on the e2m1 lattice; at most 1e-4 of the blocks may
+differ in scale, by one step; the GEMM result is compared, on the codes the GPU actually
+produced, to 1e-3 relative Frobenius error."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from helpers import dev_bf16, dev_u8, gpu_quantized_to_numpy, mismatch_report
+from paper_2605_19561_b200 import inputs as I
+from paper_2605_19561_b200 import torq
+
+pytestmark = pytest.mark.gpu
+
+
+def _rotate_quantize_case(xb, rb, rib, check_exact=False):
+    M, d = xb.shape
+    codes_t, scales_t = torq.torq_rotate_quantize(dev_bf16(xb), None if rb is None else dev_bf16(rb),
+                                                  None if rib is None else dev_bf16(rib))
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    g_codes, g_sb = gpu_quantized_to_numpy(codes_t, scales_t, M, d)
+    o_codes, o_sb = O.quantize_mxfp4(O.round_to_f32(O.rotate(xb, rb, rib)))
+    rep = mismatch_report(g_codes, g_sb, o_codes, o_sb)
+    if check_exact:
+        assert (g_sb == o_sb).all() and (g_codes == o_codes).all()
+    assert rep["non_adjacent"] == 0 and rep["scale_off_by_more_than_one"] == 0, rep
+    assert rep["elem_mismatch_frac"] <= 1e-4, rep
+    assert rep["block_scale_mismatch_frac"] <= 1e-4, rep
+    return g_codes, g_sb, rep
+
+
+def _hadamard(n):
+    H = np.array([[1.0]])
+    while H.shape[0] < n:
+        H = np.block([[H, H], [H, -H]])
+    return H
+
+
+def test_exact_rotations_give_bit_exact_codes():
+    """Permutation and Walsh-Hadamard rotations with small-integer activations: every partial
+    sum is exact in fp32, so codes and scales must equal the oracle's bit for bit.  A non-symmetric
+    permutation also pins the operand orientation of the tensor-core contraction."""
+    d, M = 256, 150
+    g = np.random.default_rng(0)
+    x = g.integers(-8, 9, size=(M, d)).astype(np.float32)
+    xb = I.to_bf16_bits(x)
+    P = np.zeros((d, d), np.float32); P[np.arange(d), g.permutation(d)] = 1
+    Q = np.zeros((d // 32, 32, 32), np.float32)
+    for b in range(d // 32):
+        Q[b, np.arange(32), g.permutation(32)] = 1
+    _rotate_quantize_case(xb, I.to_bf16_bits(P), None, check_exact=True)
+    _rotate_quantize_case(xb, I.to_bf16_bits(P), I.to_bf16_bits(Q), check_exact=True)
+    _rotate_quantize_case(xb, None, I.to_bf16_bits(Q), check_exact=True)
+    H = (_hadamard(d) / 16.0).astype(np.float32)
+    H32 = (_hadamard(32) / 4.0).astype(np.float32)
+    _rotate_quantize_case(xb, I.to_bf16_bits(H), I.to_bf16_bits(np.stack([H32] * (d // 32))), check_exact=True)
+
+
+@pytest.mark.parametrize("M,d", [(64, 256), (1, 256), (130, 512), (257, 320), (100, 64), (33, 1024)])
+def test_random_rotations_small_shapes(M, d):
+    cfg = I.CONFIGS["tiny"]
+    xb = I.activations(cfg, M=M, d=d)
+    rb, rib, _, _ = I.rotations(cfg, d=d)
+    _rotate_quantize_case(xb, rb, rib)
+    _rotate_quantize_case(xb, rb, None)
+
+
+def test_tiny_config_end_to_end():
+    """Config 1: X 64x256 Student-t with 4 outlier channels, W 256x256, fp32 output."""
+    cfg = I.CONFIGS["tiny"]
+    xb = I.activations(cfg)
+    rb, rib, _, _ = I.rotations(cfg)
+    w = I.weights(cfg)
+    w_codes, w_sb = O.prepare_weights(rb, rib, w)
+    Wq, Ws = dev_u8(O.pack_codes(w_codes)), dev_u8(O.swizzle_scales(w_sb, cfg.d, fill=0))
+    dbg_c = torch.empty((cfg.M, cfg.d // 2), dtype=torch.uint8, device="cuda")
+    dbg_s = torch.empty(torq.torq_scales_bytes(cfg.M, cfg.d), dtype=torch.uint8, device="cuda")
+    y = torq.torq_rotated_linear(dev_bf16(xb), dev_bf16(rb), dev_bf16(rib), Wq, Ws, out_dtype=torch.float32,
+                                 dbg_codes=dbg_c, dbg_scales=dbg_s)
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    g_codes, g_sb = gpu_quantized_to_numpy(dbg_c, dbg_s, cfg.M, cfg.d)
+    o_out, o_codes, o_sb = O.rotated_linear(xb, rb, rib, w_codes, w_sb)
+    rep = mismatch_report(g_codes, g_sb, o_codes, o_sb)
+    assert rep["non_adjacent"] == 0 and rep["elem_mismatch_frac"] <= 1e-4, rep
+    # GEMM parity on the operands actually fed
+    ref = O.gemm_dequant(g_codes, g_sb, w_codes, w_sb)
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-3
+    # and the whole layer stays close to the all-oracle result (a few flipped codes at most)
+    assert np.linalg.norm(got - o_out) / np.linalg.norm(o_out) <= 2e-2
+
+
+def test_device_weight_preparation_matches_oracle_weights():
+    cfg = I.CONFIGS["tiny"]
+    rb, rib, _, _ = I.rotations(cfg)
+    w = I.weights(cfg)
+    Wq, Ws = torq.prepare_weights(dev_bf16(rb), dev_bf16(rib), torch.from_numpy(w).cuda())
+    torch.cuda.synchronize()
+    g_codes, g_sb = gpu_quantized_to_numpy(Wq, Ws, cfg.N, cfg.d)
+    o_codes, o_sb = O.prepare_weights(rb, rib, w)
+    rep = mismatch_report(g_codes, g_sb, o_codes, o_sb)
+    assert rep["non_adjacent"] == 0 and rep["elem_mismatch_frac"] <= 1e-3, rep
+
+
+def test_llama3_qkv_shape_sampled_rows():
+    """Config 2 at full size (2048 x 4096 -> 6144): rotate+quantize checked on sampled rows that
+    span several row tiles, the GEMM on the same rows, bf16 output."""
+    cfg = I.CONFIGS["llama3_8b_qkv"]
+    xb = I.activations(cfg)
+    rb, rib, _, _ = I.rotations(cfg)
+    Xd, Rd, Rid = dev_bf16(xb), dev_bf16(rb), dev_bf16(rib)
+    w = I.weights(cfg)
+    Wq, Ws = torq.prepare_weights(Rd, Rid, torch.from_numpy(w).cuda())
+    dbg_c = torch.empty((cfg.M, cfg.d // 2), dtype=torch.uint8, device="cuda")
+    dbg_s = torch.empty(torq.torq_scales_bytes(cfg.M, cfg.d), dtype=torch.uint8, device="cuda")
+    y = torq.torq_rotated_linear(Xd, Rd, Rid, Wq, Ws, out_dtype=torch.bfloat16, dbg_codes=dbg_c, dbg_scales=dbg_s)
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    rows = np.array([0, 1, 127, 128, 129, 640, 1023, 1024, 1777, 2046, 2047])
+    g_codes = O.unpack_codes(dbg_c.cpu().numpy()[rows])
+    g_sb = O.unswizzle_scales(dbg_s.cpu().numpy(), cfg.M, cfg.d)[rows]
+    o_codes, o_sb = O.quantize_mxfp4(O.round_to_f32(O.rotate(xb[rows], rb, rib)))
+    rep = mismatch_report(g_codes, g_sb, o_codes, o_sb)
+    assert rep["non_adjacent"] == 0 and rep["scale_off_by_more_than_one"] == 0, rep
+    assert rep["elem_mismatch_frac"] <= 1e-4 and rep["block_scale_mismatch_frac"] <= 1e-4, rep
+    w_codes, w_sb = gpu_quantized_to_numpy(Wq, Ws, cfg.N, cfg.d)
+    ref = O.round_to_bf16(O.gemm_dequant(g_codes, g_sb, w_codes, w_sb))
+    got = y.float().cpu().numpy()[rows].astype(np.float64)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-3
