@@ -1,0 +1,284 @@
+#!/usr/bin/env python
+"""Benchmark of the rotated-MXFP4 linear hot path (rotate -> MXFP4 quantize -> block-scaled FP4
+GEMM) at the LLaMA3-8B QKV-projection shape (M=2048 tokens, d=4096, N=6144, bf16 output).
+
+One step = one pass of the whole path over one batch of seeded synthetic activations.  Prints ONE
+JSON line (rank 0).  `--impl reference` times the CPU checker (oracle/) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "rotate+MXFP4-quant GB/s and MXFP4 GEMM TFLOP/s, % of roofline (8B shapes)"
+WORKLOAD = "llama3_8b_qkv"
+N_BUFFER_SETS = 4          # rotated between steps: 4 x ~92 MB of operands > 126 MB of L2
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_burst": d["bf16_tflops"], "bf16_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons of one GPU while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def time_oracle(cfg, rows: int, steps: int, warmup: int):
+    """The CPU checker, as it stands, on the first `rows` rows of the workload (every stage is
+    independent per row).  Weight codes are random: their values do not change the run time."""
+    import oracle as O
+    from paper_2605_19561_b200 import inputs as I
+    xb = I.activations(cfg)[:rows]
+    rb, rib, _, _ = I.rotations(cfg)
+    wp, wsb = I.random_codes(cfg.N, cfg.d, seed=3)
+    wc = O.unpack_codes(wp)
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        O.rotated_linear(xb, rb, rib, wc, wsb)
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count()
+    return float(np.mean(times)), cores
+
+
+def run_reference(args):
+    from paper_2605_19561_b200 import inputs as I
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = I.CONFIGS[WORKLOAD]
+    rows = 512
+    t, cores = time_oracle(cfg, rows, max(1, args.steps), min(args.warmup, 1))
+    v = rows / t
+    sample = f"first {rows} of {cfg.M} rows per step, all {cfg.d} features and {cfg.N} outputs"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "M": cfg.M, "d": cfg.d, "N": cfg.N, "sample": sample},
+        "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    from paper_2605_19561_b200 import inputs as I
+    from paper_2605_19561_b200 import torq
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    warmup = max(args.warmup, 3)
+    cfg = I.CONFIGS[WORKLOAD]
+    M, d, N = cfg.M, cfg.d, cfg.N
+    pk = peaks()
+
+    # ---- inputs (seeded, synthetic; every rank holds its own M rows: weak scaling over tokens)
+    xb = I.activations(cfg)
+    rb, rib, _, _ = I.rotations(cfg)
+    w = I.weights(cfg)
+    X0 = I.bf16_bits_to_tensor(xb, "cuda")
+    R0, Ri0 = I.bf16_bits_to_tensor(rb, "cuda"), I.bf16_bits_to_tensor(rib, "cuda")
+    Wq0, Ws0 = torq.prepare_weights(R0, Ri0, torch.from_numpy(w).cuda())
+    sets = []
+    for i in range(N_BUFFER_SETS):
+        sets.append(dict(X=X0.clone(), R=R0.clone(), Ri=Ri0.clone(), Wq=Wq0.clone(), Ws=Ws0.clone(),
+                         Y=torch.empty((M, N), dtype=torch.bfloat16, device="cuda"),
+                         ws=torch.empty(torq.torq_workspace_bytes(M, d, N), dtype=torch.uint8, device="cuda")))
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        b = sets[i % N_BUFFER_SETS]
+        torq.torq_rotated_linear(b["X"], b["R"], b["Ri"], b["Wq"], b["Ws"], Y=b["Y"], workspace=b["ws"])
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(warmup):
+        step(i)
+    barrier()
+    assert torq.torq_last_device_error() == 0
+
+    # ---- timed region: exactly K steps of the whole path, inputs resident in HBM
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = torq.torq_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    launches = torq.torq_launch_count() - launches0
+    ms_total = e0.elapsed_time(e1)
+
+    # ---- per-kernel durations, same launches issued as the two stage calls with events between
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    for i in range(args.steps):
+        b = sets[i % N_BUFFER_SETS]
+        codes = b["ws"][: M * d // 2].view(M, d // 2)
+        scales = b["ws"][(M * d // 2 + 255) // 256 * 256:]
+        ev[i][0].record(stream)
+        torq.torq_rotate_quantize(b["X"], b["R"], b["Ri"], out_codes=codes, out_scales=scales)
+        ev[i][1].record(stream)
+        torq.torq_mxfp4_gemm(codes, scales, b["Wq"], b["Ws"], Y=b["Y"])
+        ev[i][2].record(stream)
+    barrier()
+    clocks = sampler.stop()
+    t_rot = float(np.mean([e[0].elapsed_time(e[1]) for e in ev])) * 1e-3
+    t_gemm = float(np.mean([e[1].elapsed_time(e[2]) for e in ev])) * 1e-3
+    assert torq.torq_last_device_error() == 0
+
+    # ---- end to end through the public call with HOST buffers (pinned), copies inside the region
+    Xh = X0.cpu().pin_memory()
+    Yh = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    e2e_steps = max(3, min(args.steps, 50))
+    b = sets[0]
+    for _ in range(3):
+        b["X"].copy_(Xh, non_blocking=True); step(0); Yh.copy_(b["Y"], non_blocking=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        b["X"].copy_(Xh, non_blocking=True)
+        step(0)
+        Yh.copy_(b["Y"], non_blocking=True)
+    e1.record(stream)
+    barrier()
+    ms_e2e = e0.elapsed_time(e1) / e2e_steps
+
+    t_local = torch.tensor([ms_total, ms_e2e, t_rot, t_gemm], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t_local, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e, t_rot, t_gemm = [float(v) for v in t_local.cpu()]
+    ms_step = ms_total / args.steps
+
+    if rank == 0:
+        rot_flop = 2.0 * M * d * d + 64.0 * M * d
+        rot_bytes = 2.0 * M * d + 2.0 * d * d + 2.0 * 32 * d + M * d / 2 + M * d / 32
+        gemm_flop = 2.0 * M * N * d
+        gemm_bytes = M * d / 2 + M * d / 32 + N * d / 2 + N * d / 32 + 2.0 * M * N
+        fp4_peak = 4.0 * pk["bf16_sustained"]
+        traffic = None
+        tp = os.path.join(ROOT, "profiles", "rotate_quantize_traffic.json")
+        if os.path.exists(tp):
+            traffic = json.load(open(tp)).get("dram_bytes_per_launch")
+        out = {
+            "metric": METRIC, "value": world * M / (ms_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 rotation (fp32 accumulate) + e2m1/E8M0 GEMM",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "M_per_gpu": M, "d": d, "N": N, "out_dtype": "bf16",
+                       "l2": f"{N_BUFFER_SETS} operand sets rotated between steps (working set > 126 MB L2)",
+                       "sharding": "rows (tokens) per GPU, no collective"},
+            "stages": {
+                "rotate_quant": {"ms": t_rot * 1e3, "GB/s": rot_bytes / t_rot / 1e9, "TFLOP/s": rot_flop / t_rot / 1e12,
+                                 "bound": "bf16 tensor", "frac_of_bf16_sustained": rot_flop / t_rot / 1e12 / pk["bf16_sustained"],
+                                 "frac_of_bf16_burst": rot_flop / t_rot / 1e12 / pk["bf16_burst"]},
+                "gemm": {"ms": t_gemm * 1e3, "TFLOP/s": gemm_flop / t_gemm / 1e12, "GB/s": gemm_bytes / t_gemm / 1e9,
+                         "bound": "fp4 tensor", "frac_of_4x_bf16_sustained": gemm_flop / t_gemm / 1e12 / fp4_peak,
+                         "frac_of_nominal_9000": gemm_flop / t_gemm / 1e12 / 9000.0},
+            },
+            "roofline": {"kernel": "rotate_quantize_kernel", "bound": "tensor", "achieved": rot_flop / t_rot / 1e12,
+                         "peak": pk["bf16_sustained"], "unit": "TFLOP/s", "frac": rot_flop / t_rot / 1e12 / pk["bf16_sustained"],
+                         "traffic": traffic, "peak_source": pk["source"] + " bf16 sustained"},
+            "e2e": {"value": world * M / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": Xh.numel() * 2,
+                    "d2h_bytes_per_step": Yh.numel() * 2},
+            "gpu_launches": int(launches), "clocks": clocks,
+        }
+        if not args.no_cpu_baseline:
+            rows = 512
+            t, cores = time_oracle(cfg, rows, 2, 1)
+            out["cpu_baseline"] = {"value": rows / t, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                                   "sample": f"first {rows} of {M} rows, all features and outputs, 2 timed passes"}
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
