@@ -1,0 +1,219 @@
+// Block-scaled MXFP4 GEMM on CTA pairs (M > 128): two CTAs share one 256 x 256 output tile through
+// tcgen05.mma cta_group::2 kind::mxf4.block_scale.  Each CTA stages its own 128 rows of A, its own
+// 128 rows of W, its own A scales and the full tile's W scales (35 KiB per 256 elements of K
+// instead of 51 KiB), six stages deep.  No multicast load.
+//
+// The 128 x 256 fp32 accumulator of each CTA fills half of tensor memory and the scale factors
+// need columns too, so there is a single accumulator buffer; to keep the tensor pipe busy the
+// eight epilogue warps first drain the whole accumulator into registers (128 values per thread),
+// hand it back to the MMA warp at once, and only then convert and store.
+//
+// Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (leader CTA only), warps 2..9 epilogue
+// (warp w reads lane quarter w%4, column half (w-2)/4).  Barriers as in the pair rotation kernel;
+// acc_empty takes one arrival per epilogue warp of both CTAs (16).
+#pragma once
+#include <cuda_bf16.h>
+#include "sm100_ptx.cuh"
+
+namespace torq {
+
+struct GemmPairCfg {
+  static constexpr int BN = 256;
+  static constexpr int BM = 128;                       // rows per CTA
+  static constexpr int BK = 256;
+  static constexpr int A_BYTES = BM * BK / 2;          // 16 KiB
+  static constexpr int B_BYTES = (BN / 2) * BK / 2;    // 16 KiB
+  static constexpr int SFA_BYTES = 1024;
+  static constexpr int SFB_BYTES = 2048;               // both 128-row tiles of the W scales
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;   // 35 KiB
+  static constexpr int STAGES = 6;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + 1024;
+  static constexpr int SFA_COL = 256;
+  static constexpr int SFB_COL = 264;
+  static constexpr int TMEM_COLS = 512;
+  static constexpr int THREADS = 320;
+  static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+};
+
+__global__ void __launch_bounds__(320, 1)
+mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                       const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB,
+                       void* __restrict__ Y, int y_is_bf16, int M, int N, int K, int* err_word) {
+  using C = GemmPairCfg;
+  constexpr int BN = C::BN;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_off = C::STAGES * C::STAGE_BYTES;
+  const uint32_t bar_base = smem_base + bar_off;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };
+  const uint32_t accf_bar = bar_base + 8u * (2 * C::STAGES);
+  const uint32_t acce_bar = bar_base + 8u * (2 * C::STAGES + 1);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + bar_off + 192);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(smem_gen + bar_off + 200);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  const int mp_tiles = (M + 255) / 256;
+  const int n_tiles = (N + BN - 1) / BN;
+  const int total_tiles = mp_tiles * n_tiles;
+  const int k_tiles = (K + C::BK - 1) / C::BK;
+  const int kb4 = K / 128;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(accf_bar, 1);
+    mbar_init(acce_bar, 16);
+    *cta_abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) { tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS); tmem_relinquish_pair(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
+      tma_prefetch_desc(&tmSFA); tma_prefetch_desc(&tmSFB);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
+        const int mt = 2 * (tile % mp_tiles) + (int)rank, nt = tile / mp_tiles;
+        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+          const int s = it % C::STAGES;
+          if (!mbar_wait_cluster(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
+                                 SITE_PRODUCER_EMPTY)) { ok = false; break; }
+          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+          const uint32_t leader_full = map_to_cta(full_bar(s), 0);
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
+          tma_load_2d_pair(st, &tmA, kt * 128, mt * C::BM, leader_full);
+          tma_load_2d_pair(st + C::A_BYTES, &tmB, kt * 128, nt * BN + (int)rank * (BN / 2), leader_full);
+          // scale tiles: one row of the [row tile, K-chunk x 512 B] view per 128 rows, 1 KiB per
+          // stage (two K-chunks); anything outside the buffer arrives as zeros (scale 2^-127,
+          // multiplying operand data that is zero there as well).
+          tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES, &tmSFA, kt * 256, mt, leader_full);
+          tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES, &tmSFB, kt * 256, 2 * nt, leader_full);
+          tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + 1024, &tmSFB, kt * 256, 2 * nt + 1,
+                           leader_full);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader only)
+    if (lane == 0 && rank == 0) {
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total_tiles && ok; tile += npairs, ++tcount) {
+        if (!mbar_wait_cluster(acce_bar, (tcount & 1) ^ 1, cta_abort, err_word, SITE_MMA_ACC_EMPTY)) {
+          ok = false; break;
+        }
+        tc_fence_after_sync();
+        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+          const int s = it % C::STAGES;
+          if (!mbar_wait_cluster(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
+            ok = false; break;
+          }
+          tc_fence_after_sync();
+          const int nchunk = min(2, kb4 - 2 * kt);
+          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+          const uint32_t sfa = st + C::A_BYTES + C::B_BYTES, sfb = sfa + C::SFA_BYTES;
+          for (int c = 0; c < nchunk; ++c) {
+            tmem_cp_32x128b_warpx4_pair(tmem_base + C::SFA_COL + 4 * c, make_desc(sfa + 512 * c, 0, 128, 0));
+            tmem_cp_32x128b_warpx4_pair(tmem_base + C::SFB_COL + 8 * c, make_desc(sfb + 512 * c, 0, 128, 0));
+            tmem_cp_32x128b_warpx4_pair(tmem_base + C::SFB_COL + 8 * c + 4,
+                                        make_desc(sfb + 1024 + 512 * c, 0, 128, 0));
+          }
+          const uint64_t adesc = make_desc(st, 16, 1024, kSwizzle128);
+          const uint64_t bdesc = make_desc(st + C::A_BYTES, 16, 1024, kSwizzle128);
+          for (int j = 0; j < 2 * nchunk; ++j) {
+            const uint32_t id = (j & 1) * 2;
+            mma_mxf4_pair(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc_mxf4(256, BN, id, id),
+                          tmem_base + C::SFA_COL + 4 * (j >> 1), tmem_base + C::SFB_COL + 8 * (j >> 1),
+                          (kt | j) != 0);
+          }
+          tc_commit_pair(empty_bar(s), 3);
+        }
+        if (ok) tc_commit_pair(accf_bar, 3);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (8 warps per CTA)
+    const int q = warp & 3;
+    const int h = (warp - 2) >> 2;                       // column half
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = pair; tile < total_tiles && ok; tile += npairs, ++tcount) {
+      const int mt = 2 * (tile % mp_tiles) + (int)rank, nt = tile / mp_tiles;
+      ok = mbar_wait_cluster(accf_bar, tcount & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + h * 128;
+      uint32_t v0[32], v1[32], v2[32], v3[32];
+      tmem_ld_32x32(tacc, v0);
+      tmem_ld_32x32(tacc + 32, v1);
+      tmem_ld_32x32(tacc + 64, v2);
+      tmem_ld_32x32(tacc + 96, v3);
+      tmem_ld_wait();
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar, 0));   // accumulator is free again
+      const int64_t row = (int64_t)mt * C::BM + q * 32 + lane;
+      const int64_t col0 = (int64_t)nt * BN + h * 128;
+      if (row < M) {
+        auto store32 = [&](const uint32_t (&v)[32], int64_t col) {
+          if (col >= N) return;
+          if (y_is_bf16) {
+            __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(Y) + row * N + col;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              if (col + 8 * g + 8 <= N) {
+                uint4 o;
+                uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                  __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[8 * g + 2 * p]),
+                                                            __uint_as_float(v[8 * g + 2 * p + 1]));
+                  ow[p] = *reinterpret_cast<uint32_t*>(&hh);
+                }
+                *reinterpret_cast<uint4*>(yp + 8 * g) = o;
+              }
+            }
+          } else {
+            float* yp = reinterpret_cast<float*>(Y) + row * N + col;
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+              if (col + 4 * g + 4 <= N)
+                *reinterpret_cast<uint4*>(yp + 4 * g) =
+                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+            }
+          }
+        };
+        store32(v0, col0);
+        store32(v1, col0 + 32);
+        store32(v2, col0 + 64);
+        store32(v3, col0 + 96);
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before_sync();
+  __syncthreads();
+  if (*cta_abort) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+  }
+}
+
+}  // namespace torq

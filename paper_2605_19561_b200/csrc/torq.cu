@@ -7,8 +7,10 @@
 
 #include "../../include/torq.h"
 #include "mxfp4_gemm.cuh"
+#include "mxfp4_gemm_pair.cuh"
 #include "quantize.cuh"
 #include "rotate_quantize.cuh"
+#include "rotate_quantize_pair.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -20,6 +22,8 @@ struct DeviceState {
   bool ready = false;
   bool arch_ok = false;
   int sm_count = 0;
+  int rot_pairs = 0;    // CTA pairs of the pair kernels that can be resident at once
+  int gemm_pairs = 0;
   int* err_word = nullptr;
 };
 static DeviceState g_dev[kMaxDevices];
@@ -36,6 +40,26 @@ template <typename K>
 static bool opt_in_smem(K kernel, int bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) ==
          cudaSuccess;
+}
+
+// How many 2-CTA clusters of `kernel` fit on the device at once (GPC boundaries can leave a few
+// SMs unpaired, so this may be below sm_count / 2).
+template <typename K>
+static int max_active_pairs(K kernel, int threads, int smem, int sm_count) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(sm_count / 2 * 2), 1, 1);
+  cfg.blockDim = dim3((unsigned)threads, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) return 0;
+  return n < sm_count / 2 ? n : sm_count / 2;
 }
 
 // Per-device one-time set-up: architecture check, SM count, error-word address, shared-memory
@@ -66,8 +90,15 @@ static DeviceState* device_state() {
     bool ok = opt_in_smem(mxfp4_gemm_kernel<256, 1>, GemmCfg<256, 1>::SMEM_BYTES) &&
               opt_in_smem(mxfp4_gemm_kernel<128, 2>, GemmCfg<128, 2>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_kernel<256>, RotCfg<256>::SMEM_BYTES) &&
-              opt_in_smem(rotate_quantize_kernel<128>, RotCfg<128>::SMEM_BYTES);
+              opt_in_smem(rotate_quantize_kernel<128>, RotCfg<128>::SMEM_BYTES) &&
+              opt_in_smem(rotate_quantize_pair_kernel, RotPairCfg::SMEM_BYTES) &&
+              opt_in_smem(mxfp4_gemm_pair_kernel, GemmPairCfg::SMEM_BYTES);
     if (!ok) return nullptr;
+    st.rot_pairs = max_active_pairs(rotate_quantize_pair_kernel, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
+                                    st.sm_count);
+    st.gemm_pairs = max_active_pairs(mxfp4_gemm_pair_kernel, GemmPairCfg::THREADS, GemmPairCfg::SMEM_BYTES,
+                                     st.sm_count);
+    if (st.rot_pairs < 1 || st.gemm_pairs < 1) return nullptr;
   }
   st.ready = true;
   return &st;
@@ -76,13 +107,14 @@ static DeviceState* device_state() {
 // 2-D row-major tensor [rows, cols] of `elem_bytes`-byte elements, box [box_rows, box_cols],
 // 128-byte swizzle, zero fill outside the tensor.
 static bool encode_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* base,
-                      uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols) {
+                      uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols,
+                      CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
   cuuint64_t dims[2] = {cols, rows};
   cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
   cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
   return g_encode(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -95,6 +127,25 @@ static inline int ew_grid(int64_t items, int per_block, int sm_count) {
 static inline torq_status launch_status() {
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return cudaGetLastError() == cudaSuccess ? TORQ_OK : TORQ_ERR_LAUNCH;
+}
+
+// Launch with a cluster of two CTAs along x (grid must be even).
+template <typename... KArgs, typename... Args>
+static void launch_pair(void (*kernel)(KArgs...), int grid, int threads, int smem, cudaStream_t s,
+                        Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3((unsigned)threads, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 static torq_status quantize_impl(DeviceState* st, const void* Z, torq_dtype dt, int64_t M, int64_t d,
@@ -199,6 +250,15 @@ torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void*
   if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d, 128, 64) ||
       !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
     return TORQ_ERR_LAUNCH;
+  if (M > 128) {
+    // CTA pairs: 256 x 256 tiles, one pair per two SMs.
+    const int ptiles = (int)((M + 255) / 256) * (int)((d + 255) / 256);
+    const int max_pairs = st->rot_pairs;
+    const int pairs = ptiles < max_pairs ? ptiles : max_pairs;
+    launch_pair(rotate_quantize_pair_kernel, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES, s, tmX,
+                tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, st->err_word);
+    return launch_status();
+  }
   const int m_tiles = (int)((M + 127) / 128);
   const int tiles = m_tiles * (int)((d + 255) / 256);
   const int grid = tiles < st->sm_count ? tiles : st->sm_count;
@@ -222,6 +282,23 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   constexpr int BN = 256;
   CUtensorMap tmA, tmB;
+  if (M > 128) {
+    CUtensorMap tmSFA, tmSFB;
+    const uint64_t kb4 = (uint64_t)(K / 128);
+    if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, (uint64_t)(K / 2), 128, 128) ||
+        !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)(K / 2), BN / 2, 128) ||
+        !encode_2d(&tmSFA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, As, (uint64_t)((M + 127) / 128), kb4 * 128, 1, 256,
+                   CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !encode_2d(&tmSFB, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, Ws, (uint64_t)((N + 127) / 128), kb4 * 128, 1, 256,
+                   CU_TENSOR_MAP_SWIZZLE_NONE))
+      return TORQ_ERR_LAUNCH;
+    const int ptiles = (int)((M + 255) / 256) * (int)((N + BN - 1) / BN);
+    const int max_pairs = st->gemm_pairs;
+    const int pairs = ptiles < max_pairs ? ptiles : max_pairs;
+    launch_pair(mxfp4_gemm_pair_kernel, 2 * pairs, GemmPairCfg::THREADS, GemmPairCfg::SMEM_BYTES, s, tmA, tmB,
+                tmSFA, tmSFB, Y, y_dtype == TORQ_BF16 ? 1 : 0, (int)M, (int)N, (int)K, st->err_word);
+    return launch_status();
+  }
   if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, (uint64_t)(K / 2), 128, 128) ||
       !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)(K / 2), BN, 128))
     return TORQ_ERR_LAUNCH;
