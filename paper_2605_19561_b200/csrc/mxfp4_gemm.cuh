@@ -78,22 +78,21 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&tmA);
-      tma_prefetch_desc(&tmB);
-      uint32_t it = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int mt = tile % m_tiles, nt = tile / m_tiles;
-        const int rt0 = nt * (BN / 128);
-        const int n_sfb_tiles = min(BN / 128, n_rowtiles - rt0);
-        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
-          const int s = it % C::STAGES;
-          if (!mbar_wait(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
-                         SITE_PRODUCER_EMPTY)) { ok = false; break; }
-          const int nchunk = min(2, kb4 - 2 * kt);
-          const uint32_t sf_bytes = 512u * nchunk;
-          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+    if (elect_one()) { tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB); }
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int mt = tile % m_tiles, nt = tile / m_tiles;
+      const int rt0 = nt * (BN / 128);
+      const int n_sfb_tiles = min(BN / 128, n_rowtiles - rt0);
+      for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+        const int s = it % C::STAGES;
+        if (!mbar_wait_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
+                       SITE_PRODUCER_EMPTY)) { ok = false; break; }
+        const int nchunk = min(2, kb4 - 2 * kt);
+        const uint32_t sf_bytes = 512u * nchunk;
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        if (elect_one()) {
           mbar_arrive_expect_tx(full_bar(s), C::A_BYTES + C::B_BYTES + sf_bytes * (1 + n_sfb_tiles));
           tma_load_2d(st, &tmA, kt * 128, mt * C::BM, full_bar(s));
           tma_load_2d(st + C::A_BYTES, &tmB, kt * 128, nt * BN, full_bar(s));
@@ -103,47 +102,57 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             bulk_load_1d(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * 1024,
                          Ws + ((size_t)(rt0 + t) * kb4 + 2 * kt) * 512, sf_bytes, full_bar(s));
         }
+        __syncwarp();
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      uint32_t it = 0, tcount = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-        const int a = tcount % NACC;
-        if (!mbar_wait(acce_bar(a), ((tcount / NACC) & 1) ^ 1, cta_abort, err_word,
-                       SITE_MMA_ACC_EMPTY)) { ok = false; break; }
+    uint32_t it = 0, tcount = 0;
+    bool ok = true;
+    constexpr uint32_t idesc0 = idesc_mxf4(128, BN, 0, 0), idesc2 = idesc_mxf4(128, BN, 2, 2);
+    const uint32_t sfa_t = tmem_base + C::SFA_COL, sfb_t = tmem_base + C::SFB_COL;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      const int a = tcount % NACC;
+      if (!mbar_wait_warp(acce_bar(a), ((tcount / NACC) & 1) ^ 1, cta_abort, err_word,
+                     SITE_MMA_ACC_EMPTY)) { ok = false; break; }
+      tc_fence_after_sync();
+      const uint32_t acc = tmem_base + a * BN;
+      for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+        const int s = it % C::STAGES;
+        if (!mbar_wait_warp(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
+          ok = false; break;
+        }
         tc_fence_after_sync();
-        const uint32_t acc = tmem_base + a * BN;
-        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
-          const int s = it % C::STAGES;
-          if (!mbar_wait(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
-            ok = false; break;
-          }
-          tc_fence_after_sync();
-          const int nchunk = min(2, kb4 - 2 * kt);
-          const uint32_t st = smem_base + s * C::STAGE_BYTES;
-          const uint32_t sfa = st + C::A_BYTES + C::B_BYTES, sfb = sfa + C::SFA_BYTES;
-          for (int c = 0; c < nchunk; ++c) {
-            tmem_cp_32x128b_warpx4(tmem_base + C::SFA_COL + 4 * c, make_desc(sfa + 512 * c, 0, 128, 0));
+        const bool two = (kb4 - 2 * kt) >= 2;              // K % 256 == 128: the last stage is half
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        const uint64_t adesc = make_desc(st, 16, 1024, kSwizzle128);
+        const uint64_t bdesc = make_desc(st + C::A_BYTES, 16, 1024, kSwizzle128);
+        const uint64_t sfa_d = make_desc(st + C::A_BYTES + C::B_BYTES, 0, 128, 0);
+        const uint64_t sfb_d = make_desc(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES, 0, 128, 0);
+        if (elect_one()) {
+          // scale tiles shared -> tensor memory (descriptor address unit = 16 B: +32 = next
+          // K-chunk, +64 = next 128-row tile of W), then 64 elements of K per instruction
 #pragma unroll
-            for (int t = 0; t < BN / 128; ++t)
-              tmem_cp_32x128b_warpx4(tmem_base + C::SFB_COL + c * (BN / 32) + 4 * t,
-                                     make_desc(sfb + 1024 * t + 512 * c, 0, 128, 0));
+          for (int c = 0; c < 2; ++c) {
+            if (c == 0 || two) {
+              tmem_cp_32x128b_warpx4(sfa_t + 4 * c, sfa_d + 32 * c);
+#pragma unroll
+              for (int t = 0; t < BN / 128; ++t)
+                tmem_cp_32x128b_warpx4(sfb_t + c * (BN / 32) + 4 * t, sfb_d + 64 * t + 32 * c);
+            }
           }
-          const uint64_t adesc = make_desc(st, 16, 1024, kSwizzle128);
-          const uint64_t bdesc = make_desc(st + C::A_BYTES, 16, 1024, kSwizzle128);
-          for (int j = 0; j < 2 * nchunk; ++j) {        // 64 elements (32 bytes) of K each
-            const uint32_t id = (j & 1) * 2;
-            mma_mxf4(acc, adesc + 2 * j, bdesc + 2 * j, idesc_mxf4(128, BN, id, id),
-                     tmem_base + C::SFA_COL + 4 * (j >> 1),
-                     tmem_base + C::SFB_COL + (j >> 1) * (BN / 32), (kt | j) != 0);
+          mma_mxf4(acc, adesc, bdesc, idesc0, sfa_t, sfb_t, kt != 0);
+          mma_mxf4(acc, adesc + 2, bdesc + 2, idesc2, sfa_t, sfb_t, 1);
+          if (two) {
+            mma_mxf4(acc, adesc + 4, bdesc + 4, idesc0, sfa_t + 4, sfb_t + BN / 32, 1);
+            mma_mxf4(acc, adesc + 6, bdesc + 6, idesc2, sfa_t + 4, sfb_t + BN / 32, 1);
           }
           tc_commit(empty_bar(s));
         }
-        if (ok) tc_commit(accf_bar(a));
+        __syncwarp();
       }
+      if (ok && elect_one()) tc_commit(accf_bar(a));
+      __syncwarp();
     }
   } else {
     // ------------------------------------------------------------------ epilogue

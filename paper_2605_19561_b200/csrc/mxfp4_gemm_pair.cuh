@@ -78,19 +78,21 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
-    if (lane == 0) {
+    if (elect_one()) {
       tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
       tma_prefetch_desc(&tmSFA); tma_prefetch_desc(&tmSFB);
-      uint32_t it = 0;
-      bool ok = true;
-      for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
-        const int mt = 2 * (tile % mp_tiles) + (int)rank, nt = tile / mp_tiles;
-        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
-          const int s = it % C::STAGES;
-          if (!mbar_wait_cluster(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
-                                 SITE_PRODUCER_EMPTY)) { ok = false; break; }
-          const uint32_t st = smem_base + s * C::STAGE_BYTES;
-          const uint32_t leader_full = map_to_cta(full_bar(s), 0);
+    }
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
+      const int mt = 2 * (tile % mp_tiles) + (int)rank, nt = tile / mp_tiles;
+      for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+        const int s = it % C::STAGES;
+        if (!mbar_wait_cluster_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
+                               SITE_PRODUCER_EMPTY)) { ok = false; break; }
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        const uint32_t leader_full = map_to_cta(full_bar(s), 0);
+        if (elect_one()) {
           if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
           tma_load_2d_pair(st, &tmA, kt * 128, mt * C::BM, leader_full);
           tma_load_2d_pair(st + C::A_BYTES, &tmB, kt * 128, nt * BN + (int)rank * (BN / 2), leader_full);
@@ -102,44 +104,56 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + 1024, &tmSFB, kt * 256, 2 * nt + 1,
                            leader_full);
         }
+        __syncwarp();
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader only)
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
       uint32_t it = 0, tcount = 0;
       bool ok = true;
+      constexpr uint32_t idesc0 = idesc_mxf4(256, BN, 0, 0), idesc2 = idesc_mxf4(256, BN, 2, 2);
+      const uint32_t sfa_t = tmem_base + C::SFA_COL, sfb_t = tmem_base + C::SFB_COL;
       for (int tile = pair; tile < total_tiles && ok; tile += npairs, ++tcount) {
-        if (!mbar_wait_cluster(acce_bar, (tcount & 1) ^ 1, cta_abort, err_word, SITE_MMA_ACC_EMPTY)) {
+        if (!mbar_wait_cluster_warp(acce_bar, (tcount & 1) ^ 1, cta_abort, err_word, SITE_MMA_ACC_EMPTY)) {
           ok = false; break;
         }
         tc_fence_after_sync();
         for (int kt = 0; kt < k_tiles; ++kt, ++it) {
           const int s = it % C::STAGES;
-          if (!mbar_wait_cluster(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
+          if (!mbar_wait_cluster_warp(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
             ok = false; break;
           }
           tc_fence_after_sync();
-          const int nchunk = min(2, kb4 - 2 * kt);
+          const bool two = (kb4 - 2 * kt) >= 2;            // K % 256 == 128: the last stage is half
           const uint32_t st = smem_base + s * C::STAGE_BYTES;
-          const uint32_t sfa = st + C::A_BYTES + C::B_BYTES, sfb = sfa + C::SFA_BYTES;
-          for (int c = 0; c < nchunk; ++c) {
-            tmem_cp_32x128b_warpx4_pair(tmem_base + C::SFA_COL + 4 * c, make_desc(sfa + 512 * c, 0, 128, 0));
-            tmem_cp_32x128b_warpx4_pair(tmem_base + C::SFB_COL + 8 * c, make_desc(sfb + 512 * c, 0, 128, 0));
-            tmem_cp_32x128b_warpx4_pair(tmem_base + C::SFB_COL + 8 * c + 4,
-                                        make_desc(sfb + 1024 + 512 * c, 0, 128, 0));
-          }
           const uint64_t adesc = make_desc(st, 16, 1024, kSwizzle128);
           const uint64_t bdesc = make_desc(st + C::A_BYTES, 16, 1024, kSwizzle128);
-          for (int j = 0; j < 2 * nchunk; ++j) {
-            const uint32_t id = (j & 1) * 2;
-            mma_mxf4_pair(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc_mxf4(256, BN, id, id),
-                          tmem_base + C::SFA_COL + 4 * (j >> 1), tmem_base + C::SFB_COL + 8 * (j >> 1),
-                          (kt | j) != 0);
+          const uint64_t sfa_d = make_desc(st + C::A_BYTES + C::B_BYTES, 0, 128, 0);
+          const uint64_t sfb_d = make_desc(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES, 0, 128, 0);
+          if (elect_one()) {
+            // scale tiles shared -> tensor memory (descriptor address unit = 16 B: +32 = next
+            // K-chunk, +64 = second 128-row tile of W), then 64 elements of K per instruction
+            tmem_cp_32x128b_warpx4_pair(sfa_t, sfa_d);
+            tmem_cp_32x128b_warpx4_pair(sfb_t, sfb_d);
+            tmem_cp_32x128b_warpx4_pair(sfb_t + 4, sfb_d + 64);
+            if (two) {
+              tmem_cp_32x128b_warpx4_pair(sfa_t + 4, sfa_d + 32);
+              tmem_cp_32x128b_warpx4_pair(sfb_t + 8, sfb_d + 32);
+              tmem_cp_32x128b_warpx4_pair(sfb_t + 12, sfb_d + 96);
+            }
+            mma_mxf4_pair(tmem_base, adesc, bdesc, idesc0, sfa_t, sfb_t, kt != 0);
+            mma_mxf4_pair(tmem_base, adesc + 2, bdesc + 2, idesc2, sfa_t, sfb_t, 1);
+            if (two) {
+              mma_mxf4_pair(tmem_base, adesc + 4, bdesc + 4, idesc0, sfa_t + 4, sfb_t + 8, 1);
+              mma_mxf4_pair(tmem_base, adesc + 6, bdesc + 6, idesc2, sfa_t + 4, sfb_t + 8, 1);
+            }
+            tc_commit_pair(empty_bar(s), 3);
           }
-          tc_commit_pair(empty_bar(s), 3);
+          __syncwarp();
         }
-        if (ok) tc_commit_pair(accf_bar, 3);
+        if (ok && elect_one()) tc_commit_pair(accf_bar, 3);
+        __syncwarp();
       }
     }
   } else {

@@ -78,18 +78,17 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&tmX);
-      tma_prefetch_desc(&tmR);
-      uint32_t it = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int mt = tile % m_tiles, nt = tile / m_tiles;
-        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
-          const int s = it % C::STAGES;
-          if (!mbar_wait(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
-                         SITE_PRODUCER_EMPTY)) { ok = false; break; }
-          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+    if (elect_one()) { tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmR); }
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int mt = tile % m_tiles, nt = tile / m_tiles;
+      for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+        const int s = it % C::STAGES;
+        if (!mbar_wait_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
+                       SITE_PRODUCER_EMPTY)) { ok = false; break; }
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        if (elect_one()) {
           mbar_arrive_expect_tx(full_bar(s), C::STAGE_BYTES);
           tma_load_2d(st, &tmX, kt * C::BK, mt * C::BM, full_bar(s));
 #pragma unroll
@@ -97,41 +96,44 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             tma_load_2d(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR, nt * BN + b * 64, kt * C::BK,
                         full_bar(s));
         }
+        __syncwarp();
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(128, BN, /*A MN-major*/ false, /*B MN-major*/ true);
-      uint32_t it = 0, tcount = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-        const int a = tcount % C::NACC;
-        if (!mbar_wait(acce_bar(a), ((tcount / C::NACC) & 1) ^ 1, cta_abort, err_word,
-                       SITE_MMA_ACC_EMPTY)) { ok = false; break; }
+    constexpr uint32_t idesc = idesc_bf16(128, BN, /*A MN-major*/ false, /*B MN-major*/ true);
+    uint32_t it = 0, tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      const int a = tcount % C::NACC;
+      if (!mbar_wait_warp(acce_bar(a), ((tcount / C::NACC) & 1) ^ 1, cta_abort, err_word,
+                     SITE_MMA_ACC_EMPTY)) { ok = false; break; }
+      tc_fence_after_sync();
+      const uint32_t acc = tmem_base + a * BN;
+      for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+        const int s = it % C::STAGES;
+        if (!mbar_wait_warp(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
+          ok = false; break;
+        }
         tc_fence_after_sync();
-        const uint32_t acc = tmem_base + a * BN;
-        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
-          const int s = it % C::STAGES;
-          if (!mbar_wait(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
-            ok = false; break;
-          }
-          tc_fence_after_sync();
-          const uint32_t st = smem_base + s * C::STAGE_BYTES;
-          // A: K-major, rows of 128 B, 8-row groups 1024 B apart.
-          const uint64_t adesc = make_desc(st, 16, 1024, kSwizzle128);
-          // B: N-major.  64 n-elements (128 B) contiguous, k rows 128 B apart, 8-row groups
-          // 1024 B apart (stride offset), next 64 n-elements one box (8 KiB) further (leading
-          // offset).
-          const uint64_t bdesc = make_desc(st + C::A_BYTES, C::B_BOX_BYTES, 1024, kSwizzle128);
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        // A: K-major, rows of 128 B, 8-row groups 1024 B apart.
+        const uint64_t adesc = make_desc(st, 16, 1024, kSwizzle128);
+        // B: N-major.  64 n-elements (128 B) contiguous, k rows 128 B apart, 8-row groups
+        // 1024 B apart (stride offset), next 64 n-elements one box (8 KiB) further (leading
+        // offset).
+        const uint64_t bdesc = make_desc(st + C::A_BYTES, C::B_BOX_BYTES, 1024, kSwizzle128);
+        if (elect_one()) {
 #pragma unroll
           for (int j = 0; j < C::BK / 16; ++j)          // K = 16 per instruction
             mma_bf16(acc, adesc + 2 * j /* 32 B */, bdesc + 128 * j /* 16 k-rows = 2 KiB */, idesc,
                      (kt | j) != 0);
           tc_commit(empty_bar(s));
         }
-        if (ok) tc_commit(accf_bar(a));
+        __syncwarp();
       }
+      if (ok && elect_one()) tc_commit(accf_bar(a));
+      __syncwarp();
     }
   } else {
     // ------------------------------------------------------------------ epilogue (128 threads)

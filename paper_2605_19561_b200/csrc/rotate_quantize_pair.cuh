@@ -80,19 +80,18 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
-    if (lane == 0) {
-      tma_prefetch_desc(&tmX);
-      tma_prefetch_desc(&tmR);
-      uint32_t it = 0;
-      bool ok = true;
-      for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
-        const int mt = 2 * (tile % mp_tiles) + (int)rank, nt = tile / mp_tiles;
-        for (int kt = 0; kt < k_tiles; ++kt, ++it) {
-          const int s = it % C::STAGES;
-          if (!mbar_wait_cluster(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
-                                 SITE_PRODUCER_EMPTY)) { ok = false; break; }
-          const uint32_t st = smem_base + s * C::STAGE_BYTES;
-          const uint32_t leader_full = map_to_cta(full_bar(s), 0);
+    if (elect_one()) { tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmR); }
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
+      const int mt = 2 * (tile % mp_tiles) + (int)rank, nt = tile / mp_tiles;
+      for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+        const int s = it % C::STAGES;
+        if (!mbar_wait_cluster_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
+                               SITE_PRODUCER_EMPTY)) { ok = false; break; }
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        const uint32_t leader_full = map_to_cta(full_bar(s), 0);
+        if (elect_one()) {
           if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
           tma_load_2d_pair(st, &tmX, kt * C::BK, mt * C::BM, leader_full);
 #pragma unroll
@@ -100,35 +99,40 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
             tma_load_2d_pair(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR,
                              nt * BN + (int)rank * (BN / 2) + b * 64, kt * C::BK, leader_full);
         }
+        __syncwarp();
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader only)
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
       constexpr uint32_t idesc = idesc_bf16(256, BN, /*A MN-major*/ false, /*B MN-major*/ true);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int tile = pair; tile < total_tiles && ok; tile += npairs, ++tcount) {
         const int a = tcount % C::NACC;
-        if (!mbar_wait_cluster(acce_bar(a), ((tcount / C::NACC) & 1) ^ 1, cta_abort, err_word,
+        if (!mbar_wait_cluster_warp(acce_bar(a), ((tcount / C::NACC) & 1) ^ 1, cta_abort, err_word,
                                SITE_MMA_ACC_EMPTY)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t acc = tmem_base + a * BN;
         for (int kt = 0; kt < k_tiles; ++kt, ++it) {
           const int s = it % C::STAGES;
-          if (!mbar_wait_cluster(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
+          if (!mbar_wait_cluster_warp(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
             ok = false; break;
           }
           tc_fence_after_sync();
           const uint32_t st = smem_base + s * C::STAGE_BYTES;
           const uint64_t adesc = make_desc(st, 16, 1024, kSwizzle128);
           const uint64_t bdesc = make_desc(st + C::A_BYTES, C::B_BOX_BYTES, 1024, kSwizzle128);
+          if (elect_one()) {
 #pragma unroll
-          for (int j = 0; j < C::BK / 16; ++j)
-            mma_bf16_pair(acc, adesc + 2 * j, bdesc + 128 * j, idesc, (kt | j) != 0);
-          tc_commit_pair(empty_bar(s), 3);             // stage free in both CTAs
+            for (int j = 0; j < C::BK / 16; ++j)
+              mma_bf16_pair(acc, adesc + 2 * j, bdesc + 128 * j, idesc, (kt | j) != 0);
+            tc_commit_pair(empty_bar(s), 3);             // stage free in both CTAs
+          }
+          __syncwarp();
         }
-        if (ok) tc_commit_pair(accf_bar(a), 3);        // accumulator ready in both CTAs
+        if (ok && elect_one()) tc_commit_pair(accf_bar(a), 3);   // accumulator ready in both CTAs
+        __syncwarp();
       }
     }
   } else {

@@ -73,6 +73,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// ---- single-lane election -----------------------------------------------------------------------
+// The producer and MMA warps walk their loops with all 32 lanes, so that every address, descriptor
+// and loop counter is warp-uniform, and only the TMA / tcgen05 instructions themselves are issued
+// by one elected lane.  (Running the whole loop inside an `if (lane == 0)` branch instead makes
+// the operands of those instructions per-thread values; issuing them then costs a few hundred
+// cycles each and the tensor pipe starves.)
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(pred));
+  return pred != 0;
+}
+
 // ---- proxies / fences -------------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -187,6 +200,13 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
 }
 
 
+// Whole-warp forms of the bounded waits: every lane waits, and all lanes agree on the outcome so
+// that the warp stays converged for the election that follows.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* cta_abort,
+                                               int* err_word, int site) {
+  return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, cta_abort, err_word, site));
+}
+
 // ---- CTA pairs (cluster of two CTAs driving one tcgen05 MMA with cta_group::2) -----------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -236,6 +256,10 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait_cluster_warp(uint32_t bar, uint32_t parity,
+                                                       volatile int* cta_abort, int* err_word, int site) {
+  return __all_sync(0xFFFFFFFFu, mbar_wait_cluster(bar, parity, cta_abort, err_word, site));
 }
 // 2-D tiled load into THIS CTA's shared memory whose completion bytes are counted on a barrier
 // that may live in the other CTA of the pair (`bar_cluster_addr` from map_to_cta).  No multicast.
