@@ -82,6 +82,40 @@ torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* 
                                 size_t workspace_bytes, void* dbg_codes, void* dbg_scales,
                                 void* stream);
 
+/* The whole layer for callers that must not allocate device memory.  (No counterpart in the
+ * paper: this exists for the library's users, not for the method.)
+ *
+ * torq_rotated_linear needs a scratch buffer for the quantized activations, and normally the
+ * caller allocates it.  Some callers cannot: a plug-in or custom operator that an inference
+ * engine hands nothing but input and output pointers; a serving process whose whole device
+ * budget was given to a KV-cache pool at start-up, where a late cudaMalloc fails or evicts;
+ * a latency-critical decode loop, where the implicit device-wide synchronisation of
+ * cudaMalloc / cudaFree is not acceptable.  For them this entry point keeps the scratch in a
+ * fixed array of TORQ_STATIC_WORKSPACE_BYTES that is part of the library image: every device
+ * that loads the library holds those bytes from load until the process exits, used or not.
+ * The call itself allocates nothing and frees nothing, on the host or the device, and neither
+ * does anything it calls.
+ *
+ * Same arguments, layouts and results as torq_rotated_linear without its workspace and debug
+ * parameters.  A problem whose scratch need, torq_workspace_bytes(M, d, N), exceeds
+ * TORQ_STATIC_WORKSPACE_BYTES is refused with TORQ_ERR_WORKSPACE before anything is launched
+ * (for example M = 2048, d = 14336 fits; M = 8192, d = 5120 does not).
+ *
+ * First call on each device: the library looks up the array's device address (and, if no other
+ * entry point ran before, performs the one-time per-device set-up every entry point shares).
+ * Make that first call during start-up, outside any stream capture.
+ *
+ * All calls on a device share the one array, and it keeps whatever the previous call left.
+ * Nothing in it has to start at zero: the rotation step rewrites every code and scale byte the
+ * multiplication step reads before it reads them, so stale contents are never observed.  But two
+ * calls that can overlap on the GPU (different streams, or different host threads without
+ * ordering between them) write the same bytes and race; run them in one stream or order them
+ * with events.  Calls on different devices do not interact. */
+#define TORQ_STATIC_WORKSPACE_BYTES (16u << 20)
+torq_status torq_rotated_linear_static(const void* X, const void* R_inter, const void* R_intra,
+                                       const void* Wq, const void* Ws, int64_t M, int64_t d,
+                                       int64_t N, void* Y, torq_dtype y_dtype, void* stream);
+
 /* Eq. 1 alone: quantize Z [M, d] (fp32 or bf16) to MXFP4.  On fp32 input the result is defined
  * bit for bit (round to nearest even on the e2m1 grid, saturation to +-6, sign bit kept). */
 torq_status torq_quantize_mxfp4(const void* Z, torq_dtype z_dtype, int64_t M, int64_t d,

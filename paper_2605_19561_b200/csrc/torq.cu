@@ -335,6 +335,43 @@ torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* 
   return TORQ_OK;
 }
 
+// ---- the layer without any allocation -----------------------------------------------------------
+// Scratch for torq_rotated_linear_static.  In host code this name is only a handle for the
+// runtime's symbol table, not an address a kernel can use: the device address comes from
+// cudaGetSymbolAddress, once per device, with that device current.
+static __device__ __align__(256) uint8_t g_static_workspace[TORQ_STATIC_WORKSPACE_BYTES];
+static void* g_static_workspace_addr[torq::kMaxDevices] = {};
+static std::mutex g_static_workspace_mutex;
+
+// Device address of the scratch array on the current device (nullptr when CUDA reports an error).
+static void* static_workspace_address() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= torq::kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_static_workspace_mutex);
+  if (!g_static_workspace_addr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();                    // leave no sticky-looking error behind for the caller
+      return nullptr;
+    }
+    g_static_workspace_addr[dev] = p;
+  }
+  return g_static_workspace_addr[dev];
+}
+
+torq_status torq_rotated_linear_static(const void* X, const void* R_inter, const void* R_intra,
+                                       const void* Wq, const void* Ws, int64_t M, int64_t d,
+                                       int64_t N, void* Y, torq_dtype y_dtype, void* stream) {
+  if (!X || !Wq || !Ws || !Y) return TORQ_ERR_NULL;
+  if (M < 1 || d < 128 || d % 128 != 0 || N < 8 || N % 8 != 0 || M > (1 << 30) || d > (1 << 24))
+    return TORQ_ERR_SHAPE;
+  if (torq_workspace_bytes(M, d, N) > (size_t)TORQ_STATIC_WORKSPACE_BYTES) return TORQ_ERR_WORKSPACE;
+  void* scratch = static_workspace_address();
+  if (!scratch) return TORQ_ERR_LAUNCH;
+  return torq_rotated_linear(X, R_inter, R_intra, Wq, Ws, M, d, N, Y, y_dtype, scratch,
+                             (size_t)TORQ_STATIC_WORKSPACE_BYTES, nullptr, nullptr, stream);
+}
+
 torq_status torq_swizzle_scales(const void* linear_scales, int64_t rows, int64_t k, void* out,
                                 void* stream) {
   if (!linear_scales || !out) return TORQ_ERR_NULL;

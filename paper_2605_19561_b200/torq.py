@@ -40,6 +40,8 @@ def lib() -> ctypes.CDLL:
     L.torq_mxfp4_gemm.restype = ci
     L.torq_rotated_linear.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, vp, sz, vp, vp, vp]
     L.torq_rotated_linear.restype = ci
+    L.torq_rotated_linear_static.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, vp]
+    L.torq_rotated_linear_static.restype = ci
     L.torq_quantize_mxfp4.argtypes = [vp, ci, i64, i64, vp, vp, vp]
     L.torq_quantize_mxfp4.restype = ci
     L.torq_scales_bytes.argtypes = [i64, i64]
@@ -163,6 +165,31 @@ def torq_rotated_linear(X, R_inter, R_intra, Wq, Ws, out_dtype=torch.bfloat16, Y
     _raise(lib().torq_rotated_linear(_ptr(X), _ptr(R_inter), _ptr(R_intra), _ptr(Wq), _ptr(Ws), M, d, N,
                                      _ptr(Y), dt, _ptr(workspace), workspace.numel(), _ptr(dbg_codes),
                                      _ptr(dbg_scales), _stream(stream)), "torq_rotated_linear")
+    return Y
+
+
+TORQ_STATIC_WORKSPACE_BYTES = 16 << 20
+
+
+def torq_rotated_linear_static(X, R_inter, R_intra, Wq, Ws, Y, stream=None):
+    """The whole layer for callers that cannot allocate device memory (a plug-in that only gets
+    input and output pointers, a server whose memory is already committed to other pools, a
+    decode loop that cannot afford the synchronisation an allocation implies).  The scratch for
+    the quantized activations is a fixed array inside the library, TORQ_STATIC_WORKSPACE_BYTES
+    long, shared by every call on the device; Y must be passed in, and this wrapper creates no
+    tensor either.  Raises TorqError(TORQ_ERR_WORKSPACE) when the problem needs more scratch than
+    the array holds.  Calls that may overlap on the GPU race on the array: keep them in one
+    stream.  Make the first call on a device during start-up (it looks up the array's address)."""
+    M, d = X.shape
+    N = Wq.shape[0]
+    for t, n in ((X, "X"), (R_inter, "R_inter"), (R_intra, "R_intra")):
+        _check(t, torch.bfloat16, n)
+    for t, n in ((Wq, "Wq"), (Ws, "Ws")):
+        _check(t, torch.uint8, n)
+    _check(Y, Y.dtype, "Y")
+    dt = TORQ_F32 if Y.dtype == torch.float32 else TORQ_BF16
+    _raise(lib().torq_rotated_linear_static(_ptr(X), _ptr(R_inter), _ptr(R_intra), _ptr(Wq), _ptr(Ws), M, d, N,
+                                            _ptr(Y), dt, _stream(stream)), "torq_rotated_linear_static")
     return Y
 
 
