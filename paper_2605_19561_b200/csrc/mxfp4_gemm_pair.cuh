@@ -1,12 +1,16 @@
 // Block-scaled MXFP4 GEMM on CTA pairs (M > 128): two CTAs share one 256 x 256 output tile through
 // tcgen05.mma cta_group::2 kind::mxf4.block_scale.  Each CTA stages its own 128 rows of A, its own
 // 128 rows of W, its own A scales and the full tile's W scales (35 KiB per 256 elements of K
-// instead of 51 KiB), six stages deep.  No multicast load.
+// instead of 51 KiB), five stages deep.  No multicast load.
 //
 // The 128 x 256 fp32 accumulator of each CTA fills half of tensor memory and the scale factors
 // need columns too, so there is a single accumulator buffer; to keep the tensor pipe busy the
 // eight epilogue warps first drain the whole accumulator into registers (128 values per thread),
-// hand it back to the MMA warp at once, and only then convert and store.
+// hand it back to the MMA warp at once, and only then convert and store: each warp writes its
+// rows into a 4 KiB swizzled staging buffer in shared memory and one lane issues a TMA store of
+// the [32 rows x 128 bytes] box, so that Y is written in whole 128-byte lines (one thread writing
+// 16 bytes of its own row per instruction made 32 partial-sector writes per warp store and ran at
+// a third of the speed).
 //
 // Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (leader CTA only), warps 2..9 epilogue
 // (warp w reads lane quarter w%4, column half (w-2)/4).  Barriers as in the pair rotation kernel;
@@ -26,8 +30,10 @@ struct GemmPairCfg {
   static constexpr int SFA_BYTES = 1024;
   static constexpr int SFB_BYTES = 2048;               // both 128-row tiles of the W scales
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;   // 35 KiB
-  static constexpr int STAGES = 6;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + 1024;
+  static constexpr int STAGES = 5;
+  static constexpr int OUT_WARP_BYTES = 32 * 128;      // per epilogue warp: 32 rows x 128 B, swizzled
+  static constexpr int OUT_BYTES = 8 * OUT_WARP_BYTES;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_BYTES + 256 + 1024;
   static constexpr int SFA_COL = 256;
   static constexpr int SFB_COL = 264;
   static constexpr int TMEM_COLS = 512;
@@ -38,13 +44,15 @@ struct GemmPairCfg {
 __global__ void __launch_bounds__(320, 1)
 mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                        const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB,
-                       void* __restrict__ Y, int y_is_bf16, int M, int N, int K, int* err_word) {
+                       const __grid_constant__ CUtensorMap tmY, int y_is_bf16, int M, int N, int K,
+                       int* err_word) {
   using C = GemmPairCfg;
   constexpr int BN = C::BN;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bar_off = C::STAGES * C::STAGE_BYTES;
+  const uint32_t out_off = C::STAGES * C::STAGE_BYTES;
+  const uint32_t bar_off = out_off + C::OUT_BYTES;
   const uint32_t bar_base = smem_base + bar_off;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };
@@ -178,43 +186,63 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar, 0));   // accumulator is free again
-      const int64_t row = (int64_t)mt * C::BM + q * 32 + lane;
-      const int64_t col0 = (int64_t)nt * BN + h * 128;
-      if (row < M) {
-        auto store32 = [&](const uint32_t (&v)[32], int64_t col) {
-          if (col >= N) return;
-          if (y_is_bf16) {
-            __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(Y) + row * N + col;
+      // Registers -> this warp's staging buffer (one 128-byte row per lane, 16-byte pieces XORed
+      // with row % 8 as the 128-byte TMA swizzle expects) -> TMA store of a [32 rows x 128 B] box.
+      // The store clips rows >= M and columns >= N by itself.
+      const int row0 = mt * C::BM + q * 32;
+      const int col0 = nt * BN + h * 128;
+      const uint32_t stage_buf = smem_base + out_off + (uint32_t)(warp - 2) * C::OUT_WARP_BYTES;
+      const uint32_t my_row = stage_buf + lane * 128;
+      const uint32_t sw = (uint32_t)(lane & 7);
+      auto put16 = [&](int piece, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                     ::"r"(my_row + (((uint32_t)piece ^ sw) << 4)), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+      };
+      auto pack2 = [](uint32_t lo, uint32_t hi) {
+        __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(lo), __uint_as_float(hi));
+        return *reinterpret_cast<uint32_t*>(&hh);
+      };
+      auto flush = [&](int col) {                        // whole warp
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && row0 < M && col < N) {
+          tma_store_2d(&tmY, col, row0, stage_buf);
+          bulk_commit_group();
+        }
+      };
+      auto reuse = [&]() {                               // the previous store has read the buffer
+        if (lane == 0) bulk_wait_group_read<0>();
+        __syncwarp();
+      };
+      if (y_is_bf16) {
+        auto half64 = [&](const uint32_t (&lo)[32], const uint32_t (&hi)[32], int col) {
+          reuse();
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              if (col + 8 * g + 8 <= N) {
-                uint4 o;
-                uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+          for (int p = 0; p < 4; ++p)
+            put16(p, pack2(lo[8 * p], lo[8 * p + 1]), pack2(lo[8 * p + 2], lo[8 * p + 3]),
+                  pack2(lo[8 * p + 4], lo[8 * p + 5]), pack2(lo[8 * p + 6], lo[8 * p + 7]));
 #pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                  __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[8 * g + 2 * p]),
-                                                            __uint_as_float(v[8 * g + 2 * p + 1]));
-                  ow[p] = *reinterpret_cast<uint32_t*>(&hh);
-                }
-                *reinterpret_cast<uint4*>(yp + 8 * g) = o;
-              }
-            }
-          } else {
-            float* yp = reinterpret_cast<float*>(Y) + row * N + col;
-#pragma unroll
-            for (int g = 0; g < 8; ++g) {
-              if (col + 4 * g + 4 <= N)
-                *reinterpret_cast<uint4*>(yp + 4 * g) =
-                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-            }
-          }
+          for (int p = 0; p < 4; ++p)
+            put16(4 + p, pack2(hi[8 * p], hi[8 * p + 1]), pack2(hi[8 * p + 2], hi[8 * p + 3]),
+                  pack2(hi[8 * p + 4], hi[8 * p + 5]), pack2(hi[8 * p + 6], hi[8 * p + 7]));
+          flush(col);
         };
-        store32(v0, col0);
-        store32(v1, col0 + 32);
-        store32(v2, col0 + 64);
-        store32(v3, col0 + 96);
+        half64(v0, v1, col0);
+        half64(v2, v3, col0 + 64);
+      } else {
+        auto quarter32 = [&](const uint32_t (&v)[32], int col) {
+          reuse();
+#pragma unroll
+          for (int p = 0; p < 8; ++p) put16(p, v[4 * p], v[4 * p + 1], v[4 * p + 2], v[4 * p + 3]);
+          flush(col);
+        };
+        quarter32(v0, col0);
+        quarter32(v1, col0 + 32);
+        quarter32(v2, col0 + 64);
+        quarter32(v3, col0 + 96);
       }
     }
+    if (lane == 0) bulk_wait_group<0>();                 // every store of this warp has landed
   }
 
   // ------------------------------------------------------------------ teardown

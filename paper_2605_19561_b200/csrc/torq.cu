@@ -292,11 +292,16 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
         !encode_2d(&tmSFB, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, Ws, (uint64_t)((N + 127) / 128), kb4 * 128, 1, 256,
                    CU_TENSOR_MAP_SWIZZLE_NONE))
       return TORQ_ERR_LAUNCH;
+    CUtensorMap tmY;
+    const bool ybf = y_dtype == TORQ_BF16;
+    if (!encode_2d(&tmY, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, ybf ? 2 : 4,
+                   Y, (uint64_t)M, (uint64_t)N, 32, ybf ? 64 : 32))
+      return TORQ_ERR_LAUNCH;
     const int ptiles = (int)((M + 255) / 256) * (int)((N + BN - 1) / BN);
     const int max_pairs = st->gemm_pairs;
     const int pairs = ptiles < max_pairs ? ptiles : max_pairs;
     launch_pair(mxfp4_gemm_pair_kernel, 2 * pairs, GemmPairCfg::THREADS, GemmPairCfg::SMEM_BYTES, s, tmA, tmB,
-                tmSFA, tmSFB, Y, y_dtype == TORQ_BF16 ? 1 : 0, (int)M, (int)N, (int)K, st->err_word);
+                tmSFA, tmSFB, tmY, ybf ? 1 : 0, (int)M, (int)N, (int)K, st->err_word);
     return launch_status();
   }
   if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, (uint64_t)(K / 2), 128, 128) ||
