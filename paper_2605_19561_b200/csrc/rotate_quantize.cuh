@@ -75,6 +75,9 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // Set-up above touched no global memory; from here on the previous kernel's results are needed.
+  griddep_launch_dependents();
+  griddep_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer

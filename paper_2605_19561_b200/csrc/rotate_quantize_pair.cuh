@@ -77,6 +77,9 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
   cluster_sync_all();                                  // both CTAs' barriers exist before any remote arrive
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // Set-up above touched no global memory; from here on the previous kernel's results are needed.
+  griddep_launch_dependents();
+  griddep_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)

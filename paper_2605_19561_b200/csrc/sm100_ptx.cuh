@@ -73,6 +73,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may start while the
+// kernel before it in the stream is still running; griddep_wait() blocks until that kernel has
+// completed and its writes are visible, so everything that touches global memory comes after it.
+// griddep_launch_dependents() tells the runtime that the NEXT kernel in the stream may begin its
+// own launch processing now (it still waits in its griddep_wait for this kernel to finish).
+__device__ __forceinline__ void griddep_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void griddep_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---- single-lane election -----------------------------------------------------------------------
 // The producer and MMA warps walk their loops with all 32 lanes, so that every address, descriptor
 // and loop counter is warp-uniform, and only the TMA / tcgen05 instructions themselves are issued

@@ -129,22 +129,27 @@ static inline torq_status launch_status() {
   return cudaGetLastError() == cudaSuccess ? TORQ_OK : TORQ_ERR_LAUNCH;
 }
 
-// Launch with a cluster of two CTAs along x (grid must be even).
+// Launch of a persistent tensor-core kernel: `cluster` CTAs per cluster along x (1 or 2; the grid
+// is a multiple of it) and programmatic stream serialization, so that the launch processing of
+// this kernel overlaps the tail of the kernel before it (the kernel itself waits for that kernel
+// to complete before it touches global memory).
 template <typename... KArgs, typename... Args>
-static void launch_pair(void (*kernel)(KArgs...), int grid, int threads, int smem, cudaStream_t s,
-                        Args... args) {
+static void launch_tc(void (*kernel)(KArgs...), int cluster, int grid, int threads, int smem, cudaStream_t s,
+                      Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid, 1, 1);
   cfg.blockDim = dim3((unsigned)threads, 1, 1);
   cfg.dynamicSmemBytes = (size_t)smem;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = (unsigned)cluster;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = cluster > 1 ? 2 : 1;
   cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
@@ -255,15 +260,15 @@ torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void*
     const int ptiles = (int)((M + 255) / 256) * (int)((d + 255) / 256);
     const int max_pairs = st->rot_pairs;
     const int pairs = ptiles < max_pairs ? ptiles : max_pairs;
-    launch_pair(rotate_quantize_pair_kernel, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES, s, tmX,
+    launch_tc(rotate_quantize_pair_kernel, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES, s, tmX,
                 tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, st->err_word);
     return launch_status();
   }
   const int m_tiles = (int)((M + 127) / 128);
   const int tiles = m_tiles * (int)((d + 255) / 256);
   const int grid = tiles < st->sm_count ? tiles : st->sm_count;
-  rotate_quantize_kernel<256><<<grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s>>>(
-      tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, st->err_word);
+  launch_tc(rotate_quantize_kernel<256>, 1, grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s, tmX, tmR,
+            static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, st->err_word);
   return launch_status();
 }
 
@@ -300,7 +305,7 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
     const int ptiles = (int)((M + 255) / 256) * (int)((N + BN - 1) / BN);
     const int max_pairs = st->gemm_pairs;
     const int pairs = ptiles < max_pairs ? ptiles : max_pairs;
-    launch_pair(mxfp4_gemm_pair_kernel, 2 * pairs, GemmPairCfg::THREADS, GemmPairCfg::SMEM_BYTES, s, tmA, tmB,
+    launch_tc(mxfp4_gemm_pair_kernel, 2, 2 * pairs, GemmPairCfg::THREADS, GemmPairCfg::SMEM_BYTES, s, tmA, tmB,
                 tmSFA, tmSFB, tmY, ybf ? 1 : 0, (int)M, (int)N, (int)K, st->err_word);
     return launch_status();
   }
@@ -309,9 +314,9 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
     return TORQ_ERR_LAUNCH;
   const int tiles = (int)((M + 127) / 128) * (int)((N + BN - 1) / BN);
   const int grid = tiles < st->sm_count ? tiles : st->sm_count;
-  mxfp4_gemm_kernel<BN, 1><<<grid, GemmCfg<BN, 1>::THREADS, GemmCfg<BN, 1>::SMEM_BYTES, s>>>(
-      tmA, tmB, static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y,
-      y_dtype == TORQ_BF16 ? 1 : 0, (int)M, (int)N, (int)K, st->err_word);
+  launch_tc(mxfp4_gemm_kernel<BN, 1>, 1, grid, GemmCfg<BN, 1>::THREADS, GemmCfg<BN, 1>::SMEM_BYTES, s, tmA, tmB,
+            static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y, y_dtype == TORQ_BF16 ? 1 : 0,
+            (int)M, (int)N, (int)K, st->err_word);
   return launch_status();
 }
 
