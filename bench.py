@@ -169,7 +169,8 @@ def main():
 
     # ---- inputs (seeded, synthetic; every rank holds its own M rows: weak scaling over tokens)
     xb = I.activations(cfg, M=M)
-    rb, rib, _, _ = I.rotations(cfg, device="cuda")
+    # QR of the seeded Gaussian: LAPACK on the host up to d = 4096, on the device above (few host cores)
+    rb, rib, _, _ = I.rotations(cfg, device="cpu" if d <= 4096 else "cuda")
     w = I.weights(cfg)
     X0 = I.bf16_bits_to_tensor(xb, "cuda")
     R0, Ri0 = I.bf16_bits_to_tensor(rb, "cuda"), I.bf16_bits_to_tensor(rib, "cuda")
