@@ -75,7 +75,10 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
 /* Algorithm 3 steps 1-5 in one call: rotate, quantize, multiply.  The quantized activations live
  * in `workspace` (>= torq_workspace_bytes(M, d, N) bytes, 256-byte aligned), laid out as codes
  * [M, d/2] followed (256-byte aligned) by the tiled scales; pass dbg_codes / dbg_scales non-NULL
- * to also receive copies of them.  Requires d % 128 == 0 and N % 8 == 0. */
+ * to also receive copies of them.  For M <= 128 the workspace also holds fp32 partial tiles: the
+ * rotation is then split along its contraction so that every SM streams a share of R_inter, and
+ * a second kernel adds the partials in a fixed order before the intra-block step and Eq. 1.
+ * Requires d % 128 == 0 and N % 8 == 0. */
 torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* R_intra,
                                 const void* Wq, const void* Ws, int64_t M, int64_t d, int64_t N,
                                 void* Y, torq_dtype y_dtype, void* workspace,
@@ -97,9 +100,11 @@ torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* 
  * does anything it calls.
  *
  * Same arguments, layouts and results as torq_rotated_linear without its workspace and debug
- * parameters.  A problem whose scratch need, torq_workspace_bytes(M, d, N), exceeds
- * TORQ_STATIC_WORKSPACE_BYTES is refused with TORQ_ERR_WORKSPACE before anything is launched
- * (for example M = 2048, d = 14336 fits; M = 8192, d = 5120 does not).
+ * parameters.  A problem whose quantized activations (M * d / 2 code bytes rounded up to 256,
+ * plus torq_scales_bytes(M, d)) exceed TORQ_STATIC_WORKSPACE_BYTES is refused with
+ * TORQ_ERR_WORKSPACE before anything is launched (for example M = 2048, d = 14336 fits;
+ * M = 8192, d = 5120 does not).  What is left of the array serves as the split-K scratch of the
+ * few-token path when it is large enough.
  *
  * First call on each device: the library looks up the array's device address (and, if no other
  * entry point ran before, performs the one-time per-device set-up every entry point shares).

@@ -1,0 +1,248 @@
+// Rotate + quantize for few tokens (M <= 128), where the work is streaming R_inter from HBM once:
+// with one 128 x 256 tile per CTA only d/256 CTAs would pull on the memory system (20 of 148 SMs at
+// d = 5120).  Here the contraction is also split along K: CTA (n tile, k split) multiplies
+// X[:, k range] by R_inter[k range, 256 columns] on the tensor cores and writes its fp32 partial
+// tile to scratch; a second, small kernel adds the partials of each (token, 32-block) in split
+// order, applies the intra-block rotation, and quantizes (Algorithm 3 steps 2-4; the quantizer
+// needs the complete sum, so it cannot run per split).  Summation order is fixed: the result does
+// not depend on timing.
+//
+// Scratch layout: P[split][128 rows][d] fp32 (rows >= M of a 32-row group that holds a token are
+// written as zeros; 32-row groups without any token are not written and not read).
+#pragma once
+#include <cuda_bf16.h>
+#include "quantize.cuh"
+#include "sm100_ptx.cuh"
+
+namespace torq {
+
+struct RotSplitCfg {
+  static constexpr int BM = 128, BN = 256, BK = 64;
+  static constexpr int A_BYTES = BM * BK * 2;          // 16 KiB
+  static constexpr int B_BOX_BYTES = 64 * BK * 2;      // 8 KiB
+  static constexpr int B_BYTES = (BN / 64) * B_BOX_BYTES;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 48 KiB
+  static constexpr int STAGES = 4;
+  static constexpr int OUT_WARP_BYTES = 32 * 128;      // staging for one [32 rows x 32 fp32] box
+  static constexpr int OUT_BYTES = 4 * OUT_WARP_BYTES;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_BYTES + 256 + 1024;
+  static constexpr int TMEM_COLS = 256;
+  static constexpr int THREADS = 192;
+  static constexpr int MAX_SPLITS = 8;
+  static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+};
+
+// grid = n_tiles * splits; CTA b works n tile b % n_tiles, k split b / n_tiles.
+// tmP: fp32 [splits * 128, d], box [32 rows x 32 columns], 128-byte swizzle.
+__global__ void __launch_bounds__(192, 1)
+rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
+                     const __grid_constant__ CUtensorMap tmP, int M, int d, int splits, int* err_word) {
+  using C = RotSplitCfg;
+  constexpr int BN = C::BN;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t out_off = C::STAGES * C::STAGE_BYTES;
+  const uint32_t bar_off = out_off + C::OUT_BYTES;
+  const uint32_t bar_base = smem_base + bar_off;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };
+  const uint32_t accf_bar = bar_base + 8u * (2 * C::STAGES);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + bar_off + 192);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(smem_gen + bar_off + 200);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_tiles = (d + BN - 1) / BN;
+  const int nt = blockIdx.x % n_tiles, ks = blockIdx.x / n_tiles;
+  const int k_tiles = (d + C::BK - 1) / C::BK;
+  const int kt0 = (int)((long long)k_tiles * ks / splits);
+  const int kt1 = (int)((long long)k_tiles * (ks + 1) / splits);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(accf_bar, 1);
+    *cta_abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS); tmem_relinquish(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  griddep_launch_dependents();
+  griddep_wait();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (elect_one()) { tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmR); }
+    bool ok = true;
+    for (int kt = kt0, it = 0; kt < kt1 && ok; ++kt, ++it) {
+      const int s = it % C::STAGES;
+      if (!mbar_wait_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
+                          SITE_PRODUCER_EMPTY)) { ok = false; break; }
+      const uint32_t st = smem_base + s * C::STAGE_BYTES;
+      if (elect_one()) {
+        mbar_arrive_expect_tx(full_bar(s), C::STAGE_BYTES);
+        tma_load_2d(st, &tmX, kt * C::BK, 0, full_bar(s));
+#pragma unroll
+        for (int b = 0; b < BN / 64; ++b)
+          tma_load_2d(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR, nt * BN + b * 64, kt * C::BK, full_bar(s));
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    constexpr uint32_t idesc = idesc_bf16(128, BN, /*A MN-major*/ false, /*B MN-major*/ true);
+    bool ok = true;
+    for (int kt = kt0, it = 0; kt < kt1 && ok; ++kt, ++it) {
+      const int s = it % C::STAGES;
+      if (!mbar_wait_warp(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
+        ok = false; break;
+      }
+      tc_fence_after_sync();
+      const uint32_t st = smem_base + s * C::STAGE_BYTES;
+      const uint64_t adesc = make_desc(st, 16, 1024, kSwizzle128);
+      const uint64_t bdesc = make_desc(st + C::A_BYTES, C::B_BOX_BYTES, 1024, kSwizzle128);
+      if (elect_one()) {
+#pragma unroll
+        for (int j = 0; j < C::BK / 16; ++j)
+          mma_bf16(tmem_base, adesc + 2 * j, bdesc + 128 * j, idesc, (it | j) != 0);
+        tc_commit(empty_bar(s));
+      }
+      __syncwarp();
+    }
+    if (ok && elect_one()) tc_commit(accf_bar);
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ epilogue: partial tile -> scratch
+    const int q = warp & 3;
+    bool ok = mbar_wait(accf_bar, 0, cta_abort, err_word, SITE_EPI_ACC_FULL);
+    ok = __all_sync(0xFFFFFFFFu, ok);
+    if (ok && q * 32 < M) {                              // this 32-row group holds at least one token
+      tc_fence_after_sync();
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
+      const uint32_t stage_buf = smem_base + out_off + (uint32_t)(warp - 2) * C::OUT_WARP_BYTES;
+      const uint32_t my_row = stage_buf + lane * 128;
+      const uint32_t sw = (uint32_t)(lane & 7);
+#pragma unroll 1
+      for (int bb = 0; bb < BN / 32; ++bb) {
+        uint32_t v[32];
+        tmem_ld_32x32(tacc + bb * 32, v);
+        tmem_ld_wait();
+        if (bb > 0) {                                    // the previous store has read the buffer
+          if (lane == 0) bulk_wait_group_read<0>();
+          __syncwarp();
+        }
+#pragma unroll
+        for (int p = 0; p < 8; ++p)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(my_row + (((uint32_t)p ^ sw) << 4)), "r"(v[4 * p]), "r"(v[4 * p + 1]),
+                         "r"(v[4 * p + 2]), "r"(v[4 * p + 3]) : "memory");
+        fence_proxy_async_smem();
+        __syncwarp();
+        const int col = nt * BN + bb * 32;
+        if (lane == 0 && col < d) {
+          tma_store_2d(&tmP, col, ks * C::BM + q * 32, stage_buf);
+          bulk_commit_group();
+        }
+      }
+      if (lane == 0) bulk_wait_group<0>();
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before_sync();
+  __syncthreads();
+  if (*cta_abort) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+}
+
+// Second phase: one CTA of four warps per 32-block b, warp w = rows 32w .. 32w+31, lane = row.
+// The CTA first stages R_intra[b] in shared memory as fp32 (one coalesced 2 KiB read); then each
+// thread adds its row's partial blocks in split order, applies the intra-block rotation in fp32
+// FMAs in index order (R read from shared memory at the same address by every lane) and quantizes
+// (Eq. 1).  Rows M .. 127 and K-blocks d/32 .. (padded to 4) only get their padding scale byte (0).
+__global__ void __launch_bounds__(128)
+splitk_reduce_quantize_kernel(const float* __restrict__ P, const __nv_bfloat16* __restrict__ R_intra,
+                              int M, int d, int splits, uint8_t* __restrict__ codes,
+                              uint8_t* __restrict__ scales) {
+  __shared__ __align__(16) float r_s[1024];
+  griddep_launch_dependents();
+  griddep_wait();
+  const int nb = d / 32;
+  const int kb4 = (nb + 3) / 4;
+  const int b = blockIdx.x, row = threadIdx.x;
+  if (b >= nb) {                                         // padding K-block
+    scales[scale_offset(row, b, kb4)] = 0;
+    return;
+  }
+  if (R_intra != nullptr) {
+    float v[8];
+    load8(R_intra + (size_t)b * 1024 + threadIdx.x * 8, v);
+    *reinterpret_cast<float4*>(r_s + threadIdx.x * 8) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(r_s + threadIdx.x * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+  }
+  __syncthreads();
+  if (row >= M) {
+    scales[scale_offset(row, b, kb4)] = 0;
+    return;
+  }
+  float y[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) y[j] = 0.f;
+  const float4* p0 = reinterpret_cast<const float4*>(P + ((size_t)row * d + b * 32));
+  const size_t split_stride = (size_t)128 * d / 4;       // in float4
+  int s = 0;
+  for (; s + 2 <= splits; s += 2) {                      // two splits' loads in flight, added in order
+    float4 u[8], w[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) { u[g] = __ldg(p0 + s * split_stride + g); w[g] = __ldg(p0 + (s + 1) * split_stride + g); }
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      y[4 * g] += u[g].x; y[4 * g + 1] += u[g].y; y[4 * g + 2] += u[g].z; y[4 * g + 3] += u[g].w;
+    }
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      y[4 * g] += w[g].x; y[4 * g + 1] += w[g].y; y[4 * g + 2] += w[g].z; y[4 * g + 3] += w[g].w;
+    }
+  }
+  if (s < splits) {
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      const float4 u = __ldg(p0 + s * split_stride + g);
+      y[4 * g] += u.x; y[4 * g + 1] += u.y; y[4 * g + 2] += u.z; y[4 * g + 3] += u.w;
+    }
+  }
+  float z[32];
+  if (R_intra != nullptr) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) z[j] = 0.f;
+    const float4* r = reinterpret_cast<const float4*>(r_s);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {
+        const float4 rv = r[i * 8 + g];
+        z[4 * g + 0] = fmaf(y[i], rv.x, z[4 * g + 0]);
+        z[4 * g + 1] = fmaf(y[i], rv.y, z[4 * g + 1]);
+        z[4 * g + 2] = fmaf(y[i], rv.z, z[4 * g + 2]);
+        z[4 * g + 3] = fmaf(y[i], rv.w, z[4 * g + 3]);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) z[j] = y[j];
+  }
+  uint4 c;
+  uint32_t sbyte;
+  quantize_block32(z, c, sbyte);
+  *reinterpret_cast<uint4*>(codes + (size_t)row * (d / 2) + b * 16) = c;
+  scales[scale_offset(row, b, kb4)] = (uint8_t)sbyte;
+}
+
+}  // namespace torq

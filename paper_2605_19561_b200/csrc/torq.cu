@@ -11,6 +11,7 @@
 #include "quantize.cuh"
 #include "rotate_quantize.cuh"
 #include "rotate_quantize_pair.cuh"
+#include "rotate_splitk.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -92,6 +93,7 @@ static DeviceState* device_state() {
               opt_in_smem(rotate_quantize_kernel<256>, RotCfg<256>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_kernel<128>, RotCfg<128>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_pair_kernel, RotPairCfg::SMEM_BYTES) &&
+              opt_in_smem(rotate_splitk_kernel, RotSplitCfg::SMEM_BYTES) &&
               opt_in_smem(mxfp4_gemm_pair_kernel, GemmPairCfg::SMEM_BYTES);
     if (!ok) return nullptr;
     st.rot_pairs = max_active_pairs(rotate_quantize_pair_kernel, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
@@ -153,6 +155,23 @@ static void launch_tc(void (*kernel)(KArgs...), int cluster, int grid, int threa
   cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// K splits of the few-token rotation: as many as fill the SMs, each at least two 64-element steps.
+// `sm_count` <= 0 gives the bound used for sizing workspaces (any device up to 160 SMs).
+static int rotation_splits(int64_t M, int64_t d, int sm_count) {
+  if (M > 128) return 1;
+  const int n_tiles = (int)((d + 255) / 256), k_tiles = (int)((d + 63) / 64);
+  int s = (sm_count > 0 ? sm_count : 160) / n_tiles;
+  if (s > RotSplitCfg::MAX_SPLITS) s = RotSplitCfg::MAX_SPLITS;
+  if (s > k_tiles / 2) s = k_tiles / 2;
+  return s < 2 ? 1 : s;
+}
+static size_t quantized_bytes(int64_t M, int64_t d) {    // codes, then 256-byte aligned the scales
+  return ((size_t)M * (size_t)(d / 2) + 255) / 256 * 256 + torq_scales_bytes(M, d);
+}
+static size_t splitk_scratch_bytes(int64_t d, int splits) {
+  return splits < 2 ? 0 : (size_t)splits * 128 * (size_t)d * sizeof(float);
+}
+
 static torq_status quantize_impl(DeviceState* st, const void* Z, torq_dtype dt, int64_t M, int64_t d,
                                  void* codes, void* scales, cudaStream_t s) {
   const int64_t kb4 = (d / 32 + 3) / 4;
@@ -186,8 +205,7 @@ size_t torq_scale_offset(int64_t row, int64_t kblock, int64_t k) {
 size_t torq_workspace_bytes(int64_t M, int64_t d, int64_t N) {
   (void)N;
   if (M <= 0 || d <= 0) return 0;
-  size_t codes = ((size_t)M * (size_t)(d / 2) + 255) / 256 * 256;
-  return codes + torq_scales_bytes(M, d);
+  return quantized_bytes(M, d) + splitk_scratch_bytes(d, rotation_splits(M, d, 0));
 }
 
 const char* torq_status_string(torq_status s) {
@@ -230,8 +248,11 @@ torq_status torq_quantize_mxfp4(const void* Z, torq_dtype z_dtype, int64_t M, in
   return quantize_impl(st, Z, z_dtype, M, d, out_codes, out_scales, static_cast<cudaStream_t>(stream));
 }
 
-torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void* R_intra, int64_t M,
-                                 int64_t d, void* out_codes, void* out_scales, void* stream) {
+// Steps 1-4.  `scratch` (may be NULL) is fp32 room for the split-K partials of the few-token path;
+// without enough of it the single-pass kernels run.
+static torq_status rotate_quantize_impl(const void* X, const void* R_inter, const void* R_intra, int64_t M,
+                                        int64_t d, void* out_codes, void* out_scales, void* scratch,
+                                        size_t scratch_bytes, void* stream) {
   if (!X || !out_codes || !out_scales) return TORQ_ERR_NULL;
   if (M < 1 || d < 32 || d % 32 != 0 || M > (1 << 30) || d > (1 << 24)) return TORQ_ERR_SHAPE;
   if (!aligned16(X) || !aligned16(out_codes) || !aligned16(out_scales) ||
@@ -255,6 +276,21 @@ torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void*
   if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d, 128, 64) ||
       !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
     return TORQ_ERR_LAUNCH;
+  const int splits = rotation_splits(M, d, st->sm_count);
+  if (splits >= 2 && scratch && scratch_bytes >= splitk_scratch_bytes(d, splits) &&
+      (reinterpret_cast<uintptr_t>(scratch) & 15u) == 0) {
+    // Few tokens: split K over the SMs, partial tiles to scratch, then reduce + intra + quantize.
+    CUtensorMap tmP;
+    if (!encode_2d(&tmP, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, scratch, (uint64_t)splits * 128, (uint64_t)d, 32, 32))
+      return TORQ_ERR_LAUNCH;
+    const int n_tiles = (int)((d + 255) / 256);
+    launch_tc(rotate_splitk_kernel, 1, n_tiles * splits, RotSplitCfg::THREADS, RotSplitCfg::SMEM_BYTES, s, tmX, tmR,
+              tmP, (int)M, (int)d, splits, st->err_word);
+    if (launch_status() != TORQ_OK) return TORQ_ERR_LAUNCH;
+    launch_tc(splitk_reduce_quantize_kernel, 1, (int)(((d / 32 + 3) / 4) * 4), 128, 0, s, static_cast<const float*>(scratch),
+              static_cast<const __nv_bfloat16*>(R_intra), (int)M, (int)d, splits, codes, scales);
+    return launch_status();
+  }
   if (M > 128) {
     // CTA pairs: 256 x 256 tiles, one pair per two SMs.
     const int ptiles = (int)((M + 255) / 256) * (int)((d + 255) / 256);
@@ -270,6 +306,11 @@ torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void*
   launch_tc(rotate_quantize_kernel<256>, 1, grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s, tmX, tmR,
             static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, st->err_word);
   return launch_status();
+}
+
+torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void* R_intra, int64_t M,
+                                 int64_t d, void* out_codes, void* out_scales, void* stream) {
+  return rotate_quantize_impl(X, R_inter, R_intra, M, d, out_codes, out_scales, nullptr, 0, stream);
 }
 
 torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, const void* Ws, int64_t M,
@@ -309,29 +350,38 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
                 tmSFA, tmSFB, tmY, ybf ? 1 : 0, (int)M, (int)N, (int)K, st->err_word);
     return launch_status();
   }
+  // One row tile: the work is streaming W once, so prefer the narrower tile while it still leaves
+  // SMs idle (128-column tiles double the number of CTAs pulling on memory).
+  const bool narrow = 2 * (int)((N + BN - 1) / BN) <= st->sm_count;
+  const uint32_t bn = narrow ? 128 : BN;
   if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, (uint64_t)(K / 2), 128, 128) ||
-      !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)(K / 2), BN, 128))
+      !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)(K / 2), bn, 128))
     return TORQ_ERR_LAUNCH;
-  const int tiles = (int)((M + 127) / 128) * (int)((N + BN - 1) / BN);
+  const int tiles = (int)((M + 127) / 128) * (int)((N + bn - 1) / bn);
   const int grid = tiles < st->sm_count ? tiles : st->sm_count;
-  launch_tc(mxfp4_gemm_kernel<BN, 1>, 1, grid, GemmCfg<BN, 1>::THREADS, GemmCfg<BN, 1>::SMEM_BYTES, s, tmA, tmB,
-            static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y, y_dtype == TORQ_BF16 ? 1 : 0,
-            (int)M, (int)N, (int)K, st->err_word);
+  if (narrow)
+    launch_tc(mxfp4_gemm_kernel<128, 2>, 1, grid, GemmCfg<128, 2>::THREADS, GemmCfg<128, 2>::SMEM_BYTES, s, tmA,
+              tmB, static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y,
+              y_dtype == TORQ_BF16 ? 1 : 0, (int)M, (int)N, (int)K, st->err_word);
+  else
+    launch_tc(mxfp4_gemm_kernel<BN, 1>, 1, grid, GemmCfg<BN, 1>::THREADS, GemmCfg<BN, 1>::SMEM_BYTES, s, tmA, tmB,
+              static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y, y_dtype == TORQ_BF16 ? 1 : 0,
+              (int)M, (int)N, (int)K, st->err_word);
   return launch_status();
 }
 
-torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* R_intra, const void* Wq,
-                                const void* Ws, int64_t M, int64_t d, int64_t N, void* Y,
-                                torq_dtype y_dtype, void* workspace, size_t workspace_bytes,
-                                void* dbg_codes, void* dbg_scales, void* stream) {
-  if (!X || !Wq || !Ws || !Y) return TORQ_ERR_NULL;
-  if (M < 1 || d < 128 || d % 128 != 0 || N < 8 || N % 8 != 0) return TORQ_ERR_SHAPE;
-  if (!workspace || workspace_bytes < torq_workspace_bytes(M, d, N)) return TORQ_ERR_WORKSPACE;
-  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return TORQ_ERR_ALIGN;
+// Steps 1-5 with `workspace_bytes` >= quantized_bytes(M, d) already checked by the caller: codes,
+// scales, then whatever is left as split-K scratch.
+static torq_status rotated_linear_impl(const void* X, const void* R_inter, const void* R_intra, const void* Wq,
+                                       const void* Ws, int64_t M, int64_t d, int64_t N, void* Y,
+                                       torq_dtype y_dtype, void* workspace, size_t workspace_bytes,
+                                       void* dbg_codes, void* dbg_scales, void* stream) {
   uint8_t* codes = static_cast<uint8_t*>(workspace);
   const size_t codes_bytes = (size_t)M * (size_t)(d / 2);
   uint8_t* scales = codes + (codes_bytes + 255) / 256 * 256;
-  torq_status rc = torq_rotate_quantize(X, R_inter, R_intra, M, d, codes, scales, stream);
+  const size_t used = quantized_bytes(M, d);
+  torq_status rc = rotate_quantize_impl(X, R_inter, R_intra, M, d, codes, scales, codes + used,
+                                        workspace_bytes - used, stream);
   if (rc != TORQ_OK) return rc;
   rc = torq_mxfp4_gemm(codes, scales, Wq, Ws, M, N, d, Y, y_dtype, stream);
   if (rc != TORQ_OK) return rc;
@@ -343,6 +393,18 @@ torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* 
                                     cudaMemcpyDeviceToDevice, s) != cudaSuccess)
     return TORQ_ERR_LAUNCH;
   return TORQ_OK;
+}
+
+torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* R_intra, const void* Wq,
+                                const void* Ws, int64_t M, int64_t d, int64_t N, void* Y,
+                                torq_dtype y_dtype, void* workspace, size_t workspace_bytes,
+                                void* dbg_codes, void* dbg_scales, void* stream) {
+  if (!X || !Wq || !Ws || !Y) return TORQ_ERR_NULL;
+  if (M < 1 || d < 128 || d % 128 != 0 || N < 8 || N % 8 != 0) return TORQ_ERR_SHAPE;
+  if (!workspace || workspace_bytes < torq_workspace_bytes(M, d, N)) return TORQ_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return TORQ_ERR_ALIGN;
+  return rotated_linear_impl(X, R_inter, R_intra, Wq, Ws, M, d, N, Y, y_dtype, workspace, workspace_bytes,
+                             dbg_codes, dbg_scales, stream);
 }
 
 // ---- the layer without any allocation -----------------------------------------------------------
@@ -375,10 +437,10 @@ torq_status torq_rotated_linear_static(const void* X, const void* R_inter, const
   if (!X || !Wq || !Ws || !Y) return TORQ_ERR_NULL;
   if (M < 1 || d < 128 || d % 128 != 0 || N < 8 || N % 8 != 0 || M > (1 << 30) || d > (1 << 24))
     return TORQ_ERR_SHAPE;
-  if (torq_workspace_bytes(M, d, N) > (size_t)TORQ_STATIC_WORKSPACE_BYTES) return TORQ_ERR_WORKSPACE;
+  if (quantized_bytes(M, d) > (size_t)TORQ_STATIC_WORKSPACE_BYTES) return TORQ_ERR_WORKSPACE;
   void* scratch = static_workspace_address();
   if (!scratch) return TORQ_ERR_LAUNCH;
-  return torq_rotated_linear(X, R_inter, R_intra, Wq, Ws, M, d, N, Y, y_dtype, scratch,
+  return rotated_linear_impl(X, R_inter, R_intra, Wq, Ws, M, d, N, Y, y_dtype, scratch,
                              (size_t)TORQ_STATIC_WORKSPACE_BYTES, nullptr, nullptr, stream);
 }
 

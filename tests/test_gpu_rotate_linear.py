@@ -133,3 +133,39 @@ def test_llama3_qkv_shape_sampled_rows():
     ref = O.round_to_bf16(O.gemm_dequant(g_codes, g_sb, w_codes, w_sb))
     got = y.float().cpu().numpy()[rows].astype(np.float64)
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-3
+
+
+@pytest.mark.parametrize("M,d", [(1, 256), (33, 256), (100, 512), (128, 1024), (64, 2048), (17, 4096)])
+def test_few_token_split_k_path_through_the_fused_call(M, d):
+    """M <= 128 through torq_rotated_linear: the rotation runs as split-K partial tiles plus the
+    reduce/intra/quantize kernel (the workspace carries the partials).  Same bounds as the
+    single-pass path, and the codes must also agree with the single-pass kernel to the same
+    bounds (only the fp32 summation order differs)."""
+    cfg = I.CONFIGS["tiny"]
+    xb = I.activations(cfg, M=M, d=d)
+    rb, rib, _, _ = I.rotations(cfg, d=d)
+    N = 64
+    wq, wsb = I.random_codes(N, d, seed=21)
+    Wq, Ws = dev_u8(wq), dev_u8(O.swizzle_scales(wsb, d, fill=0))
+    for intra in (rib, None):
+        dbg_c = torch.empty((M, d // 2), dtype=torch.uint8, device="cuda")
+        dbg_s = torch.empty(torq.torq_scales_bytes(M, d), dtype=torch.uint8, device="cuda")
+        before = torq.torq_launch_count()
+        y = torq.torq_rotated_linear(dev_bf16(xb), dev_bf16(rb), None if intra is None else dev_bf16(intra), Wq, Ws,
+                                     out_dtype=torch.float32, dbg_codes=dbg_c, dbg_scales=dbg_s)
+        torch.cuda.synchronize()
+        assert torq.torq_launch_count() - before == 3          # split-K, reduce, GEMM
+        assert torq.torq_last_device_error() == 0
+        g_codes, g_sb = gpu_quantized_to_numpy(dbg_c, dbg_s, M, d)
+        o_codes, o_sb = O.quantize_mxfp4(O.round_to_f32(O.rotate(xb, rb, intra)))
+        rep = mismatch_report(g_codes, g_sb, o_codes, o_sb)
+        assert rep["non_adjacent"] == 0 and rep["scale_off_by_more_than_one"] == 0, rep
+        assert rep["elem_mismatch_frac"] <= max(1e-4, 1.5 / g_codes.size), rep
+        assert rep["block_scale_mismatch_frac"] <= max(1e-4, 1.5 / g_sb.size), rep
+        # padding rows of the scale tiles are zero
+        raw = dbg_s.cpu().numpy()
+        for r in range(M, (M + 127) // 128 * 128):
+            assert raw[torq.torq_scale_offset(r, 0, d)] == 0
+        ref = O.gemm_dequant(g_codes, g_sb, O.unpack_codes(wq), wsb)
+        got = y.cpu().numpy().astype(np.float64)
+        assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-3
