@@ -52,6 +52,89 @@ __device__ __forceinline__ void quantize_block32(const float (&z)[32], uint4& co
                        z[29] * inv, z[30] * inv, z[31] * inv);
 }
 
+// Intra-block rotation of one block held by one thread (Algorithm 3 step 3):
+// z[j] = sum_i y[i] * R[i][j], fp32, i in index order, with R (fp32, row-major 32 x 32) read from
+// shared memory at `r_saddr` -- every lane reads the same address, so each load is one broadcast.
+// The FMAs are issued as packed pairs (fma.rn.f32x2: two independent IEEE fused multiply-adds per
+// instruction, same results as 32 scalar chains).
+__device__ __forceinline__ void intra_rotate32(const uint32_t (&y)[32], uint32_t r_saddr, float (&z)[32]) {
+  uint64_t zp[16];
+#pragma unroll
+  for (int k = 0; k < 16; ++k) zp[k] = 0ull;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    uint64_t yy;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(yy) : "r"(y[i]));
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      uint64_t r0, r1;
+      asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(r0), "=l"(r1) : "r"(r_saddr + (uint32_t)((i * 8 + g) * 16)));
+      asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(zp[2 * g]) : "l"(yy), "l"(r0));
+      asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(zp[2 * g + 1]) : "l"(yy), "l"(r1));
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+    uint32_t lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(zp[k]));
+    z[2 * k] = __uint_as_float(lo);
+    z[2 * k + 1] = __uint_as_float(hi);
+  }
+}
+
+// ---- intra-block rotation on the warp-level tensor-core path -------------------------------------
+// y (fp32) is split into three bfloat16 terms, y = hi + mid + lo up to 2^-24 relative; R_intra is
+// bfloat16 already, so every product is exact in fp32 and the fp32-accumulating warp MMA
+// (m16n8k16) reproduces the fp32 rotation to accumulation-order rounding.
+// Two fp32 values -> packed pairs (element 0 in the low half) of the three terms.
+__device__ __forceinline__ void split3_bf16x2(uint32_t x0, uint32_t x1, uint32_t& hi, uint32_t& mid,
+                                              uint32_t& lo) {
+  float f0 = __uint_as_float(x0), f1 = __uint_as_float(x1);
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hi) : "f"(f1), "f"(f0));
+  f0 -= __uint_as_float(hi << 16);                       // exact: hi is within half a bf16 ulp of f
+  f1 -= __uint_as_float(hi & 0xFFFF0000u);
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(mid) : "f"(f1), "f"(f0));
+  f0 -= __uint_as_float(mid << 16);
+  f1 -= __uint_as_float(mid & 0xFFFF0000u);
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo) : "f"(f1), "f"(f0));
+}
+// D[16x8] += A[16x16] . B[16x8], bf16 inputs, fp32 accumulate (fragment layouts of the PTX ISA).
+__device__ __forceinline__ void mma_16816_bf16(float (&c)[4], const uint32_t* a, const uint32_t* b) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+// Four 8x8 bf16 matrices from shared memory, transposed on the way (B fragments of a row-major
+// [k][n] matrix).  Lane l supplies the address of row l % 8 of matrix l / 8.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t saddr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                                  uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(saddr));
+}
+// One row of a 32-block spread over the four lanes that share it in the accumulator layout: lane
+// p = lane % 4 holds v[2 nt + e] = element 8 nt + 2 p + e.  Returns the scale byte and, in `word`,
+// the four code bytes 4p .. 4p+3 of the block (so the four lanes together store 16 contiguous bytes).
+__device__ __forceinline__ void quantize_row_fragment(const float (&v)[8], int p, uint32_t& word,
+                                                      uint32_t& sbyte) {
+  float amax = 0.f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fabsf(v[j]));
+  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+  float inv;
+  block_scale(amax, sbyte, inv);
+  // byte nt of w = codes of elements 8 nt + 2 p, 8 nt + 2 p + 1 = byte 4 nt + p of the block
+  const uint32_t w = pack8_e2m1(v[0] * inv, v[1] * inv, v[2] * inv, v[3] * inv, v[4] * inv, v[5] * inv,
+                                v[6] * inv, v[7] * inv);
+  // 4 x 4 byte transpose across the four lanes
+  const uint32_t w1 = __shfl_xor_sync(0xFFFFFFFFu, w, 1);
+  const uint32_t x = (p & 1) ? __byte_perm(w, w1, 0x3715) : __byte_perm(w, w1, 0x6240);
+  const uint32_t x2 = __shfl_xor_sync(0xFFFFFFFFu, x, 2);
+  word = (p & 2) ? __byte_perm(x, x2, 0x3276) : __byte_perm(x, x2, 0x5410);
+}
+
 __host__ __device__ __forceinline__ size_t scale_offset(int64_t row, int64_t kblock, int64_t kb4) {
   return (size_t)(((row >> 7) * kb4 + (kblock >> 2)) * 512 + (row & 31) * 16 +
                   ((row & 127) >> 5) * 4 + (kblock & 3));

@@ -7,10 +7,10 @@
 // reads both CTAs' shared memory.
 //
 // Roles per CTA: warp 0 TMA producer (both CTAs), warp 1 MMA issuer (leader CTA only; both
-// allocate tensor memory), warps 2..5 epilogue (each CTA drains its own 128 x 256 accumulator).
+// allocate tensor memory), warps 2..9 epilogue (each CTA drains its own 128 x 256 accumulator).
 // Barriers: full[s] lives in the leader and counts the bytes of both CTAs' loads; empty[s] and
 // acc_full[a] are local to each CTA and are signalled by the leader's tcgen05.commit to both;
-// acc_empty[a] lives in the leader and takes one arrival per epilogue warp of both CTAs.
+// acc_empty[a] lives in the leader and takes one arrival per epilogue warp of both CTAs (16).
 #pragma once
 #include <cuda_bf16.h>
 #include "quantize.cuh"
@@ -27,15 +27,17 @@ struct RotPairCfg {
   static constexpr int B_BYTES = (BN / 2 / 64) * B_BOX_BYTES;   // this CTA's 128 columns = 16 KiB
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;         // 32 KiB
   static constexpr int STAGES = 6;
-  static constexpr int RI_BYTES = (BN / 32) * 32 * 32 * 4;
+  static constexpr int RI_ROW_BYTES = 80;              // 32 bf16 + 16 B pad: conflict-free ldmatrix
+  static constexpr int RI_BLOCK_BYTES = 32 * RI_ROW_BYTES;
+  static constexpr int RI_BYTES = (BN / 32) * 32 * 32 * 4;     // the tile's R_intra blocks: fp32, or bf16 padded
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + RI_BYTES + 256 + 1024;
   static constexpr int NACC = 2;
   static constexpr int TMEM_COLS = 512;
-  static constexpr int THREADS = 192;
+  static constexpr int THREADS = 320;               // producer, MMA issuer, 8 epilogue warps
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
 
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(320, 1)
 rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
                             const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
                             uint8_t* __restrict__ scales, int M, int d, int* err_word) {
@@ -44,7 +46,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  float* ri_smem = reinterpret_cast<float*>(smem_gen + C::STAGES * C::STAGE_BYTES);
+  uint8_t* ri_smem = smem_gen + C::STAGES * C::STAGE_BYTES;
   const uint32_t bar_off = C::STAGES * C::STAGE_BYTES + C::RI_BYTES;
   const uint32_t bar_base = smem_base + bar_off;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
@@ -67,7 +69,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < C::NACC; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 8); }
+    for (int a = 0; a < C::NACC; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 16); }
     *cta_abort = 0;
     fence_mbar_init();
   }
@@ -139,83 +141,165 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (128 threads per CTA)
+    // ------------------------------------------------------------------ epilogue (8 warps per CTA)
+    // warp w reads lane quarter w % 4 (32 rows) and column half (w - 2) / 4 (four 32-blocks = one
+    // 4-byte group of scale bytes).  Two forms of the intra-block rotation:
+    //  * fp32 FMAs, one row per thread, R_intra broadcast from shared memory as fp32.  Bound by
+    //    that broadcast (8 bytes per lane and cycle): about 3/4 of a mainloop per tile, which does
+    //    not matter while the next tile's mainloop runs beside it on the tensor pipe.
+    //  * warp-level tensor-core MMAs on the accumulator fragment layout (y split into three bf16
+    //    terms, R_intra exact in bf16, fp32 accumulation): half the time when the tensor pipe is
+    //    otherwise idle, but it fights the mainloop when both run.  Used for the CTA's LAST tile,
+    //    whose epilogue nothing overlaps.
     const int q = warp & 3;
-    const int et = (warp - 2) * 32 + lane;
+    const int h = (warp - 2) >> 2;
+    const int et = (warp - 2) * 32 + lane;               // 0..255 among the epilogue threads
+    const int p = lane & 3, r8 = lane >> 2;
+    const uint32_t ri_saddr = smem_u32(ri_smem);
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles; tile += npairs, ++tcount) {
       const int mt = 2 * (tile % mp_tiles) + (int)rank, nt = tile / mp_tiles;
       const int a = tcount % C::NACC;
       const int b0 = nt * (BN / 32);
+      const bool last = tile + npairs >= total_tiles;
       if (R_intra != nullptr) {
         // Executed by every epilogue thread for every tile, also after a wait has given up.
-        named_barrier_sync(1, 128);
-        for (int idx = et * 8; ok && idx < (BN / 32) * 1024; idx += 128 * 8) {
-          const int blk = b0 + (idx >> 10);
-          float v[8];
-          if (blk < nblocks) load8(R_intra + (size_t)blk * 1024 + (idx & 1023), v);
-          else {
+        named_barrier_sync(1, 256);
+        for (int idx = et * 8; ok && idx < (BN / 32) * 1024; idx += 256 * 8) {
+          const int lb = idx >> 10, blk = b0 + lb;
+          if (last) {                                    // bf16 rows of 80 bytes: conflict-free ldmatrix
+            const int i = (idx & 1023) >> 5, c = idx & 31;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (blk < nblocks) v = __ldg(reinterpret_cast<const uint4*>(R_intra + (size_t)blk * 1024 + (idx & 1023)));
+            *reinterpret_cast<uint4*>(ri_smem + lb * C::RI_BLOCK_BYTES + i * C::RI_ROW_BYTES + c * 2) = v;
+          } else {                                       // fp32, dense
+            float v[8];
+            if (blk < nblocks) load8(R_intra + (size_t)blk * 1024 + (idx & 1023), v);
+            else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = 0.f;
+              for (int i = 0; i < 8; ++i) v[i] = 0.f;
+            }
+            float* dst = reinterpret_cast<float*>(ri_smem) + idx;
+            *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
           }
-          *reinterpret_cast<float4*>(ri_smem + idx) = make_float4(v[0], v[1], v[2], v[3]);
-          *reinterpret_cast<float4*>(ri_smem + idx + 4) = make_float4(v[4], v[5], v[6], v[7]);
         }
-        named_barrier_sync(1, 128);
+        named_barrier_sync(1, 256);
       }
       if (ok) ok = mbar_wait_cluster(accf_bar(a), (tcount / C::NACC) & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) continue;
       tc_fence_after_sync();
-      const int64_t row = (int64_t)mt * C::BM + q * 32 + lane;
-      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
-      uint32_t sc_word = 0;
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + h * 128;
+      const int chunk = (b0 + h * 4) >> 2;
+      if (!last) {
+        // ---- one row per thread, fp32 FMAs
+        const int64_t row = (int64_t)mt * C::BM + q * 32 + lane;
+        uint32_t sc_word = 0;
 #pragma unroll 1
-      for (int bb = 0; bb < BN / 32; ++bb) {
-        uint32_t yv[32];
-        tmem_ld_32x32(tacc + bb * 32, yv);
-        tmem_ld_wait();
-        if (bb == BN / 32 - 1) {                         // accumulator fully read: tell the leader
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar(a), 0));
-        }
-        float z[32];
-        if (R_intra != nullptr) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) z[j] = 0.f;
-          const float4* r = reinterpret_cast<const float4*>(ri_smem + bb * 1024);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float yi = __uint_as_float(yv[i]);
-#pragma unroll
-            for (int g = 0; g < 8; ++g) {
-              const float4 rv = r[i * 8 + g];
-              z[4 * g + 0] = fmaf(yi, rv.x, z[4 * g + 0]);
-              z[4 * g + 1] = fmaf(yi, rv.y, z[4 * g + 1]);
-              z[4 * g + 2] = fmaf(yi, rv.z, z[4 * g + 2]);
-              z[4 * g + 3] = fmaf(yi, rv.w, z[4 * g + 3]);
-            }
+        for (int bb = 0; bb < 4; ++bb) {
+          uint32_t yv[32];
+          tmem_ld_32x32(tacc + bb * 32, yv);
+          tmem_ld_wait();
+          if (bb == 3) {                                 // this warp's share is read: tell the leader
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar(a), 0));
           }
-        } else {
+          float z[32];
+          if (R_intra != nullptr) {
+            intra_rotate32(yv, ri_saddr + (uint32_t)(h * 4 + bb) * 4096, z);
+          } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) z[j] = __uint_as_float(yv[j]);
+            for (int j = 0; j < 32; ++j) z[j] = __uint_as_float(yv[j]);
+          }
+          uint4 cw;
+          uint32_t sbyte;
+          quantize_block32(z, cw, sbyte);
+          const int blk = b0 + h * 4 + bb;
+          if (row < M && blk < nblocks)
+            *reinterpret_cast<uint4*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+          sc_word |= sbyte << (8 * bb);
         }
-        uint4 cw;
-        uint32_t sbyte;
-        quantize_block32(z, cw, sbyte);
-        const int blk = b0 + bb;
-        if (row < M && blk < nblocks)
-          *reinterpret_cast<uint4*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
-        sc_word |= sbyte << (8 * (bb & 3));
-        if ((bb & 3) == 3) {
-          const int chunk = (b0 + bb) >> 2;
-          if (chunk < kb4 && mt < m_tiles)               // the pair's second row tile may not exist
-            *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4 + chunk) * 512 + lane * 16 + q * 4) =
-                sc_word;
-          sc_word = 0;
+        if (chunk < kb4 && mt < m_tiles)                 // the pair's second row tile may not exist
+          *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4 + chunk) * 512 + lane * 16 + q * 4) = sc_word;
+        continue;
+      }
+      // ---- accumulator fragment layout (16 rows at a time): thread t holds rows t/4 and t/4 + 8,
+      //      eight columns of each per block
+      const int64_t row_base = (int64_t)mt * C::BM + q * 32 + r8;     // + 16 mh + 8 rh
+      uint32_t sc_word[4] = {0u, 0u, 0u, 0u};            // rows r8 + 16 mh + 8 rh -> index 2 mh + rh
+#pragma unroll 1
+      for (int bb = 0; bb < 4; ++bb) {
+        const int blk = b0 + h * 4 + bb;
+        uint32_t bfrag[2][4][2];                         // [k chunk][n tile][2]
+        if (R_intra != nullptr) {
+          // lane l: row l % 8 of matrix l / 8; matrices (k 0-7, n), (k 8-15, n), (k 0-7, n+8), (k 8-15, n+8)
+          const uint32_t rb = ri_saddr + (uint32_t)(h * 4 + bb) * C::RI_BLOCK_BYTES +
+                              (uint32_t)(((lane >> 3) & 1) * 8 + (lane & 7)) * C::RI_ROW_BYTES +
+                              (uint32_t)(lane >> 4) * 16;
+#pragma unroll
+          for (int kc = 0; kc < 2; ++kc)
+#pragma unroll
+            for (int np = 0; np < 2; ++np)
+              ldmatrix_x4_trans(rb + kc * 16 * C::RI_ROW_BYTES + np * 32, bfrag[kc][2 * np][0], bfrag[kc][2 * np][1],
+                                bfrag[kc][2 * np + 1][0], bfrag[kc][2 * np + 1][1]);
         }
+#pragma unroll
+        for (int mh = 0; mh < 2; ++mh) {
+          uint32_t y[16];
+          tmem_ld_16x256b_x4(tacc + ((uint32_t)(16 * mh) << 16) + bb * 32, y);
+          tmem_ld_wait();
+          if (bb == 3 && mh == 1) {                      // this warp's share is read: tell the leader
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar(a), 0));
+          }
+          float acc[4][4];
+          if (R_intra != nullptr) {
+            uint32_t ah[8], am[8], al[8];                // A fragments: [k chunk * 4 + (n & 1) * 2 + row half]
+#pragma unroll
+            for (int n = 0; n < 4; ++n)
+#pragma unroll
+              for (int rh = 0; rh < 2; ++rh) {
+                const int ai = (n >> 1) * 4 + (n & 1) * 2 + rh;
+                split3_bf16x2(y[4 * n + 2 * rh], y[4 * n + 2 * rh + 1], ah[ai], am[ai], al[ai]);
+              }
+#pragma unroll
+            for (int n = 0; n < 4; ++n) { acc[n][0] = 0.f; acc[n][1] = 0.f; acc[n][2] = 0.f; acc[n][3] = 0.f; }
+#pragma unroll
+            for (int kc = 0; kc < 2; ++kc)
+#pragma unroll
+              for (int n = 0; n < 4; ++n) {
+                mma_16816_bf16(acc[n], al + 4 * kc, bfrag[kc][n]);
+                mma_16816_bf16(acc[n], am + 4 * kc, bfrag[kc][n]);
+                mma_16816_bf16(acc[n], ah + 4 * kc, bfrag[kc][n]);
+              }
+          } else {
+#pragma unroll
+            for (int n = 0; n < 4; ++n)
+#pragma unroll
+              for (int e = 0; e < 4; ++e) acc[n][e] = __uint_as_float(y[4 * n + e]);
+          }
+#pragma unroll
+          for (int rh = 0; rh < 2; ++rh) {
+            const float v[8] = {acc[0][2 * rh], acc[0][2 * rh + 1], acc[1][2 * rh], acc[1][2 * rh + 1],
+                                acc[2][2 * rh], acc[2][2 * rh + 1], acc[3][2 * rh], acc[3][2 * rh + 1]};
+            uint32_t word, sbyte;
+            quantize_row_fragment(v, p, word, sbyte);
+            const int64_t row = row_base + 16 * mh + 8 * rh;
+            if (row < M && blk < nblocks)
+              *reinterpret_cast<uint32_t*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16 + 4 * p) = word;
+            sc_word[2 * mh + rh] |= sbyte << (8 * bb);
+          }
+        }
+      }
+      if (p == 0 && chunk < kb4 && mt < m_tiles) {       // the pair's second row tile may not exist
+#pragma unroll
+        for (int rs = 0; rs < 4; ++rs)
+          *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4 + chunk) * 512 +
+                                       (r8 + 16 * (rs >> 1) + 8 * (rs & 1)) * 16 + q * 4) = sc_word[rs];
       }
     }
   }
