@@ -214,21 +214,39 @@ def main():
     launches = torq.torq_launch_count() - launches0
     ms_total = e0.elapsed_time(e1)
 
-    # ---- per-kernel durations, same launches issued as the two stage calls with events between
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    for i in range(args.steps):
-        b = sets[i % n_sets]
-        codes = b["ws"][: M * d // 2].view(M, d // 2)
-        scales = b["ws"][(M * d // 2 + 255) // 256 * 256:]
-        ev[i][0].record(stream)
-        torq.torq_rotate_quantize(b["X"], b["R"], b["Ri"], out_codes=codes, out_scales=scales)
-        ev[i][1].record(stream)
-        torq.torq_mxfp4_gemm(codes, scales, b["Wq"], b["Ws"], Y=b["Y"])
-        ev[i][2].record(stream)
+    # ---- per-kernel durations: K back-to-back launches of one kernel (operand sets rotated), one
+    # event pair around them on the launching stream; average = event time / K.  (With an event
+    # between every launch the launch latency that normally overlaps the previous kernel's tail
+    # would be charged to the kernel.)
+    def codes_scales(b):
+        return b["ws"][: M * d // 2].view(M, d // 2), b["ws"][(M * d // 2 + 255) // 256 * 256:][: torq.torq_scales_bytes(M, d)]
+
+    def timed_loop(fn):
+        for i in range(3):
+            fn(sets[i % n_sets])
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        for i in range(args.steps):
+            fn(sets[i % n_sets])
+        a1.record(stream)
+        torch.cuda.synchronize()
+        return a0.elapsed_time(a1) / args.steps * 1e-3
+
+    def gemm_only(b):
+        c, sc = codes_scales(b)
+        torq.torq_mxfp4_gemm(c, sc, b["Wq"], b["Ws"], Y=b["Y"])
+
+    def rot_only(b):
+        c, sc = codes_scales(b)
+        torq.torq_rotate_quantize(b["X"], b["R"], b["Ri"], out_codes=c, out_scales=sc)
+
+    t_gemm = timed_loop(gemm_only)
+    # few tokens: the rotation of the fused call is the split-K pair of kernels, which only runs with
+    # the workspace of the fused call; its time is the step minus the GEMM
+    t_rot = timed_loop(rot_only) if M > 128 else max(ms_total / args.steps * 1e-3 - t_gemm, 1e-9)
     barrier()
     clocks = sampler.stop()
-    t_rot = float(np.mean([e[0].elapsed_time(e[1]) for e in ev])) * 1e-3
-    t_gemm = float(np.mean([e[1].elapsed_time(e[2]) for e in ev])) * 1e-3
     assert torq.torq_last_device_error() == 0
 
     # ---- end to end through the public call with HOST buffers (pinned), copies inside the region

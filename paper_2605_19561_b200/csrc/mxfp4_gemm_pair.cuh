@@ -83,16 +83,33 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   cluster_sync_all();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  // Set-up above touched no global memory; from here on the previous kernel's results are needed.
+  // Set-up above touched no global memory.  The weights and their scales are constants of the
+  // layer, never the output of the kernel that runs just before this one, so the producer starts
+  // the first stages' W loads right away; everything else waits until that kernel has completed
+  // (its output, the activations' codes and scales, is what the A-side loads read).
   griddep_launch_dependents();
+  const int pre = pair < total_tiles ? (k_tiles < C::STAGES ? k_tiles : C::STAGES) : 0;
+  if (warp == 0) {
+    if (elect_one()) {
+      tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
+      tma_prefetch_desc(&tmSFA); tma_prefetch_desc(&tmSFB);
+      const int nt = pair / mp_tiles;
+      for (int kt = 0; kt < pre; ++kt) {
+        const uint32_t st = smem_base + kt * C::STAGE_BYTES;
+        const uint32_t leader_full = map_to_cta(full_bar(kt), 0);
+        if (rank == 0) mbar_arrive_expect_tx(full_bar(kt), 2 * C::STAGE_BYTES);
+        tma_load_2d_pair(st + C::A_BYTES, &tmB, kt * 128, nt * BN + (int)rank * (BN / 2), leader_full);
+        tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES, &tmSFB, kt * 256, 2 * nt, leader_full);
+        tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + 1024, &tmSFB, kt * 256, 2 * nt + 1,
+                         leader_full);
+      }
+    }
+    __syncwarp();
+  }
   griddep_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
-    if (elect_one()) {
-      tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
-      tma_prefetch_desc(&tmSFA); tma_prefetch_desc(&tmSFB);
-    }
     uint32_t it = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
@@ -104,16 +121,20 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
         const uint32_t leader_full = map_to_cta(full_bar(s), 0);
         if (elect_one()) {
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
+          const bool w_issued = it < (uint32_t)pre;      // W side of this stage went out before the wait above
+          if (rank == 0 && !w_issued) mbar_arrive_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
           tma_load_2d_pair(st, &tmA, kt * 128, mt * C::BM, leader_full);
-          tma_load_2d_pair(st + C::A_BYTES, &tmB, kt * 128, nt * BN + (int)rank * (BN / 2), leader_full);
+          if (!w_issued)
+            tma_load_2d_pair(st + C::A_BYTES, &tmB, kt * 128, nt * BN + (int)rank * (BN / 2), leader_full);
           // scale tiles: one row of the [row tile, K-chunk x 512 B] view per 128 rows, 1 KiB per
           // stage (two K-chunks); anything outside the buffer arrives as zeros (scale 2^-127,
           // multiplying operand data that is zero there as well).
           tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES, &tmSFA, kt * 256, mt, leader_full);
-          tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES, &tmSFB, kt * 256, 2 * nt, leader_full);
-          tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + 1024, &tmSFB, kt * 256, 2 * nt + 1,
-                           leader_full);
+          if (!w_issued) {
+            tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES, &tmSFB, kt * 256, 2 * nt, leader_full);
+            tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + 1024, &tmSFB, kt * 256, 2 * nt + 1,
+                             leader_full);
+          }
         }
         __syncwarp();
       }
@@ -245,7 +266,7 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         quarter32(v3, col0 + 96);
       }
     }
-    if (lane == 0) bulk_wait_group<0>();                 // every store of this warp has landed
+    if (lane == 0) bulk_wait_group_read<0>();            // shared memory must outlive the stores' reads
   }
 
   // ------------------------------------------------------------------ teardown

@@ -80,12 +80,32 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   // Set-up above touched no global memory; from here on the previous kernel's results are needed.
+  // R_inter is a constant of the layer, never the output of the kernel that runs just before this
+  // one: the producer starts the first stages' R_inter loads right away; the X loads and all
+  // other global accesses wait until that kernel has completed.
   griddep_launch_dependents();
+  const int pre = pair < total_tiles ? (k_tiles < C::STAGES ? k_tiles : C::STAGES) : 0;
+  if (warp == 0) {
+    if (elect_one()) {
+      tma_prefetch_desc(&tmX);
+      tma_prefetch_desc(&tmR);
+      const int nt = pair / mp_tiles;
+      for (int kt = 0; kt < pre; ++kt) {
+        const uint32_t st = smem_base + kt * C::STAGE_BYTES;
+        const uint32_t leader_full = map_to_cta(full_bar(kt), 0);
+        if (rank == 0) mbar_arrive_expect_tx(full_bar(kt), 2 * C::STAGE_BYTES);
+#pragma unroll
+        for (int b = 0; b < BN / 2 / 64; ++b)
+          tma_load_2d_pair(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR,
+                           nt * BN + (int)rank * (BN / 2) + b * 64, kt * C::BK, leader_full);
+      }
+    }
+    __syncwarp();
+  }
   griddep_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
-    if (elect_one()) { tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmR); }
     uint32_t it = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
@@ -97,12 +117,15 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
         const uint32_t leader_full = map_to_cta(full_bar(s), 0);
         if (elect_one()) {
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
+          const bool r_issued = it < (uint32_t)pre;      // R side of this stage went out before the wait above
+          if (rank == 0 && !r_issued) mbar_arrive_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
           tma_load_2d_pair(st, &tmX, kt * C::BK, mt * C::BM, leader_full);
+          if (!r_issued) {
 #pragma unroll
-          for (int b = 0; b < BN / 2 / 64; ++b)
-            tma_load_2d_pair(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR,
-                             nt * BN + (int)rank * (BN / 2) + b * 64, kt * C::BK, leader_full);
+            for (int b = 0; b < BN / 2 / 64; ++b)
+              tma_load_2d_pair(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR,
+                               nt * BN + (int)rank * (BN / 2) + b * 64, kt * C::BK, leader_full);
+          }
         }
         __syncwarp();
       }
