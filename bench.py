@@ -38,6 +38,15 @@ def profiled_traffic(kernel: str, workload: str):
     return float(m.group(1)) if m else None
 
 
+def hold_gpu(stream, ms: float = 5.0):
+    """Keeps the stream busy for a few milliseconds BEFORE the first timing event, so that the host
+    enqueues the timed launches ahead of the GPU.  Steps of a few tens of microseconds are otherwise
+    paced by the Python call overhead rather than by the kernels; the events still measure only
+    what lies between them on the device."""
+    with torch.cuda.stream(stream):
+        torch.cuda._sleep(int(ms * 1e-3 * 1.9e9))
+
+
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -206,6 +215,7 @@ def main():
     launches0 = torq.torq_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    hold_gpu(stream)
     e0.record(stream)
     for i in range(args.steps):
         step(i)
@@ -226,6 +236,7 @@ def main():
             fn(sets[i % n_sets])
         torch.cuda.synchronize()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        hold_gpu(stream)
         a0.record(stream)
         for i in range(args.steps):
             fn(sets[i % n_sets])
@@ -249,22 +260,52 @@ def main():
     clocks = sampler.stop()
     assert torq.torq_last_device_error() == 0
 
-    # ---- end to end through the public call with HOST buffers (pinned), copies inside the region
+    # ---- end to end through the public call with HOST buffers (pinned): every step copies its X
+    # host -> device, runs the layer, and copies its Y device -> host, all inside the timed region.
+    # Three streams with two device buffers each way: the upload of step i+1 and the download of
+    # step i-1 run beside the kernels of step i (PCIe is full duplex), ordered by events.
     Xh = X0.cpu().pin_memory()
-    Yh = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    Yh = [torch.empty((M, N), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
     e2e_steps = max(3, min(args.steps, 50))
-    b = sets[0]
-    for _ in range(3):
-        b["X"].copy_(Xh, non_blocking=True); step(0); Yh.copy_(b["Y"], non_blocking=True)
+    up, down = torch.cuda.Stream(), torch.cuda.Stream()
+    Xd = [sets[0]["X"], sets[1]["X"]]
+    Yd = [sets[0]["Y"], sets[1]["Y"]]
+    wsd = [sets[0]["ws"], sets[1]["ws"]]
+    p0 = sets[0]
+
+    def e2e_loop(n):
+        x_ready = [torch.cuda.Event() for _ in range(n)]
+        y_ready = [torch.cuda.Event() for _ in range(n)]
+        x_free = [torch.cuda.Event() for _ in range(n)]
+        y_free = [torch.cuda.Event() for _ in range(n)]
+        for i in range(n):
+            k = i & 1
+            with torch.cuda.stream(up):
+                if i >= 2:
+                    up.wait_event(x_free[i - 2])             # the kernels of step i-2 have read this buffer
+                Xd[k].copy_(Xh, non_blocking=True)
+                x_ready[i].record(up)
+            stream.wait_event(x_ready[i])
+            if i >= 2:
+                stream.wait_event(y_free[i - 2])             # the download of step i-2 has left this buffer
+            torq.torq_rotated_linear(Xd[k], p0["R"], p0["Ri"], p0["Wq"], p0["Ws"], Y=Yd[k], workspace=wsd[k])
+            x_free[i].record(stream)
+            y_ready[i].record(stream)
+            with torch.cuda.stream(down):
+                down.wait_event(y_ready[i])
+                Yh[k].copy_(Yd[k], non_blocking=True)
+                y_free[i].record(down)
+        stream.wait_stream(down)
+        stream.wait_stream(up)
+
+    e2e_loop(4)
     barrier()
     e0.record(stream)
-    for _ in range(e2e_steps):
-        b["X"].copy_(Xh, non_blocking=True)
-        step(0)
-        Yh.copy_(b["Y"], non_blocking=True)
+    e2e_loop(e2e_steps)
     e1.record(stream)
     barrier()
     ms_e2e = e0.elapsed_time(e1) / e2e_steps
+    Yh = Yh[0]
 
     from paper_2605_19561_b200.sharding import max_over_ranks
     ms_total, ms_e2e, t_rot, t_gemm = max_over_ranks([ms_total, ms_e2e, t_rot, t_gemm], device="cuda")
