@@ -21,6 +21,10 @@
  *     buffer always has torq_scales_bytes(rows, k) bytes: rows are padded to a multiple of 128
  *     and K-blocks to a multiple of 4.  Producers in this library write 0x00 (2^-127) into the
  *     padding rows; consumers never let padding reach a stored output.
+ *   - R_inter, R_intra, Wq and Ws are constants of the layer.  The tensor-core kernels may start
+ *     reading them while the kernel launched just before on the same stream is still finishing
+ *     (everything else waits for that kernel), so they must not be written by that kernel: put a
+ *     stream synchronisation or any other kernel between producing them and the first call.
  *   - Return value: TORQ_OK or a host-detected error; nothing is launched on error.  Conditions
  *     only the device can see (a bounded wait that ran out) are latched in an error word read by
  *     torq_last_device_error(); a kernel that hits one stops issuing work, drains and returns --
