@@ -51,7 +51,7 @@ CODEBOOK = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0], dtype=np.float64)
 E2M1_EMAX = 2  # largest power of two in the codebook is 2^2
 
 __all__ = [
-    "K_BLOCK", "CODEBOOK", "decode_bf16", "rotate", "round_to_f32", "shared_exponent",
+    "K_BLOCK", "CODEBOOK", "decode_bf16", "rotate", "rotate_structured", "round_to_f32", "shared_exponent",
     "quantize_mxfp4", "pack_codes", "unpack_codes", "dequantize", "gemm_dequant",
     "round_to_bf16", "merged_rotation", "prepare_weights", "scale_layout_offset",
     "scale_layout_bytes", "swizzle_scales", "unswizzle_scales", "rotated_linear",
@@ -90,6 +90,30 @@ def rotate(x_bits: np.ndarray, r_inter_bits, r_intra_bits) -> np.ndarray:
     z = np.empty_like(y)
     for b in range(nb):
         z[:, b * K_BLOCK:(b + 1) * K_BLOCK] = y[:, b * K_BLOCK:(b + 1) * K_BLOCK] @ ri[b]
+    return z
+
+
+def rotate_structured(x_bits: np.ndarray, r_b_bits, r_intra_bits) -> np.ndarray:
+    """Algorithm 3 steps 1-3 in the paper's own structure: one B x B inter-block matrix acting
+    across the blocks of a token (the same for every position inside a block) and one K x K
+    intra-block matrix shared by all blocks (Section 5; App. A.7 counts B^2 + K^2 parameters and
+    O(B^2 K) + O(B K^2) work per token).  Per token: reshape x to X [B, K] (step 1),
+    Y = R_B X (step 2), Z = Y R_intra (step 3); returned flattened, Z [M, d] float64.
+    r_b_bits [B, B] and r_intra_bits [K, K] are bfloat16 bit patterns; None = identity."""
+    x = decode_bf16(x_bits)
+    m, d = x.shape
+    assert d % K_BLOCK == 0
+    nb = d // K_BLOCK
+    z = np.empty((m, d), dtype=np.float64)
+    rb = None if r_b_bits is None else decode_bf16(r_b_bits)
+    ri = None if r_intra_bits is None else decode_bf16(r_intra_bits)
+    assert rb is None or rb.shape == (nb, nb)
+    assert ri is None or ri.shape == (K_BLOCK, K_BLOCK)
+    for t in range(m):
+        xt = x[t].reshape(nb, K_BLOCK)                  # step 1: B blocks (rows) of K elements
+        yt = xt if rb is None else rb @ xt               # step 2: Y = R_B X
+        zt = yt if ri is None else yt @ ri               # step 3: Z = Y R_intra
+        z[t] = zt.reshape(d)
     return z
 
 

@@ -204,3 +204,61 @@ def test_round_to_bf16_matches_library_cast():
     assert (O.round_to_bf16(y32) == lib).all()
     assert O.round_to_bf16(np.array([1.00390625]))[0] == 1.0        # 1 + 2^-8: tie -> even
     assert O.round_to_bf16(np.array([1.01171875]))[0] == 1.015625   # 1 + 3*2^-8: tie -> even (up)
+
+
+# ------------------------------------------------------------------ structured rotation (paper's form)
+def _structured_case(M, nb, seed):
+    g = np.random.default_rng(seed)
+    xb = I.to_bf16_bits(g.standard_t(3.0, size=(M, nb * 32)))
+    rb = I.to_bf16_bits(I.orthogonal(nb, g))
+    ri = I.to_bf16_bits(I.orthogonal(32, g))
+    return xb, rb, ri
+
+
+def test_structured_rotation_equals_the_dense_one_with_kronecker_operands():
+    """R_B acting across blocks is the dense inter rotation kron(R_B^T, I_32) in the row-vector
+    convention, and one shared R_intra is the same matrix in every block: the two oracle
+    functions must agree to summation-order rounding."""
+    for M, nb in [(5, 4), (3, 8), (7, 16)]:
+        xb, rb, ri = _structured_case(M, nb, seed=nb)
+        z = O.rotate_structured(xb, rb, ri)
+        RB, RI = O.decode_bf16(rb), O.decode_bf16(ri)
+        dense = np.kron(RB.T, np.eye(32))                 # [32b+k, 32b'+k'] = R_B[b', b] delta(k, k')
+        # the dense oracle takes bf16 bit patterns; every entry of `dense` is an entry of R_B or 0
+        zd = O.rotate(xb, I.to_bf16_bits(dense), I.to_bf16_bits(np.stack([RI] * nb)))
+        np.testing.assert_allclose(z, zd, rtol=1e-12, atol=1e-12)
+        # each step alone
+        np.testing.assert_allclose(O.rotate_structured(xb, rb, None), O.rotate(xb, I.to_bf16_bits(dense), None),
+                                   rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(O.rotate_structured(xb, None, ri),
+                                   O.rotate(xb, None, I.to_bf16_bits(np.stack([RI] * nb))), rtol=1e-12, atol=1e-12)
+
+
+def test_structured_rotation_against_pure_python_loops_and_exact_cases():
+    xb, rb, ri = _structured_case(2, 4, seed=99)
+    x, RB, RI = O.decode_bf16(xb), O.decode_bf16(rb), O.decode_bf16(ri)
+    z = O.rotate_structured(xb, rb, ri)
+    for t in range(2):
+        for bo in range(4):
+            for j in range(32):
+                acc = 0.0
+                for k in range(32):
+                    y = 0.0
+                    for b in range(4):
+                        y += RB[bo, b] * x[t, 32 * b + k]        # Y = R_B X: mixes blocks, keeps position k
+                    acc += y * RI[k, j]                            # Z = Y R_intra: mixes positions
+                assert abs(z[t, 32 * bo + j] - acc) <= 1e-12 * max(1.0, abs(acc))
+    # a block permutation moves whole blocks, a position permutation acts inside every block alike
+    g = np.random.default_rng(1)
+    xi = g.integers(-8, 9, size=(3, 4 * 32)).astype(np.float64)
+    pb, pk = g.permutation(4), g.permutation(32)
+    PB = np.zeros((4, 4)); PB[np.arange(4), pb] = 1                # (PB X)[b'] = X[pb[b']]
+    PK = np.zeros((32, 32)); PK[pk, np.arange(32)] = 1             # (Y PK)[., j] = Y[., pk[j]]
+    z = O.rotate_structured(I.to_bf16_bits(xi), I.to_bf16_bits(PB), I.to_bf16_bits(PK))
+    want = xi.reshape(3, 4, 32)[:, pb][:, :, pk].reshape(3, 128)
+    assert np.array_equal(z, want)
+    # energy conservation (total variance across blocks, App. A.1) with the float64 orthogonal factors
+    Q, P = I.orthogonal(4, g), I.orthogonal(32, g)
+    xt = O.decode_bf16(xb)[0].reshape(4, 32)
+    zt = Q @ xt @ P
+    assert abs((zt ** 2).sum() - (xt ** 2).sum()) <= 1e-10 * (xt ** 2).sum()
