@@ -66,6 +66,23 @@ torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void*
                                  int64_t M, int64_t d, void* out_codes, void* out_scales,
                                  void* stream);
 
+/* Algorithm 3 steps 1-4 with the rotation in the paper's own structure (Section 5; App. A.7 counts
+ * B^2 + K^2 parameters and O(B^2 K) + O(B K^2) work per token): ONE inter-block matrix R_B that
+ * mixes the B = d/32 blocks of a token, the same for each of the 32 positions, and ONE intra-block
+ * matrix shared by all blocks.  Per token, with X the token's [B, 32] reshape:
+ *   Y = R_B X        y[32 b' + k] = sum_b  R_B[b'][b] x[32 b + k]
+ *   Z = Y R_intra    z[32 b' + j] = sum_k  y[32 b' + k] R_intra[k][j]
+ * then Eq. 1 as in torq_rotate_quantize (same output layouts).  Equivalent to torq_rotate_quantize
+ * with R_inter = kron(R_B^T, I_32) and R_intra repeated for every block, at 2 d (B + 32) instead of
+ * 2 d^2 flop per token.
+ *   X [M, d] bf16;  R_B [d/32, d/32] bf16 (required);  R_intra [32, 32] bf16 or NULL = identity
+ * Requires d % 256 == 0, 16-byte aligned pointers.  fp32 accumulation: step 2 on the tensor cores
+ * with exact bf16 products, step 3 with y split into three bf16 terms (y to 2^-24) against the
+ * bf16 R_intra on the warp-level tensor-core path. */
+torq_status torq_rotate_quantize_structured(const void* X, const void* R_B, const void* R_intra,
+                                            int64_t M, int64_t d, void* out_codes, void* out_scales,
+                                            void* stream);
+
 /* Algorithm 3 step 5 (option B): Y[m,n] = sum_k a^[m,k] w^[n,k], a^/w^ the dequantized MXFP4
  * values (codeword x 2^e), fp32 accumulation on the block-scaled FP4 tensor cores.
  *   Aq [M, K/2] u8, As scales of A (tiled, torq_scales_bytes(M, K))

@@ -127,6 +127,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* m, 
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(bar)
       : "memory");
 }
+// 3-D tiled load (c0 innermost), same rules.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, int32_t c0, int32_t c1,
+                                            int32_t c2, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
 // Untiled bulk copy, global -> shared; both addresses 16-byte aligned, bytes % 16 == 0.
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes,
                                              uint32_t bar) {
@@ -204,9 +213,10 @@ __device__ __forceinline__ void tmem_ld_wait() {
 
 // ---- shared-memory matrix descriptors ----------------------------------------------------------
 // 64-bit descriptor: [0,14) start>>4, [16,30) leading byte offset>>4, [32,46) stride byte
-// offset>>4, [46,48) version (1 on sm_100), [61,64) swizzle (0 none, 2 = 128 B).
+// offset>>4, [46,48) version (1 on sm_100), [61,64) swizzle (0 none, 2 = 128 B, 4 = 64 B).
 constexpr uint64_t kDescVersion = 1ull << 46;
 constexpr uint64_t kSwizzle128 = 2ull << 61;
+constexpr uint64_t kSwizzle64 = 4ull << 61;
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes,
                                               uint32_t sbo_bytes, uint64_t swizzle) {
   return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16) |

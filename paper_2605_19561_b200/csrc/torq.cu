@@ -12,6 +12,7 @@
 #include "rotate_quantize.cuh"
 #include "rotate_quantize_pair.cuh"
 #include "rotate_splitk.cuh"
+#include "rotate_structured.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -94,6 +95,7 @@ static DeviceState* device_state() {
               opt_in_smem(rotate_quantize_kernel<128>, RotCfg<128>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_pair_kernel, RotPairCfg::SMEM_BYTES) &&
               opt_in_smem(rotate_splitk_kernel, RotSplitCfg::SMEM_BYTES) &&
+              opt_in_smem(rotate_structured_kernel, RotStructCfg::SMEM_BYTES) &&
               opt_in_smem(mxfp4_gemm_pair_kernel, GemmPairCfg::SMEM_BYTES);
     if (!ok) return nullptr;
     st.rot_pairs = max_active_pairs(rotate_quantize_pair_kernel, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
@@ -118,6 +120,18 @@ static bool encode_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, 
   return g_encode(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// X [M, d] bf16 seen as (position k: 32, token: M, block: d/32) with box (32, 1, 64): the box lands
+// in shared memory as 64 rows (blocks) of 64 bytes (one token's 32 positions), 64-byte swizzle.
+static bool encode_x_blocks_3d(CUtensorMap* map, const void* base, uint64_t M, uint64_t d) {
+  cuuint64_t dims[3] = {32, M, d / 32};
+  cuuint64_t strides[2] = {d * 2, 64};
+  cuuint32_t box[3] = {32, 1, 64};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -311,6 +325,37 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
 torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void* R_intra, int64_t M,
                                  int64_t d, void* out_codes, void* out_scales, void* stream) {
   return rotate_quantize_impl(X, R_inter, R_intra, M, d, out_codes, out_scales, nullptr, 0, stream);
+}
+
+torq_status torq_rotate_quantize_structured(const void* X, const void* R_B, const void* R_intra, int64_t M,
+                                            int64_t d, void* out_codes, void* out_scales, void* stream) {
+  if (!X || !R_B || !out_codes || !out_scales) return TORQ_ERR_NULL;
+  if (M < 1 || d < 256 || d % 256 != 0 || M > (1 << 30) || d > (1 << 24)) return TORQ_ERR_SHAPE;
+  if (!aligned16(X) || !aligned16(R_B) || !aligned16(out_codes) || !aligned16(out_scales) ||
+      (R_intra && !aligned16(R_intra)))
+    return TORQ_ERR_ALIGN;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t nb = d / 32;
+  CUtensorMap tmRB, tmX3;
+  if (!encode_2d(&tmRB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_B, (uint64_t)nb, (uint64_t)nb, 128, 64) ||
+      !encode_x_blocks_3d(&tmX3, X, (uint64_t)M, (uint64_t)d))
+    return TORQ_ERR_LAUNCH;
+  const int64_t tiles = ((nb + 127) / 128) * ((M + RotStructCfg::TOK - 1) / RotStructCfg::TOK);
+  const int grid = (int)(tiles < st->sm_count ? tiles : st->sm_count);
+  launch_tc(rotate_structured_kernel, 1, grid, RotStructCfg::THREADS, RotStructCfg::SMEM_BYTES, s, tmRB, tmX3,
+            static_cast<const __nv_bfloat16*>(R_intra), static_cast<uint8_t*>(out_codes),
+            static_cast<uint8_t*>(out_scales), (int)M, (int)d, st->err_word);
+  if (launch_status() != TORQ_OK) return TORQ_ERR_LAUNCH;
+  const int64_t kc = (nb + 3) / 4 * 4, mpad = (M + 127) / 128 * 128;
+  const int64_t pad = (mpad - M) * kc + M * (kc - nb);
+  if (pad > 0) {
+    scale_padding_kernel<<<ew_grid(pad, 256, st->sm_count), 256, 0, s>>>(static_cast<uint8_t*>(out_scales), M, nb);
+    return launch_status();
+  }
+  return TORQ_OK;
 }
 
 torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, const void* Ws, int64_t M,

@@ -36,6 +36,8 @@ def lib() -> ctypes.CDLL:
     vp, i64, sz, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_int
     L.torq_rotate_quantize.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp]
     L.torq_rotate_quantize.restype = ci
+    L.torq_rotate_quantize_structured.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp]
+    L.torq_rotate_quantize_structured.restype = ci
     L.torq_mxfp4_gemm.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, ci, vp]
     L.torq_mxfp4_gemm.restype = ci
     L.torq_rotated_linear.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, vp, sz, vp, vp, vp]
@@ -130,6 +132,21 @@ def torq_rotate_quantize(X, R_inter, R_intra, out_codes=None, out_scales=None, s
         out_scales = torch.empty(torq_scales_bytes(M, d), dtype=torch.uint8, device=X.device)
     _raise(lib().torq_rotate_quantize(_ptr(X), _ptr(R_inter), _ptr(R_intra), M, d, _ptr(out_codes),
                                       _ptr(out_scales), _stream(stream)), "torq_rotate_quantize")
+    return out_codes, out_scales
+
+
+def torq_rotate_quantize_structured(X, R_B, R_intra, out_codes=None, out_scales=None, stream=None):
+    """X [M,d] bf16, R_B [d/32,d/32] bf16 (mixes the blocks of a token), R_intra [32,32] bf16 or None
+    (shared by all blocks): the rotation in the structure the paper gives it."""
+    M, d = X.shape
+    for t, n in ((X, "X"), (R_B, "R_B"), (R_intra, "R_intra")):
+        _check(t, torch.bfloat16, n)
+    if out_codes is None:
+        out_codes = torch.empty((M, d // 2), dtype=torch.uint8, device=X.device)
+    if out_scales is None:
+        out_scales = torch.empty(torq_scales_bytes(M, d), dtype=torch.uint8, device=X.device)
+    _raise(lib().torq_rotate_quantize_structured(_ptr(X), _ptr(R_B), _ptr(R_intra), M, d, _ptr(out_codes),
+                                                 _ptr(out_scales), _stream(stream)), "torq_rotate_quantize_structured")
     return out_codes, out_scales
 
 
