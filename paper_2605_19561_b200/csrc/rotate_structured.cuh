@@ -2,22 +2,27 @@
 // App. A.7): ONE B x B inter-block matrix R_B that mixes the B = d/32 blocks of a token position
 // by position (Y = R_B X on the token's B x 32 reshape) and ONE 32 x 32 intra-block matrix shared
 // by all blocks (Z = Y R_intra).  Per token that is 2 d (B + 32) flop instead of 2 d^2: the kernel
-// is bound by reading X and writing the codes, not by the tensor pipe.
+// should be bound by reading X and writing the codes, so both steps run on the tcgen05 tensor
+// cores and the CUDA cores only split, quantize and store.
 //
-// Step 2 as a tensor-core contraction without moving X: D[b', (t, k)] = sum_b R_B[b', b] X[b, (t, k)]
-//   A operand = R_B tile [128 b' x 64 b], K-major (b contiguous), plain 2-D TMA;
+// Step 2 without moving X: D1[b', (t, k)] = sum_b R_B[b', b] X[b, (t, k)]
+//   A operand = R_B tile [128 b' x 64 b], K-major (b contiguous), 2-D TMA, 128-byte swizzle;
 //   B operand = X, N-major with the 64-byte swizzle: row b of a token's sub-tile is that token's
 //   32 positions of block b (64 contiguous bytes of X).  A 3-D tensor map over X with dimensions
 //   (k: 32, stride 1; token: M, stride d; block: B, stride 32) and box (32, 1, 64) lands in shared
 //   memory in exactly that layout, one 4 KiB sub-tile per token.  (With the 128-byte swizzle a
 //   64-byte inner box row is padded to a 128-byte pitch, so two tokens cannot share a line.)
-// The accumulator then has lanes = output block b' and columns = (token, position): the 32 columns
-// of one token are one (token, block) row of step 3, which the epilogue reads in the warp-MMA
-// fragment layout, rotates on the warp-level tensor-core path (three bf16 terms of y against
-// R_intra, whose fragments stay in registers for the whole kernel) and quantizes (Eq. 1).
+//   D1 has lanes = output block b' and columns = (token, position).
+// Step 3 as a second contraction: D2[b', j] = sum_k y[b', k] R_intra[k, j] per token, with y (fp32,
+//   read back from tensor memory) split into three bf16 terms y = hi + mid + lo (to 2^-24) that the
+//   epilogue writes to shared memory as K-major A tiles (rows of 64 bytes, 64-byte swizzle), and
+//   R_intra (bf16, exact) as the N-major B tile.  Six small MMAs (M 128, N 32, K 16) per token.
+//   D2 has lanes = b', 32 columns per token: one thread reads one (token, block) row and runs Eq. 1.
 //
-// Persistent, warp-specialised: warp 0 TMA producer, warp 1 MMA issuer, warps 2..9 epilogue
-// (lane quarter w % 4, tokens 4 * ((w - 2) / 4) .. + 3 of the tile's eight).
+// Persistent, warp-specialised: warp 0 TMA producer, warp 1 issues both kinds of MMA, warps 2..9
+// epilogue in two groups of four (lane quarter w % 4; group g = (w - 2) / 4 owns tokens 2g, 2g + 1
+// of the tile's four).  Per tile a group splits token 0, hands it to the MMA warp, splits token 1
+// while those MMAs run, then quantizes both.
 #pragma once
 #include <cuda_bf16.h>
 #include "quantize.cuh"
@@ -27,18 +32,20 @@ namespace torq {
 
 struct RotStructCfg {
   static constexpr int BM = 128;                       // output blocks b' per tile (MMA M)
-  static constexpr int TOK = 8;                        // tokens per tile
-  static constexpr int BN = TOK * 32;                  // MMA N = 256
+  static constexpr int TOK = 4;                        // tokens per tile
+  static constexpr int BN = TOK * 32;                  // step-2 MMA N = 128
   static constexpr int BK = 64;                        // input blocks b per stage
   static constexpr int A_BYTES = BM * BK * 2;          // 16 KiB
   static constexpr int B_BOX_BYTES = 32 * BK * 2;      // one token x 64 blocks = 4 KiB
-  static constexpr int B_BYTES = TOK * B_BOX_BYTES;
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 48 KiB
-  static constexpr int STAGES = 4;
-  static constexpr int RI_ROW_BYTES = 80;              // 32 bf16 + 16 B pad: conflict-free ldmatrix
-  static constexpr int RI_BYTES = 32 * RI_ROW_BYTES;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + RI_BYTES + 256 + 1024;
-  static constexpr int NACC = 2;
+  static constexpr int B_BYTES = TOK * B_BOX_BYTES;    // 16 KiB
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 32 KiB
+  static constexpr int STAGES = 3;
+  static constexpr int A2_TERM_BYTES = BM * 64;        // 128 rows x 32 bf16 = 8 KiB
+  static constexpr int A2_TOKEN_BYTES = 3 * A2_TERM_BYTES;
+  static constexpr int A2_BYTES = TOK * A2_TOKEN_BYTES;   // 96 KiB
+  static constexpr int RI_BYTES = 32 * 64;             // R_intra, 64-byte swizzle
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + A2_BYTES + RI_BYTES + 256 + 1024;
+  static constexpr int ACC2_COL = 2 * BN;              // D1 double-buffered in columns [0, 256)
   static constexpr int TMEM_COLS = 512;
   static constexpr int THREADS = 320;
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
@@ -55,13 +62,17 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  uint8_t* ri_smem = smem_gen + C::STAGES * C::STAGE_BYTES;
-  const uint32_t bar_off = C::STAGES * C::STAGE_BYTES + C::RI_BYTES;
+  const uint32_t a2_base = smem_base + C::STAGES * C::STAGE_BYTES;
+  const uint32_t ri_base = a2_base + C::A2_BYTES;
+  const uint32_t bar_off = C::STAGES * C::STAGE_BYTES + C::A2_BYTES + C::RI_BYTES;
   const uint32_t bar_base = smem_base + bar_off;
+  // barrier map (8 bytes each)
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };
-  auto accf_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + a); };
-  auto acce_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + C::NACC + a); };
+  auto acc1f_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + a); };
+  auto acc1e_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + 2 + a); };
+  auto a2f_bar = [&](int tok) { return bar_base + 8u * (2 * C::STAGES + 4 + tok); };   // epilogue -> MMA
+  auto a2d_bar = [&](int tok) { return bar_base + 8u * (2 * C::STAGES + 8 + tok); };   // MMA -> epilogue
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + bar_off + 192);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(smem_gen + bar_off + 200);
 
@@ -72,10 +83,12 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
   const int total_tiles = b_tiles * t_tiles;
   const int k_tiles = (nblocks + C::BK - 1) / C::BK;
   const int kb4 = (nblocks + 3) / 4;
+  const bool intra = R_intra != nullptr;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < C::NACC; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 8); }
+    for (int a = 0; a < 2; ++a) { mbar_init(acc1f_bar(a), 1); mbar_init(acc1e_bar(a), 8); }
+    for (int t = 0; t < C::TOK; ++t) { mbar_init(a2f_bar(t), 4); mbar_init(a2d_bar(t), 1); }
     *cta_abort = 0;
     fence_mbar_init();
   }
@@ -111,20 +124,24 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    constexpr uint32_t idesc = idesc_bf16(128, BN, /*A MN-major*/ false, /*B MN-major*/ true);
-    uint32_t it = 0, tcount = 0;
+    // ------------------------------------------------------------------ MMA issuer (both steps)
+    constexpr uint32_t idesc1 = idesc_bf16(128, BN, /*A MN-major*/ false, /*B MN-major*/ true);
+    constexpr uint32_t idesc2 = idesc_bf16(128, 32, /*A MN-major*/ false, /*B MN-major*/ true);
+    const uint64_t rdesc = make_desc(ri_base, 2048, 512, kSwizzle64);
+    uint32_t it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-      const int a = tcount % C::NACC;
-      if (!mbar_wait_warp(acce_bar(a), ((tcount / C::NACC) & 1) ^ 1, cta_abort, err_word,
-                          SITE_MMA_ACC_EMPTY)) { ok = false; break; }
+    // step 2 of tile number `tc` (this CTA's count) into D1 buffer tc % 2
+    auto step2 = [&](uint32_t tc) {
+      const int a = tc & 1;
+      if (!mbar_wait_warp(acc1e_bar(a), ((tc >> 1) & 1) ^ 1, cta_abort, err_word, SITE_MMA_ACC_EMPTY)) {
+        ok = false; return;
+      }
       tc_fence_after_sync();
       const uint32_t acc = tmem_base + a * BN;
       for (int kt = 0; kt < k_tiles; ++kt, ++it) {
         const int s = it % C::STAGES;
         if (!mbar_wait_warp(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
-          ok = false; break;
+          ok = false; return;
         }
         tc_fence_after_sync();
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
@@ -135,101 +152,142 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
         if (elect_one()) {
 #pragma unroll
           for (int j = 0; j < C::BK / 16; ++j)          // 16 k-rows = 1 KiB
-            mma_bf16(acc, adesc + 2 * j, bdesc + 64 * j, idesc, (kt | j) != 0);
+            mma_bf16(acc, adesc + 2 * j, bdesc + 64 * j, idesc1, (kt | j) != 0);
           tc_commit(empty_bar(s));
         }
         __syncwarp();
       }
-      if (ok && elect_one()) tc_commit(accf_bar(a));
+      if (elect_one()) tc_commit(acc1f_bar(a));
       __syncwarp();
+    };
+    uint32_t tcount = 0;
+    if (blockIdx.x < (unsigned)total_tiles) step2(0);
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      if (tile + (int)gridDim.x < total_tiles) step2(tcount + 1);    // next tile's step 2 runs beside this tile's step 3
+      if (!ok) break;
+      if (intra) {
+        for (int tok = 0; tok < C::TOK && ok; ++tok) {
+          const int tq = (tok & 1) * 2 + (tok >> 1);     // order: group 0 token 0, group 1 token 0, then tokens 1
+          if (!mbar_wait_warp(a2f_bar(tq), tcount & 1, cta_abort, err_word, SITE_MMA_FULL)) { ok = false; break; }
+          tc_fence_after_sync();
+          if (elect_one()) {
+            const uint32_t d2 = tmem_base + C::ACC2_COL + tq * 32;
+#pragma unroll
+            for (int term = 0; term < 3; ++term) {
+              const uint64_t adesc = make_desc(a2_base + tq * C::A2_TOKEN_BYTES + term * C::A2_TERM_BYTES, 16, 512,
+                                               kSwizzle64);
+              mma_bf16(d2, adesc, rdesc, idesc2, term != 0);
+              mma_bf16(d2, adesc + 2, rdesc + 64, idesc2, 1);        // k 16..31: +32 B in A rows, +16 rows of R
+            }
+            tc_commit(a2d_bar(tq));
+          }
+          __syncwarp();
+        }
+      }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (8 warps)
+    // ------------------------------------------------------------------ epilogue (two groups of 4 warps)
     const int q = warp & 3;
-    const int h = (warp - 2) >> 2;
+    const int g = (warp - 2) >> 2;
     const int et = (warp - 2) * 32 + lane;
-    const int p = lane & 3, r8 = lane >> 2;
-    // R_intra -> shared memory (bf16 rows of 80 bytes) -> B fragments, once
-    uint32_t bfrag[2][4][2];
-    if (R_intra != nullptr) {
+    if (intra) {
+      // R_intra -> shared memory once: row k = 64 bytes, 16-byte piece c stored at c ^ ((k >> 1) & 3)
       if (et < 128) {
-        const int i = et >> 2, c = (et & 3) * 8;
-        *reinterpret_cast<uint4*>(ri_smem + i * C::RI_ROW_BYTES + c * 2) =
-            __ldg(reinterpret_cast<const uint4*>(R_intra + i * 32 + c));
+        const int k = et >> 2, c = et & 3;
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(R_intra + k * 32 + c * 8));
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                     ::"r"(ri_base + (uint32_t)k * 64 + (uint32_t)((c ^ ((k >> 1) & 3)) << 4)), "r"(v.x), "r"(v.y),
+                       "r"(v.z), "r"(v.w) : "memory");
       }
+      fence_proxy_async_smem();                          // visible to the tensor core's reads
       named_barrier_sync(1, 256);
-      const uint32_t rb = smem_u32(ri_smem) + (uint32_t)(((lane >> 3) & 1) * 8 + (lane & 7)) * C::RI_ROW_BYTES +
-                          (uint32_t)(lane >> 4) * 16;
-#pragma unroll
-      for (int kc = 0; kc < 2; ++kc)
-#pragma unroll
-        for (int np = 0; np < 2; ++np)
-          ldmatrix_x4_trans(rb + kc * 16 * C::RI_ROW_BYTES + np * 32, bfrag[kc][2 * np][0], bfrag[kc][2 * np][1],
-                            bfrag[kc][2 * np + 1][0], bfrag[kc][2 * np + 1][1]);
     }
+    const int row = q * 32 + lane;                       // b' within the tile = tensor-memory lane
+    const uint32_t row_sw = (uint32_t)((row >> 1) & 3);
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
       const int bt = tile % b_tiles, tg = tile / b_tiles;
-      const int a = tcount % C::NACC;
-      ok = mbar_wait(accf_bar(a), (tcount / C::NACC) & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
+      const int a = tcount & 1;
+      ok = mbar_wait(acc1f_bar(a), (tcount >> 1) & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + h * 128;
-      const int blk_base = bt * C::BM + q * 32 + r8;     // + 16 mh + 8 rh
+      const uint32_t t1 = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
+      const int blk = bt * C::BM + row;
+      auto emit = [&](const float (&z)[32], int64_t token) {
+        uint4 cw;
+        uint32_t sbyte;
+        quantize_block32(z, cw, sbyte);
+        if (token < M && blk < nblocks) {
+          *reinterpret_cast<uint4*>(codes + token * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+          scales[scale_offset(token, blk, kb4)] = (uint8_t)sbyte;
+        }
+      };
+      if (!intra) {
 #pragma unroll 1
-      for (int t = 0; t < 4; ++t) {
-        const int64_t token = (int64_t)tg * C::TOK + h * 4 + t;
-#pragma unroll
-        for (int mh = 0; mh < 2; ++mh) {
-          uint32_t y[16];
-          tmem_ld_16x256b_x4(tacc + ((uint32_t)(16 * mh) << 16) + t * 32, y);
+        for (int j = 0; j < 2; ++j) {
+          uint32_t y[32];
+          tmem_ld_32x32(t1 + (2 * g + j) * 32, y);
           tmem_ld_wait();
-          if (t == 3 && mh == 1) {                       // this warp's share of the accumulator is read
+          if (j == 1) {
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acce_bar(a));
+            if (lane == 0) mbar_arrive(acc1e_bar(a));
           }
-          float acc[4][4];
-          if (R_intra != nullptr) {
-            uint32_t ah[8], am[8], al[8];
+          float z[32];
 #pragma unroll
-            for (int n = 0; n < 4; ++n)
-#pragma unroll
-              for (int rh = 0; rh < 2; ++rh) {
-                const int ai = (n >> 1) * 4 + (n & 1) * 2 + rh;
-                split3_bf16x2(y[4 * n + 2 * rh], y[4 * n + 2 * rh + 1], ah[ai], am[ai], al[ai]);
-              }
-#pragma unroll
-            for (int n = 0; n < 4; ++n) { acc[n][0] = 0.f; acc[n][1] = 0.f; acc[n][2] = 0.f; acc[n][3] = 0.f; }
-#pragma unroll
-            for (int kc = 0; kc < 2; ++kc)
-#pragma unroll
-              for (int n = 0; n < 4; ++n) {
-                mma_16816_bf16(acc[n], al + 4 * kc, bfrag[kc][n]);
-                mma_16816_bf16(acc[n], am + 4 * kc, bfrag[kc][n]);
-                mma_16816_bf16(acc[n], ah + 4 * kc, bfrag[kc][n]);
-              }
-          } else {
-#pragma unroll
-            for (int n = 0; n < 4; ++n)
-#pragma unroll
-              for (int e = 0; e < 4; ++e) acc[n][e] = __uint_as_float(y[4 * n + e]);
-          }
-#pragma unroll
-          for (int rh = 0; rh < 2; ++rh) {
-            const float v[8] = {acc[0][2 * rh], acc[0][2 * rh + 1], acc[1][2 * rh], acc[1][2 * rh + 1],
-                                acc[2][2 * rh], acc[2][2 * rh + 1], acc[3][2 * rh], acc[3][2 * rh + 1]};
-            uint32_t word, sbyte;
-            quantize_row_fragment(v, p, word, sbyte);
-            const int blk = blk_base + 16 * mh + 8 * rh;
-            if (token < M && blk < nblocks) {
-              *reinterpret_cast<uint32_t*>(codes + token * (int64_t)(d / 2) + (int64_t)blk * 16 + 4 * p) = word;
-              if (p == 0) scales[scale_offset(token, blk, kb4)] = (uint8_t)sbyte;
-            }
-          }
+          for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(y[i]);
+          emit(z, (int64_t)tg * C::TOK + 2 * g + j);
         }
+        continue;
+      }
+      // ---- split y into three bf16 terms, one A tile row (64 B) per term and token
+#pragma unroll 1
+      for (int j = 0; j < 2; ++j) {
+        const int tok = 2 * g + j;
+        uint32_t y[32];
+        tmem_ld_32x32(t1 + tok * 32, y);
+        tmem_ld_wait();
+        if (j == 1) {                                    // this warp's share of D1 is read
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc1e_bar(a));
+        }
+        const uint32_t dst = a2_base + tok * C::A2_TOKEN_BYTES + (uint32_t)row * 64;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {                    // 8 values = one 16-byte piece per term
+          uint32_t hi[4], mid[4], lo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) split3_bf16x2(y[8 * c + 2 * e], y[8 * c + 2 * e + 1], hi[e], mid[e], lo[e]);
+          const uint32_t off = (uint32_t)((c ^ row_sw) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(dst + off), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(dst + C::A2_TERM_BYTES + off), "r"(mid[0]), "r"(mid[1]), "r"(mid[2]), "r"(mid[3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(dst + 2 * C::A2_TERM_BYTES + off), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(a2f_bar(tok));        // four warps (the lane quarters) per token
+      }
+      // ---- D2 -> Eq. 1 -> codes and scales
+#pragma unroll 1
+      for (int j = 0; j < 2; ++j) {
+        const int tok = 2 * g + j;
+        ok = mbar_wait(a2d_bar(tok), tcount & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        uint32_t y[32];
+        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + C::ACC2_COL + tok * 32, y);
+        tmem_ld_wait();
+        tc_fence_before_sync();
+        float z[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(y[i]);
+        emit(z, (int64_t)tg * C::TOK + tok);
       }
     }
   }
