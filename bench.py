@@ -256,6 +256,19 @@ def main():
     # few tokens: the rotation of the fused call is the split-K pair of kernels, which only runs with
     # the workspace of the fused call; its time is the step minus the GEMM
     t_rot = timed_loop(rot_only) if M > 128 else max(ms_total / args.steps * 1e-3 - t_gemm, 1e-9)
+    # the same activations through the rotation in the paper's own structure (one B x B matrix
+    # across blocks, one shared intra-block matrix): reported beside the dense-R_inter path
+    t_struct = None
+    if d % 256 == 0:
+        RB = I.bf16_bits_to_tensor(I.to_bf16_bits(I.orthogonal(d // 32, np.random.Generator(
+            np.random.PCG64(I.BASE_SEED + 100 * cfg.cfg_id + 5)))), "cuda")
+        Ri1 = Ri0[0].contiguous()
+
+        def struct_only(b):
+            c, sc = codes_scales(b)
+            torq.torq_rotate_quantize_structured(b["X"], RB, Ri1, out_codes=c, out_scales=sc)
+
+        t_struct = timed_loop(struct_only)
     barrier()
     clocks = sampler.stop()
     assert torq.torq_last_device_error() == 0
@@ -353,6 +366,13 @@ def main():
             "rotate_quant_GBps": rot_bytes / t_rot / 1e9, "rotate_quant_TFLOPs": rot_flop / t_rot / 1e12,
             "gemm_TFLOPs": gemm_flop / t_gemm / 1e12,
             "roofline": dominant, "roofline_other_kernel": other,
+            "structured_rotation": None if t_struct is None else (lambda nbytes: {
+                "kernel": "rotate_structured_kernel", "what": "rotate+quantize with R_inter = R_B (x) I_32 and one shared "
+                "R_intra (the paper's structure, 2d(B+32) flop per token) on the same activations", "bound": "hbm",
+                "ms_per_launch": t_struct * 1e3, "achieved": nbytes / t_struct / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": nbytes / t_struct / 1e9 / pk["hbm_gbs"], "algorithmic_bytes": nbytes,
+                "speedup_over_dense_rotation": t_rot / t_struct})(
+                    2.0 * M * d + 2.0 * (d // 32) ** 2 + 2048.0 + M * d / 2 + M * d / 32),
             "e2e": {"value": world * M / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": Xh.numel() * 2,
                     "d2h_bytes_per_step": Yh.numel() * 2},
             "gpu_launches": int(launches), "clocks": clocks,
