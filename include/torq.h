@@ -164,6 +164,15 @@ torq_status torq_swizzle_scales(const void* linear_scales, int64_t rows, int64_t
 torq_status torq_merge_rotations(const void* R_inter, const void* R_intra, int64_t d,
                                  void* R_merged_f32, void* stream);
 
+/* Measurement tool (no counterpart in the paper): runs `groups` groups of four block-scaled FP4
+ * tensor-core instructions (256 x 256 x 64 each, the GEMM's own instruction) per CTA pair on operands
+ * that already sit in shared memory, with no loads and no epilogue, times them with CUDA events on
+ * `stream`, synchronises, and writes the rate in TFLOP/s to *tflops (host pointer).  This is the
+ * issue-bound peak of the FP4 tensor pipe on the device at hand: the denominator for the GEMM's
+ * roofline fraction where no vendor-measured FP4 peak exists.  Includes the kernel's launch, so use
+ * groups >= 20000 (about a millisecond). */
+torq_status torq_probe_fp4_peak(int groups, double* tflops, void* stream);
+
 const char* torq_status_string(torq_status s);
 
 /* Synchronises `stream`, then returns and clears the device error word of the current device:

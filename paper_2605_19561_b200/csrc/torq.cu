@@ -13,6 +13,7 @@
 #include "rotate_quantize_pair.cuh"
 #include "rotate_splitk.cuh"
 #include "rotate_structured.cuh"
+#include "fp4_peak_probe.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -487,6 +488,33 @@ torq_status torq_rotated_linear_static(const void* X, const void* R_inter, const
   if (!scratch) return TORQ_ERR_LAUNCH;
   return rotated_linear_impl(X, R_inter, R_intra, Wq, Ws, M, d, N, Y, y_dtype, scratch,
                              (size_t)TORQ_STATIC_WORKSPACE_BYTES, nullptr, nullptr, stream);
+}
+
+torq_status torq_probe_fp4_peak(int groups, double* tflops, void* stream) {
+  if (!tflops) return TORQ_ERR_NULL;
+  if (groups < 1 || groups > (1 << 24)) return TORQ_ERR_SHAPE;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (!opt_in_smem(fp4_peak_probe_kernel, Fp4ProbeCfg::SMEM_BYTES)) return TORQ_ERR_LAUNCH;
+  const int pairs = st->gemm_pairs;
+  cudaEvent_t e0, e1;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return TORQ_ERR_LAUNCH;
+  launch_tc(fp4_peak_probe_kernel, 2, 2 * pairs, Fp4ProbeCfg::THREADS, Fp4ProbeCfg::SMEM_BYTES, s, 64, st->err_word);
+  cudaEventRecord(e0, s);
+  launch_tc(fp4_peak_probe_kernel, 2, 2 * pairs, Fp4ProbeCfg::THREADS, Fp4ProbeCfg::SMEM_BYTES, s, groups,
+            st->err_word);
+  cudaEventRecord(e1, s);
+  g_launches.fetch_add(2, std::memory_order_relaxed);
+  float ms = 0.f;
+  const bool ok = cudaEventSynchronize(e1) == cudaSuccess && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess &&
+                  cudaGetLastError() == cudaSuccess && ms > 0.f;
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (!ok) return TORQ_ERR_LAUNCH;
+  *tflops = (double)pairs * groups * 4.0 * 2.0 * 256.0 * 256.0 * 64.0 / ((double)ms * 1e-3) / 1e12;
+  return TORQ_OK;
 }
 
 torq_status torq_swizzle_scales(const void* linear_scales, int64_t rows, int64_t k, void* out,

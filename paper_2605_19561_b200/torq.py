@@ -56,6 +56,8 @@ def lib() -> ctypes.CDLL:
     L.torq_swizzle_scales.restype = ci
     L.torq_merge_rotations.argtypes = [vp, vp, i64, vp, vp]
     L.torq_merge_rotations.restype = ci
+    L.torq_probe_fp4_peak.argtypes = [ci, ctypes.POINTER(ctypes.c_double), vp]
+    L.torq_probe_fp4_peak.restype = ci
     L.torq_status_string.argtypes = [ci]
     L.torq_status_string.restype = ctypes.c_char_p
     L.torq_last_device_error.argtypes = [vp]
@@ -208,6 +210,13 @@ def torq_rotated_linear_static(X, R_inter, R_intra, Wq, Ws, Y, stream=None):
     _raise(lib().torq_rotated_linear_static(_ptr(X), _ptr(R_inter), _ptr(R_intra), _ptr(Wq), _ptr(Ws), M, d, N,
                                             _ptr(Y), dt, _stream(stream)), "torq_rotated_linear_static")
     return Y
+
+
+def torq_probe_fp4_peak(groups: int = 40000, stream=None) -> float:
+    """Issue-bound rate (TFLOP/s) of the block-scaled FP4 tensor-core instruction on this device."""
+    out = ctypes.c_double(0.0)
+    _raise(lib().torq_probe_fp4_peak(groups, ctypes.byref(out), _stream(stream)), "torq_probe_fp4_peak")
+    return out.value
 
 
 def torq_swizzle_scales(linear, k: int, out=None, stream=None):

@@ -62,4 +62,7 @@ def test_argument_errors_are_status_codes():
     assert L.torq_rotated_linear(one, one, one, one, one, 4, 128, 8, one, 0, None, 0, None, None, None) == 7
     assert L.torq_rotated_linear(one, one, one, one, one, 4, 128, 8, one, 0, one, 16, None, None, None) == 7
     assert L.torq_rotated_linear(one, one, one, one, one, 4, 96, 8, one, 0, one, 1 << 20, None, None, None) == 2
+    assert L.torq_probe_fp4_peak(100, None, None) == 1
+    import ctypes as _c
+    assert L.torq_probe_fp4_peak(0, _c.byref(_c.c_double()), None) == 2
     assert L.torq_status_string(0) == b"ok" and L.torq_status_string(6)

@@ -101,3 +101,11 @@ def test_full_size_sampled_outputs_llama3_qkv_shape():
     ref2 = O.gemm_dequant(ac, asb, wc[cols], wsb[cols])
     got2 = y.cpu().numpy()[:, cols].astype(np.float64)
     assert np.linalg.norm(got2 - ref2) / np.linalg.norm(ref2) <= 1e-5
+
+
+def test_fp4_peak_probe_reports_a_plausible_rate():
+    """The measurement tool behind the GEMM's roofline denominator: finite, positive, and not above
+    what the instruction can do at the maximum clock (about 9.3 PFLOP/s on 148 SMs at 1965 MHz)."""
+    rate = torq.torq_probe_fp4_peak(20000)
+    assert torq.torq_last_device_error() == 0
+    assert 1000.0 < rate < 9500.0, rate
