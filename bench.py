@@ -237,13 +237,17 @@ def main():
             fn(sets[i % n_sets])
         torch.cuda.synchronize()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        hold_gpu(stream)
+        # at most 400 launches per measurement: a kernel shorter than the host's cost of enqueuing it
+        # (about 15 us through ctypes) is only timed correctly while the launches queued during the
+        # hold last
+        k = min(args.steps, 400)
+        hold_gpu(stream, ms=10.0)
         a0.record(stream)
-        for i in range(args.steps):
+        for i in range(k):
             fn(sets[i % n_sets])
         a1.record(stream)
         torch.cuda.synchronize()
-        return a0.elapsed_time(a1) / args.steps * 1e-3
+        return a0.elapsed_time(a1) / k * 1e-3
 
     def gemm_only(b):
         c, sc = codes_scales(b)
