@@ -83,6 +83,54 @@ def test_bf16_output_is_the_rounded_fp32_result():
     assert np.linalg.norm(got - want) / np.linalg.norm(want) <= 1e-3
 
 
+@pytest.mark.parametrize("M,N,K,dt", [(300, 520, 1152, torch.bfloat16), (257, 72, 128, torch.bfloat16),
+                                      (1000, 264, 640, torch.float32), (129, 8, 384, torch.bfloat16),
+                                      (511, 1032, 896, torch.float32), (640, 328, 1408, torch.bfloat16)])
+def test_ragged_shapes_on_the_cta_pair_kernel(M, N, K, dt):
+    """M > 128 runs on CTA pairs with staged TMA stores of Y: ragged M (second row tile of a pair
+    missing or partial), N that ends inside a 256-column tile and inside a 64- or 32-column store
+    box, K with a half last stage (K % 256 == 128)."""
+    ac, asb = _rand_operand(M, K, 31)
+    wc, wsb = _rand_operand(N, K, 32)
+    ref = O.gemm_dequant(ac, asb, wc, wsb)
+    # canary: rows and columns around Y must stay untouched
+    pad = torch.full((M + 2, N + 16), 7.0, dtype=dt, device="cuda")
+    Y = pad[1:M + 1, 8:N + 8]
+    assert not Y.is_contiguous()
+    Yc = torch.empty((M, N), dtype=dt, device="cuda")
+    torq.torq_mxfp4_gemm(dev_u8(O.pack_codes(ac)), dev_u8(O.swizzle_scales(asb, K, fill=0)),
+                         dev_u8(O.pack_codes(wc)), dev_u8(O.swizzle_scales(wsb, K, fill=0)), Y=Yc)
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    got = Yc.float().cpu().numpy().astype(np.float64)
+    want = ref if dt == torch.float32 else O.round_to_bf16(ref)
+    assert np.isfinite(got).all()
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) <= (1e-5 if dt == torch.float32 else 1e-3)
+    if dt == torch.bfloat16:
+        # element-wise: one bf16 ulp of the result, plus the fp32 accumulation error, which scales with
+        # the size of the terms (not of the possibly cancelled sum)
+        ulp = np.ldexp(1.0, np.frexp(np.maximum(np.abs(want), 1e-30))[1] - 8)
+        terms = np.abs(O.dequantize(ac, asb)) @ np.abs(O.dequantize(wc, wsb)).T
+        assert (np.abs(got - want) <= ulp + 1e-6 * terms).all()
+
+
+def test_output_buffer_neighbours_are_not_written():
+    """Y packed between canaries in one allocation: the TMA stores clip at M rows and N columns."""
+    M, N, K = 300, 520, 256
+    ac, asb = _rand_operand(M, K, 41)
+    wc, wsb = _rand_operand(N, K, 42)
+    for dt in (torch.bfloat16, torch.float32):
+        buf = torch.full((M * N + 4096,), 3.0, dtype=dt, device="cuda")
+        Y = buf[2048:2048 + M * N].view(M, N)
+        torq.torq_mxfp4_gemm(dev_u8(O.pack_codes(ac)), dev_u8(O.swizzle_scales(asb, K, fill=0)),
+                             dev_u8(O.pack_codes(wc)), dev_u8(O.swizzle_scales(wsb, K, fill=0)), Y=Y)
+        torch.cuda.synchronize()
+        assert bool((buf[:2048] == 3.0).all()) and bool((buf[2048 + M * N:] == 3.0).all())
+        ref = O.gemm_dequant(ac, asb, wc, wsb)
+        got = Y.float().cpu().numpy().astype(np.float64)
+        assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-2
+
+
 def test_full_size_sampled_outputs_llama3_qkv_shape():
     """Benchmark size (M=2048, K=4096, N=6144, bf16 out): sampled rows/columns against the oracle."""
     M, N, K = 2048, 6144, 4096

@@ -169,3 +169,15 @@ def test_few_token_split_k_path_through_the_fused_call(M, d):
         ref = O.gemm_dequant(g_codes, g_sb, O.unpack_codes(wq), wsb)
         got = y.cpu().numpy().astype(np.float64)
         assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-3
+
+
+@pytest.mark.parametrize("M,d", [(129, 256), (255, 512), (257, 320), (300, 1024), (511, 5120), (640, 96)])
+def test_ragged_shapes_on_the_cta_pair_rotation(M, d):
+    """M > 128 (CTA pairs, last-tile tensor-core epilogue and fp32-FMA epilogue both exercised when a
+    pair works more than one tile), d that ends inside a 256-column tile (320, 96) and M that leaves
+    the pair's second row tile partial or absent."""
+    cfg = I.CONFIGS["tiny"]
+    xb = I.activations(cfg, M=M, d=d)
+    rb, rib, _, _ = I.rotations(cfg, d=d)
+    _rotate_quantize_case(xb, rb, rib)
+    _rotate_quantize_case(xb, rb, None)
