@@ -274,6 +274,11 @@ def main():
             torq.torq_rotate_quantize_structured(b["X"], RB, Ri1, out_codes=c, out_scales=sc)
 
         t_struct = timed_loop(struct_only)
+
+        def struct_layer(b):
+            torq.torq_rotated_linear_structured(b["X"], RB, Ri1, b["Wq"], b["Ws"], Y=b["Y"], workspace=b["ws"])
+
+        t_struct_layer = timed_loop(struct_layer)
     barrier()
     clocks = sampler.stop()
     assert torq.torq_last_device_error() == 0
@@ -379,7 +384,8 @@ def main():
                 "R_intra (the paper's structure, 2d(B+32) flop per token) on the same activations", "bound": "hbm",
                 "ms_per_launch": t_struct * 1e3, "achieved": nbytes / t_struct / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": nbytes / t_struct / 1e9 / pk["hbm_gbs"], "algorithmic_bytes": nbytes,
-                "speedup_over_dense_rotation": t_rot / t_struct})(
+                "speedup_over_dense_rotation": t_rot / t_struct,
+                "whole_layer_ms_per_step": t_struct_layer * 1e3, "whole_layer_tokens_per_s": world * M / t_struct_layer})(
                     2.0 * M * d + 2.0 * (d // 32) ** 2 + 2048.0 + M * d / 2 + M * d / 32),
             "e2e": {"value": world * M / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": Xh.numel() * 2,
                     "d2h_bytes_per_step": Yh.numel() * 2},

@@ -83,6 +83,17 @@ torq_status torq_rotate_quantize_structured(const void* X, const void* R_B, cons
                                             int64_t M, int64_t d, void* out_codes, void* out_scales,
                                             void* stream);
 
+/* Algorithm 3 steps 1-5 with the structured rotation: torq_rotate_quantize_structured into
+ * `workspace` (codes [M, d/2], then 256-byte aligned the tiled scales; >= M*d/2 rounded up to 256
+ * plus torq_scales_bytes(M, d) bytes, 256-byte aligned), then torq_mxfp4_gemm against weights that
+ * were rotated with the same R_B and R_intra offline.  dbg_codes / dbg_scales as in
+ * torq_rotated_linear.  Requires d % 256 == 0 and N % 8 == 0. */
+torq_status torq_rotated_linear_structured(const void* X, const void* R_B, const void* R_intra,
+                                           const void* Wq, const void* Ws, int64_t M, int64_t d,
+                                           int64_t N, void* Y, torq_dtype y_dtype, void* workspace,
+                                           size_t workspace_bytes, void* dbg_codes, void* dbg_scales,
+                                           void* stream);
+
 /* Algorithm 3 step 5 (option B): Y[m,n] = sum_k a^[m,k] w^[n,k], a^/w^ the dequantized MXFP4
  * values (codeword x 2^e), fp32 accumulation on the block-scaled FP4 tensor cores.
  *   Aq [M, K/2] u8, As scales of A (tiled, torq_scales_bytes(M, K))

@@ -453,6 +453,31 @@ torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* 
                              dbg_codes, dbg_scales, stream);
 }
 
+torq_status torq_rotated_linear_structured(const void* X, const void* R_B, const void* R_intra, const void* Wq,
+                                           const void* Ws, int64_t M, int64_t d, int64_t N, void* Y,
+                                           torq_dtype y_dtype, void* workspace, size_t workspace_bytes,
+                                           void* dbg_codes, void* dbg_scales, void* stream) {
+  if (!X || !R_B || !Wq || !Ws || !Y) return TORQ_ERR_NULL;
+  if (M < 1 || d < 256 || d % 256 != 0 || N < 8 || N % 8 != 0) return TORQ_ERR_SHAPE;
+  if (!workspace || workspace_bytes < quantized_bytes(M, d)) return TORQ_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return TORQ_ERR_ALIGN;
+  uint8_t* codes = static_cast<uint8_t*>(workspace);
+  const size_t codes_bytes = (size_t)M * (size_t)(d / 2);
+  uint8_t* scales = codes + (codes_bytes + 255) / 256 * 256;
+  torq_status rc = torq_rotate_quantize_structured(X, R_B, R_intra, M, d, codes, scales, stream);
+  if (rc != TORQ_OK) return rc;
+  rc = torq_mxfp4_gemm(codes, scales, Wq, Ws, M, N, d, Y, y_dtype, stream);
+  if (rc != TORQ_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dbg_codes &&
+      cudaMemcpyAsync(dbg_codes, codes, codes_bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return TORQ_ERR_LAUNCH;
+  if (dbg_scales && cudaMemcpyAsync(dbg_scales, scales, torq_scales_bytes(M, d),
+                                    cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return TORQ_ERR_LAUNCH;
+  return TORQ_OK;
+}
+
 // ---- the layer without any allocation -----------------------------------------------------------
 // Scratch for torq_rotated_linear_static.  In host code this name is only a handle for the
 // runtime's symbol table, not an address a kernel can use: the device address comes from

@@ -38,6 +38,8 @@ def lib() -> ctypes.CDLL:
     L.torq_rotate_quantize.restype = ci
     L.torq_rotate_quantize_structured.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp]
     L.torq_rotate_quantize_structured.restype = ci
+    L.torq_rotated_linear_structured.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, vp, sz, vp, vp, vp]
+    L.torq_rotated_linear_structured.restype = ci
     L.torq_mxfp4_gemm.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, ci, vp]
     L.torq_mxfp4_gemm.restype = ci
     L.torq_rotated_linear.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, vp, sz, vp, vp, vp]
@@ -184,6 +186,26 @@ def torq_rotated_linear(X, R_inter, R_intra, Wq, Ws, out_dtype=torch.bfloat16, Y
     _raise(lib().torq_rotated_linear(_ptr(X), _ptr(R_inter), _ptr(R_intra), _ptr(Wq), _ptr(Ws), M, d, N,
                                      _ptr(Y), dt, _ptr(workspace), workspace.numel(), _ptr(dbg_codes),
                                      _ptr(dbg_scales), _stream(stream)), "torq_rotated_linear")
+    return Y
+
+
+def torq_rotated_linear_structured(X, R_B, R_intra, Wq, Ws, out_dtype=torch.bfloat16, Y=None, workspace=None,
+                                   dbg_codes=None, dbg_scales=None, stream=None):
+    """The whole layer with the rotation in the paper's structure (R_B [d/32,d/32], shared R_intra [32,32])."""
+    M, d = X.shape
+    N = Wq.shape[0]
+    for t, n in ((X, "X"), (R_B, "R_B"), (R_intra, "R_intra")):
+        _check(t, torch.bfloat16, n)
+    for t, n in ((Wq, "Wq"), (Ws, "Ws"), (dbg_codes, "dbg_codes"), (dbg_scales, "dbg_scales")):
+        _check(t, torch.uint8, n)
+    if Y is None:
+        Y = torch.empty((M, N), dtype=out_dtype, device=X.device)
+    if workspace is None:
+        workspace = torch.empty(torq_workspace_bytes(M, d, N), dtype=torch.uint8, device=X.device)
+    dt = TORQ_F32 if Y.dtype == torch.float32 else TORQ_BF16
+    _raise(lib().torq_rotated_linear_structured(_ptr(X), _ptr(R_B), _ptr(R_intra), _ptr(Wq), _ptr(Ws), M, d, N,
+                                                _ptr(Y), dt, _ptr(workspace), workspace.numel(), _ptr(dbg_codes),
+                                                _ptr(dbg_scales), _stream(stream)), "torq_rotated_linear_structured")
     return Y
 
 

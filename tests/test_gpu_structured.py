@@ -97,3 +97,39 @@ def test_argument_errors():
     assert L.torq_rotate_quantize_structured(one, None, None, 4, 256, one, one, None) == 1     # R_B required
     assert L.torq_rotate_quantize_structured(one, one, None, 4, 128, one, one, None) == 2      # d % 256 != 0
     assert L.torq_rotate_quantize_structured(one, one, None, 0, 256, one, one, None) == 2
+
+
+def test_whole_layer_with_the_structured_rotation():
+    """Steps 1-5 in one call.  Weights are rotated by the same operator offline (oracle, dense form
+    kron(R_B^T, I) . blockdiag(R_intra)) and quantized; the GEMM is checked on the codes the GPU
+    produced, and the layer output against the all-oracle result."""
+    g = np.random.default_rng(11)
+    M, nb, N = 200, 8, 136
+    d = nb * 32
+    cfg = I.CONFIGS["tiny"]
+    xb = I.activations(cfg, M=M, d=d)
+    rb = I.to_bf16_bits(I.orthogonal(nb, g))
+    ri = I.to_bf16_bits(I.orthogonal(32, g))
+    dense = I.to_bf16_bits(np.kron(O.decode_bf16(rb).T, np.eye(32)))
+    w = (g.standard_normal(size=(d, N)) * 0.02).astype(np.float32)
+    w_codes, w_sb = O.prepare_weights(dense, np.stack([ri] * nb), w)
+    dev_u8 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.uint8)).cuda()
+    Wq, Ws = dev_u8(O.pack_codes(w_codes)), dev_u8(O.swizzle_scales(w_sb, d, fill=0))
+    dbg_c = torch.empty((M, d // 2), dtype=torch.uint8, device="cuda")
+    dbg_s = torch.empty(torq.torq_scales_bytes(M, d), dtype=torch.uint8, device="cuda")
+    y = torq.torq_rotated_linear_structured(dev_bf16(xb), dev_bf16(rb), dev_bf16(ri), Wq, Ws, out_dtype=torch.float32,
+                                            dbg_codes=dbg_c, dbg_scales=dbg_s)
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    g_codes, g_sb = gpu_quantized_to_numpy(dbg_c, dbg_s, M, d)
+    o_codes, o_sb = O.quantize_mxfp4(O.round_to_f32(O.rotate_structured(xb, rb, ri)))
+    rep = mismatch_report(g_codes, g_sb, o_codes, o_sb)
+    assert rep["non_adjacent"] == 0 and rep["elem_mismatch_frac"] <= 1e-4, rep
+    got = y.cpu().numpy().astype(np.float64)
+    ref = O.gemm_dequant(g_codes, g_sb, w_codes, w_sb)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-3
+    full = O.gemm_dequant(o_codes, o_sb, w_codes, w_sb)
+    assert np.linalg.norm(got - full) / np.linalg.norm(full) <= 2e-2
+    # and the rotated-quantized layer approximates the unrotated full-precision one (identity chain)
+    exact = O.decode_bf16(xb) @ w.astype(np.float64)
+    assert np.linalg.norm(got - exact) / np.linalg.norm(exact) <= 0.25
