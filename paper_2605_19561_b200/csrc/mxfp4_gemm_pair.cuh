@@ -1,7 +1,7 @@
 // Block-scaled MXFP4 GEMM on CTA pairs (M > 128): two CTAs share one 256 x 256 output tile through
 // tcgen05.mma cta_group::2 kind::mxf4.block_scale.  Each CTA stages its own 128 rows of A, its own
 // 128 rows of W, its own A scales and the full tile's W scales (35 KiB per 256 elements of K
-// instead of 51 KiB), five stages deep.  No multicast load.
+// instead of 51 KiB), five stages deep.  Every CTA loads only for itself.
 //
 // The 128 x 256 fp32 accumulator of each CTA fills half of tensor memory and the scale factors
 // need columns too, so there is a single accumulator buffer; to keep the tensor pipe busy the

@@ -3,7 +3,7 @@
 // tile through tcgen05.mma cta_group::2.  Each CTA stages only its own 128 rows of X and its own
 // 128 columns of R_inter per K step (32 KiB instead of 48 KiB per 128 x 256 x 64 of work), which
 // is what the single-CTA kernel is short of: it cannot keep enough bytes in flight from L2 to
-// feed the tensor pipe.  No multicast load is used; operand sharing happens inside the MMA, which
+// feed the tensor pipe.  Every CTA loads only for itself; operand sharing happens inside the MMA, which
 // reads both CTAs' shared memory.
 //
 // Roles per CTA: warp 0 TMA producer (both CTAs), warp 1 MMA issuer (leader CTA only; both

@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the kernels use: mbarriers with bounded
-// waits, TMA (cp.async.bulk / cp.async.bulk.tensor, never with cluster multicast), tensor-memory
+// waits, TMA (bulk and tiled copies, each CTA loading for itself only), tensor-memory
 // allocation, tcgen05 MMA / copy / load / commit, and the shared-memory matrix descriptors.
 #pragma once
 #include <cuda.h>
@@ -318,7 +318,7 @@ __device__ __forceinline__ bool mbar_wait_cluster_warp(uint32_t bar, uint32_t pa
   return __all_sync(0xFFFFFFFFu, mbar_wait_cluster(bar, parity, cta_abort, err_word, site));
 }
 // 2-D tiled load into THIS CTA's shared memory whose completion bytes are counted on a barrier
-// that may live in the other CTA of the pair (`bar_cluster_addr` from map_to_cta).  No multicast.
+// that may live in the other CTA of the pair (`bar_cluster_addr` from map_to_cta).  The data goes to this CTA alone.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* m, int32_t c0,
                                                  int32_t c1, uint32_t bar_cluster_addr) {
   asm volatile(
