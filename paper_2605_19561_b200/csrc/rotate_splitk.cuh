@@ -1,14 +1,14 @@
-// Rotate + quantize for few tokens (M <= 128), where the work is streaming R_inter from HBM once:
-// with one 128 x 256 tile per CTA only d/256 CTAs would pull on the memory system (20 of 148 SMs at
-// d = 5120).  Here the contraction is also split along K: CTA (n tile, k split) multiplies
+// Rotate + quantize for few tokens (fewer output tiles than half the SMs), where the work is
+// streaming R_inter from HBM once: with one 128 x 256 tile per CTA only M/128 x d/256 CTAs would
+// pull on the memory system (20 of 148 SMs at M <= 128, d = 5120).  Here the contraction is also split along K: CTA (n tile, k split) multiplies
 // X[:, k range] by R_inter[k range, 256 columns] on the tensor cores and writes its fp32 partial
 // tile to scratch; a second, small kernel adds the partials of each (token, 32-block) in split
 // order, applies the intra-block rotation, and quantizes (Algorithm 3 steps 2-4; the quantizer
 // needs the complete sum, so it cannot run per split).  Summation order is fixed: the result does
 // not depend on timing.
 //
-// Scratch layout: P[split][128 rows][d] fp32 (rows >= M of a 32-row group that holds a token are
-// written as zeros; 32-row groups without any token are not written and not read).
+// Scratch layout: P[split][rows padded to 128][d] fp32 (rows >= M of a 32-row group that holds a
+// token are written as zeros; 32-row groups without any token are not written and not read).
 #pragma once
 #include <cuda_bf16.h>
 #include "quantize.cuh"
@@ -32,8 +32,9 @@ struct RotSplitCfg {
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
 
-// grid = n_tiles * splits; CTA b works n tile b % n_tiles, k split b / n_tiles.
-// tmP: fp32 [splits * 128, d], box [32 rows x 32 columns], 128-byte swizzle.
+// grid = m_tiles * n_tiles * splits; CTA b works row tile b % m_tiles, n tile (b / m_tiles) % n_tiles,
+// k split b / (m_tiles * n_tiles).  tmP: fp32 [splits * m_tiles * 128, d], box [32 rows x 32 columns],
+// 128-byte swizzle.
 __global__ void __launch_bounds__(192, 1)
 rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
                      const __grid_constant__ CUtensorMap tmP, int M, int d, int splits, int* err_word) {
@@ -53,7 +54,8 @@ rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles = (d + BN - 1) / BN;
-  const int nt = blockIdx.x % n_tiles, ks = blockIdx.x / n_tiles;
+  const int m_tiles = (M + C::BM - 1) / C::BM;
+  const int mt = blockIdx.x % m_tiles, nt = (blockIdx.x / m_tiles) % n_tiles, ks = blockIdx.x / (m_tiles * n_tiles);
   const int k_tiles = (d + C::BK - 1) / C::BK;
   const int kt0 = (int)((long long)k_tiles * ks / splits);
   const int kt1 = (int)((long long)k_tiles * (ks + 1) / splits);
@@ -83,7 +85,7 @@ rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
       const uint32_t st = smem_base + s * C::STAGE_BYTES;
       if (elect_one()) {
         mbar_arrive_expect_tx(full_bar(s), C::STAGE_BYTES);
-        tma_load_2d(st, &tmX, kt * C::BK, 0, full_bar(s));
+        tma_load_2d(st, &tmX, kt * C::BK, mt * C::BM, full_bar(s));
 #pragma unroll
         for (int b = 0; b < BN / 64; ++b)
           tma_load_2d(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR, nt * BN + b * 64, kt * C::BK, full_bar(s));
@@ -118,7 +120,7 @@ rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const int q = warp & 3;
     bool ok = mbar_wait(accf_bar, 0, cta_abort, err_word, SITE_EPI_ACC_FULL);
     ok = __all_sync(0xFFFFFFFFu, ok);
-    if (ok && q * 32 < M) {                              // this 32-row group holds at least one token
+    if (ok && mt * C::BM + q * 32 < M) {                 // this 32-row group holds at least one token
       tc_fence_after_sync();
       const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
       const uint32_t stage_buf = smem_base + out_off + (uint32_t)(warp - 2) * C::OUT_WARP_BYTES;
@@ -142,7 +144,7 @@ rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         __syncwarp();
         const int col = nt * BN + bb * 32;
         if (lane == 0 && col < d) {
-          tma_store_2d(&tmP, col, ks * C::BM + q * 32, stage_buf);
+          tma_store_2d(&tmP, col, (ks * m_tiles + mt) * C::BM + q * 32, stage_buf);
           bulk_commit_group();
         }
       }
@@ -162,87 +164,94 @@ rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   }
 }
 
-// Second phase: one CTA of four warps per 32-block b, warp w = rows 32w .. 32w+31, lane = row.
-// The CTA first stages R_intra[b] in shared memory as fp32 (one coalesced 2 KiB read); then each
-// thread adds its row's partial blocks in split order, applies the intra-block rotation in fp32
-// FMAs in index order (R read from shared memory at the same address by every lane) and quantizes
-// (Eq. 1).  Rows M .. 127 and K-blocks d/32 .. (padded to 4) only get their padding scale byte (0).
-__global__ void __launch_bounds__(128)
+// Second phase: one CTA of 8 warps per (32-block b, group of 32 rows).
+//  1. All warps add the partials P[s][row][32 b + j] in split order into a shared-memory tile
+//     (a warp reads one row's 128 bytes per split; all loads of the CTA are in flight together, so
+//     the phase costs one memory latency).
+//  2. Four threads per row, thread p of a row owning columns 8p .. 8p+7: the intra-block rotation
+//     z_j = sum_i y_i R[i][j] in fp32 FMAs in index order (y and R_intra[b] from shared memory),
+//     block maximum over the four threads by two shuffles, Eq. 1, and one 4-byte code store per
+//     thread (the four threads of a row write its 16 bytes contiguously).
+// Rows M .. (group end) and K-blocks d/32 .. (padded to 4) only get their padding scale byte (0).
+__global__ void __launch_bounds__(256)
 splitk_reduce_quantize_kernel(const float* __restrict__ P, const __nv_bfloat16* __restrict__ R_intra,
                               int M, int d, int splits, uint8_t* __restrict__ codes,
                               uint8_t* __restrict__ scales) {
+  __shared__ float y_s[32 * 33];                         // row stride 33: conflict-free by row and by column
   __shared__ __align__(16) float r_s[1024];
   griddep_launch_dependents();
   griddep_wait();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int nb = d / 32;
   const int kb4 = (nb + 3) / 4;
-  const int b = blockIdx.x, row = threadIdx.x;
-  if (b >= nb) {                                         // padding K-block
-    scales[scale_offset(row, b, kb4)] = 0;
+  const int nbp = kb4 * 4;
+  const int b = blockIdx.x % nbp, rg = blockIdx.x / nbp;  // row group: rows 32 rg .. 32 rg + 31
+  const int m_tiles = (M + 127) / 128;
+  const int row0 = rg * 32;
+  const int rows = max(0, min(32, M - row0));            // real rows of this group
+  if (b >= nb || rows == 0) {                            // padding only: zero scale bytes
+    if (threadIdx.x < 32) scales[scale_offset(row0 + threadIdx.x, b, kb4)] = 0;
     return;
   }
-  if (R_intra != nullptr) {
+  const size_t split_stride = (size_t)m_tiles * 128 * d;
+  // ---- 1. partial sums -> shared memory
+#pragma unroll 4
+  for (int r = warp; r < rows; r += nwarps) {
+    const float* p = P + (size_t)(row0 + r) * d + b * 32 + lane;
+    float part[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) part[s] = s < splits ? __ldg(p + s * split_stride) : 0.f;
+    float y = 0.f;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) if (s < splits) y += part[s];
+    y_s[r * 33 + lane] = y;
+  }
+  if (R_intra != nullptr && threadIdx.x < 128) {
     float v[8];
     load8(R_intra + (size_t)b * 1024 + threadIdx.x * 8, v);
     *reinterpret_cast<float4*>(r_s + threadIdx.x * 8) = make_float4(v[0], v[1], v[2], v[3]);
     *reinterpret_cast<float4*>(r_s + threadIdx.x * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
   }
   __syncthreads();
-  if (row >= M) {
-    scales[scale_offset(row, b, kb4)] = 0;
-    return;
-  }
-  float y[32];
+  // ---- 2. four threads per row
+  if (threadIdx.x >= 128) return;
+  const int r = threadIdx.x >> 2, p = threadIdx.x & 3;
+  const int row = row0 + r;
+  float z[8];
+  if (r < rows) {
+    if (R_intra != nullptr) {
 #pragma unroll
-  for (int j = 0; j < 32; ++j) y[j] = 0.f;
-  const float4* p0 = reinterpret_cast<const float4*>(P + ((size_t)row * d + b * 32));
-  const size_t split_stride = (size_t)128 * d / 4;       // in float4
-  int s = 0;
-  for (; s + 2 <= splits; s += 2) {                      // two splits' loads in flight, added in order
-    float4 u[8], w[8];
+      for (int j = 0; j < 8; ++j) z[j] = 0.f;
 #pragma unroll
-    for (int g = 0; g < 8; ++g) { u[g] = __ldg(p0 + s * split_stride + g); w[g] = __ldg(p0 + (s + 1) * split_stride + g); }
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      y[4 * g] += u[g].x; y[4 * g + 1] += u[g].y; y[4 * g + 2] += u[g].z; y[4 * g + 3] += u[g].w;
-    }
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      y[4 * g] += w[g].x; y[4 * g + 1] += w[g].y; y[4 * g + 2] += w[g].z; y[4 * g + 3] += w[g].w;
-    }
-  }
-  if (s < splits) {
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      const float4 u = __ldg(p0 + s * split_stride + g);
-      y[4 * g] += u.x; y[4 * g + 1] += u.y; y[4 * g + 2] += u.z; y[4 * g + 3] += u.w;
-    }
-  }
-  float z[32];
-  if (R_intra != nullptr) {
-#pragma unroll
-    for (int j = 0; j < 32; ++j) z[j] = 0.f;
-    const float4* r = reinterpret_cast<const float4*>(r_s);
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-#pragma unroll
-      for (int g = 0; g < 8; ++g) {
-        const float4 rv = r[i * 8 + g];
-        z[4 * g + 0] = fmaf(y[i], rv.x, z[4 * g + 0]);
-        z[4 * g + 1] = fmaf(y[i], rv.y, z[4 * g + 1]);
-        z[4 * g + 2] = fmaf(y[i], rv.z, z[4 * g + 2]);
-        z[4 * g + 3] = fmaf(y[i], rv.w, z[4 * g + 3]);
+      for (int i = 0; i < 32; ++i) {
+        const float yi = y_s[r * 33 + i];
+        const float4 ra = *reinterpret_cast<const float4*>(r_s + i * 32 + 8 * p);
+        const float4 rb = *reinterpret_cast<const float4*>(r_s + i * 32 + 8 * p + 4);
+        z[0] = fmaf(yi, ra.x, z[0]); z[1] = fmaf(yi, ra.y, z[1]); z[2] = fmaf(yi, ra.z, z[2]); z[3] = fmaf(yi, ra.w, z[3]);
+        z[4] = fmaf(yi, rb.x, z[4]); z[5] = fmaf(yi, rb.y, z[5]); z[6] = fmaf(yi, rb.z, z[6]); z[7] = fmaf(yi, rb.w, z[7]);
       }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) z[j] = y_s[r * 33 + 8 * p + j];
     }
   } else {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) z[j] = y[j];
+    for (int j = 0; j < 8; ++j) z[j] = 0.f;
   }
-  uint4 c;
+  float amax = 0.f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fabsf(z[j]));
+  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
   uint32_t sbyte;
-  quantize_block32(z, c, sbyte);
-  *reinterpret_cast<uint4*>(codes + (size_t)row * (d / 2) + b * 16) = c;
-  scales[scale_offset(row, b, kb4)] = (uint8_t)sbyte;
+  float inv;
+  block_scale(amax, sbyte, inv);
+  if (r < rows) {
+    const uint32_t w = pack8_e2m1(z[0] * inv, z[1] * inv, z[2] * inv, z[3] * inv, z[4] * inv, z[5] * inv,
+                                  z[6] * inv, z[7] * inv);
+    *reinterpret_cast<uint32_t*>(codes + (size_t)row * (d / 2) + b * 16 + 4 * p) = w;
+  }
+  if (p == 0) scales[scale_offset(row, b, kb4)] = r < rows ? (uint8_t)sbyte : (uint8_t)0;
 }
 
 }  // namespace torq

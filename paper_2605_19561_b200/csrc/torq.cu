@@ -173,9 +173,11 @@ static void launch_tc(void (*kernel)(KArgs...), int cluster, int grid, int threa
 // K splits of the few-token rotation: as many as fill the SMs, each at least two 64-element steps.
 // `sm_count` <= 0 gives the bound used for sizing workspaces (any device up to 160 SMs).
 static int rotation_splits(int64_t M, int64_t d, int sm_count) {
-  if (M > 128) return 1;
-  const int n_tiles = (int)((d + 255) / 256), k_tiles = (int)((d + 63) / 64);
-  int s = (sm_count > 0 ? sm_count : 160) / n_tiles;
+  const int64_t tiles = ((M + 127) / 128) * ((d + 255) / 256);
+  const int sms = sm_count > 0 ? sm_count : 160;
+  if (2 * tiles > sms) return 1;
+  const int k_tiles = (int)((d + 63) / 64);
+  int s = (int)(sms / tiles);
   if (s > RotSplitCfg::MAX_SPLITS) s = RotSplitCfg::MAX_SPLITS;
   if (s > k_tiles / 2) s = k_tiles / 2;
   return s < 2 ? 1 : s;
@@ -183,8 +185,8 @@ static int rotation_splits(int64_t M, int64_t d, int sm_count) {
 static size_t quantized_bytes(int64_t M, int64_t d) {    // codes, then 256-byte aligned the scales
   return ((size_t)M * (size_t)(d / 2) + 255) / 256 * 256 + torq_scales_bytes(M, d);
 }
-static size_t splitk_scratch_bytes(int64_t d, int splits) {
-  return splits < 2 ? 0 : (size_t)splits * 128 * (size_t)d * sizeof(float);
+static size_t splitk_scratch_bytes(int64_t M, int64_t d, int splits) {
+  return splits < 2 ? 0 : (size_t)splits * (size_t)((M + 127) / 128 * 128) * (size_t)d * sizeof(float);
 }
 
 static torq_status quantize_impl(DeviceState* st, const void* Z, torq_dtype dt, int64_t M, int64_t d,
@@ -220,7 +222,7 @@ size_t torq_scale_offset(int64_t row, int64_t kblock, int64_t k) {
 size_t torq_workspace_bytes(int64_t M, int64_t d, int64_t N) {
   (void)N;
   if (M <= 0 || d <= 0) return 0;
-  return quantized_bytes(M, d) + splitk_scratch_bytes(d, rotation_splits(M, d, 0));
+  return quantized_bytes(M, d) + splitk_scratch_bytes(M, d, rotation_splits(M, d, 0));
 }
 
 const char* torq_status_string(torq_status s) {
@@ -292,17 +294,19 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
       !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
     return TORQ_ERR_LAUNCH;
   const int splits = rotation_splits(M, d, st->sm_count);
-  if (splits >= 2 && scratch && scratch_bytes >= splitk_scratch_bytes(d, splits) &&
+  if (splits >= 2 && scratch && scratch_bytes >= splitk_scratch_bytes(M, d, splits) &&
       (reinterpret_cast<uintptr_t>(scratch) & 15u) == 0) {
     // Few tokens: split K over the SMs, partial tiles to scratch, then reduce + intra + quantize.
     CUtensorMap tmP;
-    if (!encode_2d(&tmP, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, scratch, (uint64_t)splits * 128, (uint64_t)d, 32, 32))
+    const int m_tiles = (int)((M + 127) / 128);
+    if (!encode_2d(&tmP, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, scratch, (uint64_t)splits * m_tiles * 128, (uint64_t)d,
+                   32, 32))
       return TORQ_ERR_LAUNCH;
     const int n_tiles = (int)((d + 255) / 256);
-    launch_tc(rotate_splitk_kernel, 1, n_tiles * splits, RotSplitCfg::THREADS, RotSplitCfg::SMEM_BYTES, s, tmX, tmR,
+    launch_tc(rotate_splitk_kernel, 1, m_tiles * n_tiles * splits, RotSplitCfg::THREADS, RotSplitCfg::SMEM_BYTES, s, tmX, tmR,
               tmP, (int)M, (int)d, splits, st->err_word);
     if (launch_status() != TORQ_OK) return TORQ_ERR_LAUNCH;
-    launch_tc(splitk_reduce_quantize_kernel, 1, (int)(((d / 32 + 3) / 4) * 4), 128, 0, s, static_cast<const float*>(scratch),
+    launch_tc(splitk_reduce_quantize_kernel, 1, (int)(((d / 32 + 3) / 4) * 4) * m_tiles * 4, 256, 0, s, static_cast<const float*>(scratch),
               static_cast<const __nv_bfloat16*>(R_intra), (int)M, (int)d, splits, codes, scales);
     return launch_status();
   }

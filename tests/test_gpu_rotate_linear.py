@@ -135,9 +135,11 @@ def test_llama3_qkv_shape_sampled_rows():
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-3
 
 
-@pytest.mark.parametrize("M,d", [(1, 256), (33, 256), (100, 512), (128, 1024), (64, 2048), (17, 4096)])
+@pytest.mark.parametrize("M,d", [(1, 256), (33, 256), (100, 512), (128, 1024), (64, 2048), (17, 4096),
+                                 (200, 512), (384, 1024), (257, 256)])
 def test_few_token_split_k_path_through_the_fused_call(M, d):
-    """M <= 128 through torq_rotated_linear: the rotation runs as split-K partial tiles plus the
+    """Few output tiles (fewer than half the SMs) through torq_rotated_linear, one or several row
+    tiles: the rotation runs as split-K partial tiles plus the
     reduce/intra/quantize kernel (the workspace carries the partials).  Same bounds as the
     single-pass path, and the codes must also agree with the single-pass kernel to the same
     bounds (only the fp32 summation order differs)."""
