@@ -75,13 +75,35 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  // Set-up above touched no global memory; from here on the previous kernel's results are needed.
+  // Set-up above touched no global memory.  The weights and their scales are constants of the
+  // layer, never the output of the kernel that runs just before this one: the first stages' W
+  // loads go out right away; everything else waits until that kernel has completed.
   griddep_launch_dependents();
+  const int pre = (int)blockIdx.x < total_tiles ? (k_tiles < C::STAGES ? k_tiles : C::STAGES) : 0;
+  if (warp == 0) {
+    if (elect_one()) {
+      tma_prefetch_desc(&tmA);
+      tma_prefetch_desc(&tmB);
+      const int mt = blockIdx.x % m_tiles, nt = blockIdx.x / m_tiles;
+      const int rt0 = nt * (BN / 128);
+      const int n_sfb_tiles = min(BN / 128, n_rowtiles - rt0);
+      (void)mt;
+      for (int kt = 0; kt < pre; ++kt) {
+        const uint32_t sf_bytes = 512u * min(2, kb4 - 2 * kt);
+        const uint32_t st = smem_base + kt * C::STAGE_BYTES;
+        mbar_arrive_expect_tx(full_bar(kt), C::A_BYTES + C::B_BYTES + sf_bytes * (1 + n_sfb_tiles));
+        tma_load_2d(st + C::A_BYTES, &tmB, kt * 128, nt * BN, full_bar(kt));
+        for (int t = 0; t < n_sfb_tiles; ++t)
+          bulk_load_1d(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * 1024,
+                       Ws + ((size_t)(rt0 + t) * kb4 + 2 * kt) * 512, sf_bytes, full_bar(kt));
+      }
+    }
+    __syncwarp();
+  }
   griddep_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (elect_one()) { tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB); }
     uint32_t it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
@@ -96,14 +118,17 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const uint32_t sf_bytes = 512u * nchunk;
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
         if (elect_one()) {
-          mbar_arrive_expect_tx(full_bar(s), C::A_BYTES + C::B_BYTES + sf_bytes * (1 + n_sfb_tiles));
+          const bool w_issued = it < (uint32_t)pre;      // W side of this stage went out before the wait above
+          if (!w_issued) mbar_arrive_expect_tx(full_bar(s), C::A_BYTES + C::B_BYTES + sf_bytes * (1 + n_sfb_tiles));
           tma_load_2d(st, &tmA, kt * 128, mt * C::BM, full_bar(s));
-          tma_load_2d(st + C::A_BYTES, &tmB, kt * 128, nt * BN, full_bar(s));
           bulk_load_1d(st + C::A_BYTES + C::B_BYTES, As + ((size_t)mt * kb4 + 2 * kt) * 512, sf_bytes,
                        full_bar(s));
-          for (int t = 0; t < n_sfb_tiles; ++t)
-            bulk_load_1d(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * 1024,
-                         Ws + ((size_t)(rt0 + t) * kb4 + 2 * kt) * 512, sf_bytes, full_bar(s));
+          if (!w_issued) {
+            tma_load_2d(st + C::A_BYTES, &tmB, kt * 128, nt * BN, full_bar(s));
+            for (int t = 0; t < n_sfb_tiles; ++t)
+              bulk_load_1d(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * 1024,
+                           Ws + ((size_t)(rt0 + t) * kb4 + 2 * kt) * 512, sf_bytes, full_bar(s));
+          }
         }
         __syncwarp();
       }

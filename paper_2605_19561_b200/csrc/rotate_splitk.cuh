@@ -71,12 +71,28 @@ rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // R_inter is a constant of the layer, never the output of the kernel that runs just before this
+  // one: its loads for the first stages go out right away; everything else waits for that kernel.
   griddep_launch_dependents();
+  const int pre = (kt1 - kt0) < C::STAGES ? (kt1 - kt0) : C::STAGES;
+  if (warp == 0) {
+    if (elect_one()) {
+      tma_prefetch_desc(&tmX);
+      tma_prefetch_desc(&tmR);
+      for (int it = 0; it < pre; ++it) {
+        const uint32_t st = smem_base + it * C::STAGE_BYTES;
+        mbar_arrive_expect_tx(full_bar(it), C::STAGE_BYTES);
+#pragma unroll
+        for (int b = 0; b < BN / 64; ++b)
+          tma_load_2d(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR, nt * BN + b * 64, (kt0 + it) * C::BK, full_bar(it));
+      }
+    }
+    __syncwarp();
+  }
   griddep_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (elect_one()) { tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmR); }
     bool ok = true;
     for (int kt = kt0, it = 0; kt < kt1 && ok; ++kt, ++it) {
       const int s = it % C::STAGES;
@@ -84,11 +100,14 @@ rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                           SITE_PRODUCER_EMPTY)) { ok = false; break; }
       const uint32_t st = smem_base + s * C::STAGE_BYTES;
       if (elect_one()) {
-        mbar_arrive_expect_tx(full_bar(s), C::STAGE_BYTES);
+        const bool r_issued = it < pre;                  // R side of this stage went out before the wait above
+        if (!r_issued) mbar_arrive_expect_tx(full_bar(s), C::STAGE_BYTES);
         tma_load_2d(st, &tmX, kt * C::BK, mt * C::BM, full_bar(s));
+        if (!r_issued) {
 #pragma unroll
-        for (int b = 0; b < BN / 64; ++b)
-          tma_load_2d(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR, nt * BN + b * 64, kt * C::BK, full_bar(s));
+          for (int b = 0; b < BN / 64; ++b)
+            tma_load_2d(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR, nt * BN + b * 64, kt * C::BK, full_bar(s));
+        }
       }
       __syncwarp();
     }
