@@ -258,9 +258,11 @@ def main():
         torq.torq_rotate_quantize(b["X"], b["R"], b["Ri"], out_codes=c, out_scales=sc)
 
     t_gemm = timed_loop(gemm_only)
-    # few tokens: the rotation of the fused call is the split-K pair of kernels, which only runs with
-    # the workspace of the fused call; its time is the step minus the GEMM
-    t_rot = timed_loop(rot_only) if M > 128 else max(ms_total / args.steps * 1e-3 - t_gemm, 1e-9)
+    # few output tiles: the rotation of the fused call is the split-K pair of kernels, which only runs
+    # with the workspace of the fused call; its time is the step minus the GEMM
+    sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    split_k = 2 * ((M + 127) // 128) * ((d + 255) // 256) <= sm_count     # the library's own rule
+    t_rot = max(ms_total / args.steps * 1e-3 - t_gemm, 1e-9) if split_k else timed_loop(rot_only)
     # the same activations through the rotation in the paper's own structure (one B x B matrix
     # across blocks, one shared intra-block matrix): reported beside the dense-R_inter path
     t_struct = None
@@ -361,7 +363,8 @@ def main():
                     "ms_per_launch": t * 1e3, "algorithmic_flop": flop, "algorithmic_bytes": nbytes}
 
         pairs = M > 128
-        r_rot = roof("rotate_quantize_pair_kernel" if pairs else "rotate_quantize_kernel", t_rot, rot_flop, rot_bytes,
+        r_rot = roof("rotate_splitk_kernel + splitk_reduce_quantize_kernel" if split_k else
+                     ("rotate_quantize_pair_kernel" if pairs else "rotate_quantize_kernel"), t_rot, rot_flop, rot_bytes,
                      bf16_peak, peak_name)
         r_gemm = roof("mxfp4_gemm_pair_kernel" if pairs else "mxfp4_gemm_kernel", t_gemm, gemm_flop, gemm_bytes,
                       fp4_peak, "self-measured: torq_probe_fp4_peak (FP4 block-scaled MMA issue loop, no loads)")
