@@ -127,19 +127,37 @@ def time_oracle(cfg, rows: int, steps: int, warmup: int):
     return float(np.mean(times)), cores
 
 
+REFERENCE_BUDGET_S = 150.0     # wall-clock bound of the whole reference run
+
+
 def run_reference(args):
+    """The oracle, as it stands, timed on the host cores.  One step = one call of the oracle's
+    rotated_linear on the first `rows` rows of the workload (every stage is independent per row).
+    A call costs about 0.75 s of set-up (decoding R_inter and dequantizing W to float64) plus about
+    2.3 ms per row, so the sample per step and, for very large K, the number of steps that fit the
+    budget are bounded: the line says what was run."""
     from paper_2605_19561_b200 import inputs as I
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     cfg = I.CONFIGS[WORKLOAD]
-    rows = 512
-    t, cores = time_oracle(cfg, rows, max(1, args.steps), min(args.warmup, 1))
+    steps_req, warmup = max(1, args.steps), min(max(args.warmup, 0), 1)
+    per_call_fixed, per_row = 0.9, 0.003
+    calls = steps_req + warmup
+    rows = int((REFERENCE_BUDGET_S / calls - per_call_fixed) / per_row)
+    steps = steps_req
+    if rows >= 64:
+        rows = min(512, rows)
+    else:                                                  # K steps of a meaningful sample do not fit: fewer steps
+        rows = 128
+        steps = max(1, int(REFERENCE_BUDGET_S / (per_call_fixed + rows * per_row)) - warmup)
+    t, cores = time_oracle(cfg, rows, steps, warmup)
     v = rows / t
-    sample = f"first {rows} of {cfg.M} rows per step, all {cfg.d} features and {cfg.N} outputs"
+    sample = (f"first {rows} of {cfg.M} rows per step, all {cfg.d} features and {cfg.N} outputs; {steps} timed steps"
+              + ("" if steps == steps_req else f" (of {steps_req} requested: bounded to {REFERENCE_BUDGET_S:.0f} s)"))
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+        "steps": steps, "warmup": warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": WORKLOAD, "M": cfg.M, "d": cfg.d, "N": cfg.N, "sample": sample},
         "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
@@ -150,13 +168,15 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=None, help="default: 2000 (the CUDA path), 20 (--impl reference)")
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default=WORKLOAD, help="one of inputs.CONFIGS (default: the LLaMA3-8B QKV shape)")
     ap.add_argument("--M", type=int, default=None, help="override the number of tokens (token sweep)")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 20 if args.impl == "reference" else 2000
     if args.impl == "reference":
         return run_reference(args)
 
