@@ -93,7 +93,9 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     if (elect_one()) {
       tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
       tma_prefetch_desc(&tmSFA); tma_prefetch_desc(&tmSFB);
-      const int nt = pair / mp_tiles;
+      int mp0, nt;
+      pair_tile_coords(pair, mp_tiles, n_tiles, mp0, nt);
+      (void)mp0;
       for (int kt = 0; kt < pre; ++kt) {
         const uint32_t st = smem_base + kt * C::STAGE_BYTES;
         const uint32_t leader_full = map_to_cta(full_bar(kt), 0);
@@ -113,7 +115,9 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     uint32_t it = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
-      const int mt = 2 * (tile % mp_tiles) + (int)rank, nt = tile / mp_tiles;
+      int mp, nt;
+      pair_tile_coords(tile, mp_tiles, n_tiles, mp, nt);
+      const int mt = 2 * mp + (int)rank;
       for (int kt = 0; kt < k_tiles; ++kt, ++it) {
         const int s = it % C::STAGES;
         if (!mbar_wait_cluster_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
@@ -195,7 +199,9 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles && ok; tile += npairs, ++tcount) {
-      const int mt = 2 * (tile % mp_tiles) + (int)rank, nt = tile / mp_tiles;
+      int mp, nt;
+      pair_tile_coords(tile, mp_tiles, n_tiles, mp, nt);
+      const int mt = 2 * mp + (int)rank;
       ok = mbar_wait_cluster(accf_bar, tcount & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;

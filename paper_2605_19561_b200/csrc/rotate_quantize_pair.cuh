@@ -89,7 +89,9 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
     if (elect_one()) {
       tma_prefetch_desc(&tmX);
       tma_prefetch_desc(&tmR);
-      const int nt = pair / mp_tiles;
+      int mp0, nt;
+      pair_tile_coords(pair, mp_tiles, n_tiles, mp0, nt);
+      (void)mp0;
       for (int kt = 0; kt < pre; ++kt) {
         const uint32_t st = smem_base + kt * C::STAGE_BYTES;
         const uint32_t leader_full = map_to_cta(full_bar(kt), 0);
@@ -109,7 +111,9 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
     uint32_t it = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
-      const int mt = 2 * (tile % mp_tiles) + (int)rank, nt = tile / mp_tiles;
+      int mp, nt;
+      pair_tile_coords(tile, mp_tiles, n_tiles, mp, nt);
+      const int mt = 2 * mp + (int)rank;
       for (int kt = 0; kt < k_tiles; ++kt, ++it) {
         const int s = it % C::STAGES;
         if (!mbar_wait_cluster_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
@@ -182,7 +186,9 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles; tile += npairs, ++tcount) {
-      const int mt = 2 * (tile % mp_tiles) + (int)rank, nt = tile / mp_tiles;
+      int mp, nt;
+      pair_tile_coords(tile, mp_tiles, n_tiles, mp, nt);
+      const int mt = 2 * mp + (int)rank;
       const int a = tcount % C::NACC;
       const int b0 = nt * (BN / 32);
       const bool last = tile + npairs >= total_tiles;

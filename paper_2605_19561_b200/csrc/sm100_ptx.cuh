@@ -372,6 +372,20 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t cta_mask) 
       ::"r"(bar), "h"(cta_mask) : "memory");
 }
 
+// Tile order of the persistent CTA-pair kernels.  Row tiles are taken in groups of eight; inside a
+// group the row tile is the fast index.  The ~74 tiles in flight at any time then cover about
+// 8 row tiles x 9 column tiles, whatever M is, so both operands of a wave stay in L2 (with the row
+// tile as the fast index over ALL of M, a wave at M = 16384 touched 64 row tiles and one or two
+// column tiles, and the row operand was re-read from HBM for every column tile).
+__device__ __forceinline__ void pair_tile_coords(int tile, int mp_tiles, int n_tiles, int& mp, int& nt) {
+  constexpr int G = 8;
+  const int per_group = G * n_tiles;
+  const int g = tile / per_group, r = tile - g * per_group;
+  const int rows_in_group = min(G, mp_tiles - g * G);
+  mp = g * G + r % rows_in_group;
+  nt = r / rows_in_group;
+}
+
 // Instruction descriptors (32-bit).  Common fields: [17,23) N>>3, [24,29) M>>4, bit 15 / 16 =
 // A / B stored MN-major.
 // kind::f16 : [4,6) D format (1 = f32), [7,10) A format (1 = bf16), [10,13) B format.
