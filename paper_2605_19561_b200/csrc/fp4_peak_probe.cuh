@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(128, 1) fp4_peak_probe_kernel(int groups, int*
   if (warp == 1) { tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512); tmem_relinquish_pair(); }
   tc_fence_before_sync();
   __syncthreads();
-  cluster_sync_all();
+  cluster_sync_after_init();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 

@@ -80,7 +80,7 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   if (warp == 1) { tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS); tmem_relinquish_pair(); }
   tc_fence_before_sync();
   __syncthreads();
-  cluster_sync_all();
+  cluster_sync_after_init();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   // Set-up above touched no global memory.  The weights and their scales are constants of the

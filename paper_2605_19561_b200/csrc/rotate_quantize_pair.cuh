@@ -76,7 +76,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
   if (warp == 1) { tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS); tmem_relinquish_pair(); }
   tc_fence_before_sync();
   __syncthreads();
-  cluster_sync_all();                                  // both CTAs' barriers exist before any remote arrive
+  cluster_sync_after_init();                                  // both CTAs' barriers exist before any remote arrive
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   // Set-up above touched no global memory; from here on the previous kernel's results are needed.
