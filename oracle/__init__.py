@@ -4,3 +4,4 @@ Nothing in the product package imports this; only the tests, the smoke check and
 the benchmark's cpu_baseline / reference legs do.
 """
 from .torq_oracle import *  # noqa: F401,F403
+from .nvfp4_oracle import *  # noqa: F401,F403,E402
