@@ -175,6 +175,55 @@ torq_status torq_swizzle_scales(const void* linear_scales, int64_t rows, int64_t
 torq_status torq_merge_rotations(const void* R_inter, const void* R_intra, int64_t d,
                                  void* R_merged_f32, void* stream);
 
+/* ---- NVFP4 variant (the paper's format study, Section 6 "Generalizability to Other Formats") -----
+ * The same layer with NVFP4 operands: e2m1 codes as above, blocks of 16 along K, one FP8 E4M3
+ * scale byte per (row, block) and one float32 scale per tensor; x^ = codeword * e4m3(byte) *
+ * tensor_scale.  The paper names the format and reports accuracies only; the arithmetic below is
+ * the library's definition (each step one IEEE float32 operation, round to nearest even):
+ *   c = 1 / (6 tensor_scale);  byte = E4M3(amax_block * c), saturating at 448;
+ *   r = 1 / (e4m3(byte) * tensor_scale), or 0 when byte == 0;  code = e2m1(z * r), saturating at
+ *   6, sign of z kept.
+ * The tensor scale is an input (calibrated beforehand; amax(tensor) / (6 * 448) uses the whole
+ * E4M3 range) and must be positive and finite.  Scale bytes use the tiled layout of
+ * torq_scale_offset with 16-element blocks: a buffer has torq_nvfp4_scales_bytes(rows, k) bytes,
+ * the byte of (row, block c) sits at torq_scale_offset(row, c, 2 * k); padding bytes are 0x00
+ * (E4M3 zero).  The intra-block rotation acts inside a quantization block, so it is [d/16, 16, 16]
+ * here; the rotation kernels take it in 32-wide block-diagonal form, made once by
+ * torq_expand_intra16. */
+size_t torq_nvfp4_scales_bytes(int64_t rows, int64_t k);
+size_t torq_nvfp4_workspace_bytes(int64_t M, int64_t d, int64_t N);
+
+/* R_intra16 [d/16, 16, 16] bf16 -> R_intra32 [d/32, 32, 32] bf16: blocks 2b and 2b+1 on the diagonal of
+ * block b, zeros elsewhere.  d % 32 == 0. */
+torq_status torq_expand_intra16(const void* R_intra16, int64_t d, void* R_intra32, void* stream);
+
+/* Quantize Z [M, d] (fp32 or bf16) to NVFP4; d % 16 == 0.  Bit-exact by the definition above. */
+torq_status torq_quantize_nvfp4(const void* Z, torq_dtype z_dtype, int64_t M, int64_t d,
+                                float tensor_scale, void* out_codes, void* out_scales, void* stream);
+
+/* Algorithm 3 steps 1-4 with the NVFP4 quantizer.  X [M, d] bf16; R_inter [d, d] bf16 (required);
+ * R_intra32 [d/32, 32, 32] bf16 or NULL = identity; d % 32 == 0.  Outputs as torq_quantize_nvfp4. */
+torq_status torq_rotate_quantize_nvfp4(const void* X, const void* R_inter, const void* R_intra32,
+                                       int64_t M, int64_t d, float tensor_scale, void* out_codes,
+                                       void* out_scales, void* stream);
+
+/* Algorithm 3 step 5 on NVFP4 operands: Y[m,n] = a_tensor_scale * w_tensor_scale *
+ * sum_k (code * e4m3 scale)_a[m,k] (code * e4m3 scale)_w[n,k], fp32 accumulation on the tensor
+ * cores (kind::mxf4nvf4, 16-element blocks).  Shapes and layouts as torq_mxfp4_gemm with
+ * 16-element blocks: K % 128 == 0, N % 8 == 0. */
+torq_status torq_nvfp4_gemm(const void* Aq, const void* As, float a_tensor_scale, const void* Wq,
+                            const void* Ws, float w_tensor_scale, int64_t M, int64_t N, int64_t K,
+                            void* Y, torq_dtype y_dtype, void* stream);
+
+/* Steps 1-5 in NVFP4: torq_rotate_quantize_nvfp4 into `workspace` (at least
+ * torq_nvfp4_workspace_bytes(M, d, N) bytes, 256-byte aligned), then torq_nvfp4_gemm.
+ * d % 128 == 0, N % 8 == 0. */
+torq_status torq_rotated_linear_nvfp4(const void* X, const void* R_inter, const void* R_intra32,
+                                      float x_tensor_scale, const void* Wq, const void* Ws,
+                                      float w_tensor_scale, int64_t M, int64_t d, int64_t N, void* Y,
+                                      torq_dtype y_dtype, void* workspace, size_t workspace_bytes,
+                                      void* dbg_codes, void* dbg_scales, void* stream);
+
 /* Measurement tool (no counterpart in the paper): runs `groups` groups of four block-scaled FP4
  * tensor-core instructions (256 x 256 x 64 each, the GEMM's own instruction) per CTA pair on operands
  * that already sit in shared memory, with no loads and no epilogue, times them with CUDA events on

@@ -9,39 +9,46 @@
 //   warps 2..5  epilogue      : tensor memory -> registers -> Y (fp32 or bf16), 32 rows per warp
 // Tile = 128 x BN x 256 (one stage = 128 bytes of K per row = one swizzle atom).  NACC
 // accumulator buffers in tensor memory let the epilogue of one tile overlap the next mainloop.
+//
+// The same kernel serves the NVFP4 variant (FMT_NVFP4: kind::mxf4nvf4, one E4M3 scale per 16
+// elements of K, the product of the two tensor scales applied in the epilogue).  Scale bytes come
+// in 512-byte chunks of 128 rows x 4 bytes; one chunk covers 128 elements of K in MXFP4 and 64 in
+// NVFP4, so a stage holds CH = 2 or 4 chunks per 128 rows, four tensor-memory columns each.
 #pragma once
 #include <cuda_bf16.h>
 #include "sm100_ptx.cuh"
 
 namespace torq {
 
-template <int BN, int NACC>
+template <int BN, int NACC, int FMT = FMT_MXFP4>
 struct GemmCfg {
   static constexpr int BM = 128;
   static constexpr int BK = 256;                       // elements of K per stage
   static constexpr int A_BYTES = BM * BK / 2;          // 16 KiB
   static constexpr int B_BYTES = BN * BK / 2;
-  static constexpr int SFA_BYTES = 1024;               // 128 rows x 8 K-blocks
-  static constexpr int SFB_BYTES = (BN / 128) * 1024;
+  static constexpr int CH = FMT == FMT_NVFP4 ? 4 : 2;  // scale chunks per stage and 128 rows
+  static constexpr int SFA_BYTES = CH * 512;
+  static constexpr int SFB_BYTES = (BN / 128) * SFA_BYTES;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
   static constexpr int STAGES = (BN == 256) ? 4 : 6;
   static constexpr int BAR_BYTES = 256;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + align slack
   static constexpr int ACC_COLS = NACC * BN;
-  static constexpr int SFA_COL = ACC_COLS;             // 2 K-chunks x 4 columns
-  static constexpr int SFB_COL = ACC_COLS + 8;         // 2 K-chunks x BN/32 columns
+  static constexpr int SFA_COL = ACC_COLS;             // CH chunks x 4 columns
+  static constexpr int SFB_COL = ACC_COLS + 4 * CH;    // CH chunks x BN/32 columns
   static constexpr int TMEM_COLS = 512;
   static constexpr int THREADS = 192;
-  static_assert(SFB_COL + 2 * (BN / 32) <= TMEM_COLS, "tensor memory budget");
+  static_assert(SFB_COL + CH * (BN / 32) <= TMEM_COLS, "tensor memory budget");
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
 
-template <int BN, int NACC>
+template <int BN, int NACC, int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(192, 1)
 mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const uint8_t* __restrict__ As, const uint8_t* __restrict__ Ws,
-                  void* __restrict__ Y, int y_is_bf16, int M, int N, int K, int* err_word) {
-  using C = GemmCfg<BN, NACC>;
+                  void* __restrict__ Y, int y_is_bf16, int M, int N, int K, float alpha, int* err_word) {
+  using C = GemmCfg<BN, NACC, FMT>;
+  constexpr int CH = C::CH;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -61,7 +68,7 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int n_tiles = (N + BN - 1) / BN;
   const int total_tiles = m_tiles * n_tiles;
   const int k_tiles = (K + C::BK - 1) / C::BK;          // K % 128 == 0: last stage may be half
-  const int kb4 = K / 128;                              // scale K-chunks (4 K-blocks each) per row
+  const int kb4 = K / (256 / CH);                       // scale chunks (4 K-blocks each) per row
   const int n_rowtiles = (N + 127) / 128;
 
   if (threadIdx.x == 0) {
@@ -89,13 +96,13 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int n_sfb_tiles = min(BN / 128, n_rowtiles - rt0);
       (void)mt;
       for (int kt = 0; kt < pre; ++kt) {
-        const uint32_t sf_bytes = 512u * min(2, kb4 - 2 * kt);
+        const uint32_t sf_bytes = 512u * min(CH, kb4 - CH * kt);
         const uint32_t st = smem_base + kt * C::STAGE_BYTES;
         mbar_arrive_expect_tx(full_bar(kt), C::A_BYTES + C::B_BYTES + sf_bytes * (1 + n_sfb_tiles));
         tma_load_2d(st + C::A_BYTES, &tmB, kt * 128, nt * BN, full_bar(kt));
         for (int t = 0; t < n_sfb_tiles; ++t)
-          bulk_load_1d(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * 1024,
-                       Ws + ((size_t)(rt0 + t) * kb4 + 2 * kt) * 512, sf_bytes, full_bar(kt));
+          bulk_load_1d(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * C::SFA_BYTES,
+                       Ws + ((size_t)(rt0 + t) * kb4 + CH * kt) * 512, sf_bytes, full_bar(kt));
       }
     }
     __syncwarp();
@@ -114,20 +121,20 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int s = it % C::STAGES;
         if (!mbar_wait_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
                        SITE_PRODUCER_EMPTY)) { ok = false; break; }
-        const int nchunk = min(2, kb4 - 2 * kt);
+        const int nchunk = min(CH, kb4 - CH * kt);
         const uint32_t sf_bytes = 512u * nchunk;
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
         if (elect_one()) {
           const bool w_issued = it < (uint32_t)pre;      // W side of this stage went out before the wait above
           if (!w_issued) mbar_arrive_expect_tx(full_bar(s), C::A_BYTES + C::B_BYTES + sf_bytes * (1 + n_sfb_tiles));
           tma_load_2d(st, &tmA, kt * 128, mt * C::BM, full_bar(s));
-          bulk_load_1d(st + C::A_BYTES + C::B_BYTES, As + ((size_t)mt * kb4 + 2 * kt) * 512, sf_bytes,
+          bulk_load_1d(st + C::A_BYTES + C::B_BYTES, As + ((size_t)mt * kb4 + CH * kt) * 512, sf_bytes,
                        full_bar(s));
           if (!w_issued) {
             tma_load_2d(st + C::A_BYTES, &tmB, kt * 128, nt * BN, full_bar(s));
             for (int t = 0; t < n_sfb_tiles; ++t)
-              bulk_load_1d(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * 1024,
-                           Ws + ((size_t)(rt0 + t) * kb4 + 2 * kt) * 512, sf_bytes, full_bar(s));
+              bulk_load_1d(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * C::SFA_BYTES,
+                           Ws + ((size_t)(rt0 + t) * kb4 + CH * kt) * 512, sf_bytes, full_bar(s));
           }
         }
         __syncwarp();
@@ -137,7 +144,8 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // ------------------------------------------------------------------ MMA issuer
     uint32_t it = 0, tcount = 0;
     bool ok = true;
-    constexpr uint32_t idesc0 = idesc_mxf4(128, BN, 0, 0), idesc2 = idesc_mxf4(128, BN, 2, 2);
+    constexpr uint32_t idesc0 = FMT == FMT_NVFP4 ? idesc_nvf4(128, BN) : idesc_mxf4(128, BN, 0, 0);
+    constexpr uint32_t idesc2 = FMT == FMT_NVFP4 ? idesc_nvf4(128, BN) : idesc_mxf4(128, BN, 2, 2);
     const uint32_t sfa_t = tmem_base + C::SFA_COL, sfb_t = tmem_base + C::SFB_COL;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
       const int a = tcount % NACC;
@@ -151,29 +159,36 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           ok = false; break;
         }
         tc_fence_after_sync();
-        const bool two = (kb4 - 2 * kt) >= 2;              // K % 256 == 128: the last stage is half
+        const bool two = (kb4 - CH * kt) >= CH;            // K % 256 == 128: the last stage is half
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
         const uint64_t adesc = make_desc(st, 16, 1024, kSwizzle128);
         const uint64_t bdesc = make_desc(st + C::A_BYTES, 16, 1024, kSwizzle128);
         const uint64_t sfa_d = make_desc(st + C::A_BYTES + C::B_BYTES, 0, 128, 0);
         const uint64_t sfb_d = make_desc(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES, 0, 128, 0);
         if (elect_one()) {
-          // scale tiles shared -> tensor memory (descriptor address unit = 16 B: +32 = next
-          // K-chunk, +64 = next 128-row tile of W), then 64 elements of K per instruction
+          // scale chunks shared -> tensor memory (descriptor address unit = 16 B: +32 = next
+          // chunk, + SFA_BYTES / 16 = next 128-row tile of W), then 64 elements of K per instruction
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            if (c == 0 || two) {
+          for (int c = 0; c < CH; ++c) {
+            if (c < CH / 2 || two) {
               tmem_cp_32x128b_warpx4(sfa_t + 4 * c, sfa_d + 32 * c);
 #pragma unroll
               for (int t = 0; t < BN / 128; ++t)
-                tmem_cp_32x128b_warpx4(sfb_t + c * (BN / 32) + 4 * t, sfb_d + 64 * t + 32 * c);
+                tmem_cp_32x128b_warpx4(sfb_t + c * (BN / 32) + 4 * t, sfb_d + (C::SFA_BYTES / 16) * t + 32 * c);
             }
           }
-          mma_mxf4(acc, adesc, bdesc, idesc0, sfa_t, sfb_t, kt != 0);
-          mma_mxf4(acc, adesc + 2, bdesc + 2, idesc2, sfa_t, sfb_t, 1);
-          if (two) {
-            mma_mxf4(acc, adesc + 4, bdesc + 4, idesc0, sfa_t + 4, sfb_t + BN / 32, 1);
-            mma_mxf4(acc, adesc + 6, bdesc + 6, idesc2, sfa_t + 4, sfb_t + BN / 32, 1);
+          if constexpr (FMT == FMT_NVFP4) {                // one chunk per instruction
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (j < 2 || two)
+                mma_nvf4(acc, adesc + 2 * j, bdesc + 2 * j, idesc0, sfa_t + 4 * j, sfb_t + j * (BN / 32), (kt | j) != 0);
+          } else {                                         // half a chunk (two scale bytes) per instruction
+            mma_mxf4(acc, adesc, bdesc, idesc0, sfa_t, sfb_t, kt != 0);
+            mma_mxf4(acc, adesc + 2, bdesc + 2, idesc2, sfa_t, sfb_t, 1);
+            if (two) {
+              mma_mxf4(acc, adesc + 4, bdesc + 4, idesc0, sfa_t + 4, sfb_t + BN / 32, 1);
+              mma_mxf4(acc, adesc + 6, bdesc + 6, idesc2, sfa_t + 4, sfb_t + BN / 32, 1);
+            }
           }
           tc_commit(empty_bar(s));
         }
@@ -201,6 +216,10 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         uint32_t v[32];
         tmem_ld_32x32(tacc + cc * 32, v);
         tmem_ld_wait();
+        if constexpr (FMT == FMT_NVFP4) {                // product of the two tensor scales
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
+        }
         if (cc == BN / 32 - 1) {                         // accumulator fully read: hand it back
           tc_fence_before_sync();
           __syncwarp();

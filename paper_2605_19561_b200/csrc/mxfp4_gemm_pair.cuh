@@ -15,38 +15,47 @@
 // Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (leader CTA only), warps 2..9 epilogue
 // (warp w reads lane quarter w%4, column half (w-2)/4).  Barriers as in the pair rotation kernel;
 // acc_empty takes one arrival per epilogue warp of both CTAs (16).
+//
+// FMT_NVFP4 runs the same pipeline with kind::mxf4nvf4 (one E4M3 scale per 16 elements of K:
+// four 512-byte scale chunks per stage and 128 rows instead of two) and multiplies the result by
+// the product of the two tensor scales in the epilogue.
 #pragma once
 #include <cuda_bf16.h>
 #include "sm100_ptx.cuh"
 
 namespace torq {
 
-struct GemmPairCfg {
+template <int FMT = FMT_MXFP4>
+struct GemmPairCfgT {
   static constexpr int BN = 256;
   static constexpr int BM = 128;                       // rows per CTA
   static constexpr int BK = 256;
   static constexpr int A_BYTES = BM * BK / 2;          // 16 KiB
   static constexpr int B_BYTES = (BN / 2) * BK / 2;    // 16 KiB
-  static constexpr int SFA_BYTES = 1024;
-  static constexpr int SFB_BYTES = 2048;               // both 128-row tiles of the W scales
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;   // 35 KiB
+  static constexpr int CH = FMT == FMT_NVFP4 ? 4 : 2;  // scale chunks per stage and 128 rows
+  static constexpr int SFA_BYTES = CH * 512;
+  static constexpr int SFB_BYTES = 2 * SFA_BYTES;      // both 128-row tiles of the W scales
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;   // 35 / 38 KiB
   static constexpr int STAGES = 5;
   static constexpr int OUT_WARP_BYTES = 32 * 128;      // per epilogue warp: 32 rows x 128 B, swizzled
   static constexpr int OUT_BYTES = 8 * OUT_WARP_BYTES;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_BYTES + 256 + 1024;
-  static constexpr int SFA_COL = 256;
-  static constexpr int SFB_COL = 264;
+  static constexpr int SFA_COL = 256;                  // CH chunks x 4 columns
+  static constexpr int SFB_COL = 256 + 4 * CH;         // CH chunks x 8 columns
   static constexpr int TMEM_COLS = 512;
   static constexpr int THREADS = 320;
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
+using GemmPairCfg = GemmPairCfgT<FMT_MXFP4>;
 
+template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(320, 1)
 mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                        const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB,
                        const __grid_constant__ CUtensorMap tmY, int y_is_bf16, int M, int N, int K,
-                       int* err_word) {
-  using C = GemmPairCfg;
+                       float alpha, int* err_word) {
+  using C = GemmPairCfgT<FMT>;
+  constexpr int CH = C::CH;
   constexpr int BN = C::BN;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -68,7 +77,7 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   const int n_tiles = (N + BN - 1) / BN;
   const int total_tiles = mp_tiles * n_tiles;
   const int k_tiles = (K + C::BK - 1) / C::BK;
-  const int kb4 = K / 128;
+  const int kb4 = K / (256 / CH);                      // scale chunks per row
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -101,9 +110,12 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         const uint32_t leader_full = map_to_cta(full_bar(kt), 0);
         if (rank == 0) mbar_arrive_expect_tx(full_bar(kt), 2 * C::STAGE_BYTES);
         tma_load_2d_pair(st + C::A_BYTES, &tmB, kt * 128, nt * BN + (int)rank * (BN / 2), leader_full);
-        tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES, &tmSFB, kt * 256, 2 * nt, leader_full);
-        tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + 1024, &tmSFB, kt * 256, 2 * nt + 1,
-                         leader_full);
+#pragma unroll
+        for (int t = 0; t < 2; ++t)                      // one 1 KiB box = two chunks
+#pragma unroll
+          for (int b = 0; b < CH / 2; ++b)
+            tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * C::SFA_BYTES + b * 1024, &tmSFB,
+                             (kt * (CH / 2) + b) * 256, 2 * nt + t, leader_full);
       }
     }
     __syncwarp();
@@ -130,14 +142,20 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           tma_load_2d_pair(st, &tmA, kt * 128, mt * C::BM, leader_full);
           if (!w_issued)
             tma_load_2d_pair(st + C::A_BYTES, &tmB, kt * 128, nt * BN + (int)rank * (BN / 2), leader_full);
-          // scale tiles: one row of the [row tile, K-chunk x 512 B] view per 128 rows, 1 KiB per
-          // stage (two K-chunks); anything outside the buffer arrives as zeros (scale 2^-127,
+          // scale tiles: one row of the [row tile, chunk x 512 B] view per 128 rows, in boxes of
+          // 1 KiB (two chunks); anything outside the buffer arrives as zeros (scale 2^-127 or 0,
           // multiplying operand data that is zero there as well).
-          tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES, &tmSFA, kt * 256, mt, leader_full);
-          if (!w_issued) {
-            tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES, &tmSFB, kt * 256, 2 * nt, leader_full);
-            tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + 1024, &tmSFB, kt * 256, 2 * nt + 1,
+#pragma unroll
+          for (int b = 0; b < CH / 2; ++b)
+            tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + b * 1024, &tmSFA, (kt * (CH / 2) + b) * 256, mt,
                              leader_full);
+          if (!w_issued) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+#pragma unroll
+              for (int b = 0; b < CH / 2; ++b)
+                tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * C::SFA_BYTES + b * 1024, &tmSFB,
+                                 (kt * (CH / 2) + b) * 256, 2 * nt + t, leader_full);
           }
         }
         __syncwarp();
@@ -148,7 +166,8 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     if (rank == 0) {
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      constexpr uint32_t idesc0 = idesc_mxf4(256, BN, 0, 0), idesc2 = idesc_mxf4(256, BN, 2, 2);
+      constexpr uint32_t idesc0 = FMT == FMT_NVFP4 ? idesc_nvf4(256, BN) : idesc_mxf4(256, BN, 0, 0);
+      constexpr uint32_t idesc2 = FMT == FMT_NVFP4 ? idesc_nvf4(256, BN) : idesc_mxf4(256, BN, 2, 2);
       const uint32_t sfa_t = tmem_base + C::SFA_COL, sfb_t = tmem_base + C::SFB_COL;
       for (int tile = pair; tile < total_tiles && ok; tile += npairs, ++tcount) {
         if (!mbar_wait_cluster_warp(acce_bar, (tcount & 1) ^ 1, cta_abort, err_word, SITE_MMA_ACC_EMPTY)) {
@@ -161,28 +180,36 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             ok = false; break;
           }
           tc_fence_after_sync();
-          const bool two = (kb4 - 2 * kt) >= 2;            // K % 256 == 128: the last stage is half
+          const bool two = (kb4 - CH * kt) >= CH;          // K % 256 == 128: the last stage is half
           const uint32_t st = smem_base + s * C::STAGE_BYTES;
           const uint64_t adesc = make_desc(st, 16, 1024, kSwizzle128);
           const uint64_t bdesc = make_desc(st + C::A_BYTES, 16, 1024, kSwizzle128);
           const uint64_t sfa_d = make_desc(st + C::A_BYTES + C::B_BYTES, 0, 128, 0);
           const uint64_t sfb_d = make_desc(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES, 0, 128, 0);
           if (elect_one()) {
-            // scale tiles shared -> tensor memory (descriptor address unit = 16 B: +32 = next
-            // K-chunk, +64 = second 128-row tile of W), then 64 elements of K per instruction
-            tmem_cp_32x128b_warpx4_pair(sfa_t, sfa_d);
-            tmem_cp_32x128b_warpx4_pair(sfb_t, sfb_d);
-            tmem_cp_32x128b_warpx4_pair(sfb_t + 4, sfb_d + 64);
-            if (two) {
-              tmem_cp_32x128b_warpx4_pair(sfa_t + 4, sfa_d + 32);
-              tmem_cp_32x128b_warpx4_pair(sfb_t + 8, sfb_d + 32);
-              tmem_cp_32x128b_warpx4_pair(sfb_t + 12, sfb_d + 96);
+            // scale chunks shared -> tensor memory (descriptor address unit = 16 B: +32 = next
+            // chunk, + SFA_BYTES / 16 = second 128-row tile of W), then 64 elements of K per instruction
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+              if (c < CH / 2 || two) {
+                tmem_cp_32x128b_warpx4_pair(sfa_t + 4 * c, sfa_d + 32 * c);
+                tmem_cp_32x128b_warpx4_pair(sfb_t + 8 * c, sfb_d + 32 * c);
+                tmem_cp_32x128b_warpx4_pair(sfb_t + 8 * c + 4, sfb_d + 32 * c + C::SFA_BYTES / 16);
+              }
             }
-            mma_mxf4_pair(tmem_base, adesc, bdesc, idesc0, sfa_t, sfb_t, kt != 0);
-            mma_mxf4_pair(tmem_base, adesc + 2, bdesc + 2, idesc2, sfa_t, sfb_t, 1);
-            if (two) {
-              mma_mxf4_pair(tmem_base, adesc + 4, bdesc + 4, idesc0, sfa_t + 4, sfb_t + 8, 1);
-              mma_mxf4_pair(tmem_base, adesc + 6, bdesc + 6, idesc2, sfa_t + 4, sfb_t + 8, 1);
+            if constexpr (FMT == FMT_NVFP4) {              // one chunk per instruction
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                if (j < 2 || two)
+                  mma_nvf4_pair(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc0, sfa_t + 4 * j, sfb_t + 8 * j,
+                                (kt | j) != 0);
+            } else {                                       // half a chunk (two scale bytes) per instruction
+              mma_mxf4_pair(tmem_base, adesc, bdesc, idesc0, sfa_t, sfb_t, kt != 0);
+              mma_mxf4_pair(tmem_base, adesc + 2, bdesc + 2, idesc2, sfa_t, sfb_t, 1);
+              if (two) {
+                mma_mxf4_pair(tmem_base, adesc + 4, bdesc + 4, idesc0, sfa_t + 4, sfb_t + 8, 1);
+                mma_mxf4_pair(tmem_base, adesc + 6, bdesc + 6, idesc2, sfa_t + 4, sfb_t + 8, 1);
+              }
             }
             tc_commit_pair(empty_bar(s), 3);
           }
@@ -216,6 +243,15 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar, 0));   // accumulator is free again
+      if constexpr (FMT == FMT_NVFP4) {                    // product of the two tensor scales
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          v0[j] = __float_as_uint(__uint_as_float(v0[j]) * alpha);
+          v1[j] = __float_as_uint(__uint_as_float(v1[j]) * alpha);
+          v2[j] = __float_as_uint(__uint_as_float(v2[j]) * alpha);
+          v3[j] = __float_as_uint(__uint_as_float(v3[j]) * alpha);
+        }
+      }
       // Registers -> this warp's staging buffer (one 128-byte row per lane, 16-byte pieces XORed
       // with row % 8 as the 128-byte TMA swizzle expects) -> TMA store of a [32 rows x 128 B] box.
       // The store clips rows >= M and columns >= N by itself.

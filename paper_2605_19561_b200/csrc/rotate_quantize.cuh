@@ -14,7 +14,7 @@
 // Two accumulator buffers (2 x BN columns) overlap the epilogue with the next tile's mainloop.
 #pragma once
 #include <cuda_bf16.h>
-#include "quantize.cuh"
+#include "nvfp4_quantize.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -37,11 +37,13 @@ struct RotCfg {
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
 
-template <int BN>
+// FMT_NVFP4: NVFP4 quantizer in the epilogue (two 16-element blocks per 32 columns, E4M3 scales,
+// `tensor_scale` the tensor's float32 scale; unused for MXFP4).
+template <int BN, int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(192, 1)
 rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
                        const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
-                       uint8_t* __restrict__ scales, int M, int d, int* err_word) {
+                       uint8_t* __restrict__ scales, int M, int d, float tensor_scale, int* err_word) {
   using C = RotCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -173,6 +175,8 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
       const int64_t row = (int64_t)mt * C::BM + q * 32 + lane;
       const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
       uint32_t sc_word = 0;
+      NvScale nvs = {};
+      if constexpr (FMT == FMT_NVFP4) nvs = nv_scale(tensor_scale);
 #pragma unroll 1
       for (int bb = 0; bb < BN / 32; ++bb) {
         uint32_t yv[32];
@@ -206,10 +210,22 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
         }
         uint4 cw;
         uint32_t sbyte;
-        quantize_block32(z, cw, sbyte);
+        if constexpr (FMT == FMT_NVFP4) nv_quantize_2x16(z, nvs, cw, sbyte);
+        else quantize_block32(z, cw, sbyte);
         const int blk = b0 + bb;
         if (row < M && blk < nblocks)
           *reinterpret_cast<uint4*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+        if constexpr (FMT == FMT_NVFP4) {                  // two 16-blocks = half a 4-byte group
+          sc_word |= sbyte << (16 * (bb & 1));
+          if (bb & 1) {
+            const int kb4n = (2 * nblocks + 3) / 4;
+            const int chunk = (b0 + bb) >> 1;
+            if (chunk < kb4n)
+              *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4n + chunk) * 512 + lane * 16 + q * 4) = sc_word;
+            sc_word = 0;
+          }
+          continue;
+        }
         sc_word |= sbyte << (8 * (bb & 3));
         if ((bb & 3) == 3) {                             // four K-blocks = one 4-byte group
           const int chunk = (b0 + bb) >> 2;

@@ -13,7 +13,7 @@
 // acc_empty[a] lives in the leader and takes one arrival per epilogue warp of both CTAs (16).
 #pragma once
 #include <cuda_bf16.h>
-#include "quantize.cuh"
+#include "nvfp4_quantize.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -37,10 +37,15 @@ struct RotPairCfg {
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
 
+// FMT_NVFP4: the same kernel with the NVFP4 quantizer in the epilogue (two 16-element blocks per
+// 32 columns, E4M3 scales, `tensor_scale` the tensor's float32 scale; unused for MXFP4).  R_intra
+// is still [d/32, 32, 32]; 16-wide rotations arrive as its block-diagonal form.  Every tile takes
+// the FMA form of the intra-block rotation.
+template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(320, 1)
 rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
                             const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
-                            uint8_t* __restrict__ scales, int M, int d, int* err_word) {
+                            uint8_t* __restrict__ scales, int M, int d, float tensor_scale, int* err_word) {
   using C = RotPairCfg;
   constexpr int BN = C::BN;
   extern __shared__ uint8_t smem_raw[];
@@ -191,7 +196,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
       const int mt = 2 * mp + (int)rank;
       const int a = tcount % C::NACC;
       const int b0 = nt * (BN / 32);
-      const bool last = tile + npairs >= total_tiles;
+      const bool last = FMT == FMT_MXFP4 && tile + npairs >= total_tiles;
       if (R_intra != nullptr) {
         // Executed by every epilogue thread for every tile, also after a wait has given up.
         named_barrier_sync(1, 256);
@@ -225,7 +230,9 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
       if (!last) {
         // ---- one row per thread, fp32 FMAs
         const int64_t row = (int64_t)mt * C::BM + q * 32 + lane;
-        uint32_t sc_word = 0;
+        uint32_t sc_word = 0, sc_word2 = 0;              // NVFP4: two groups of four 16-blocks
+        NvScale nvs = {};
+        if constexpr (FMT == FMT_NVFP4) nvs = nv_scale(tensor_scale);
 #pragma unroll 1
         for (int bb = 0; bb < 4; ++bb) {
           uint32_t yv[32];
@@ -245,14 +252,31 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
           }
           uint4 cw;
           uint32_t sbyte;
-          quantize_block32(z, cw, sbyte);
+          if constexpr (FMT == FMT_NVFP4) nv_quantize_2x16(z, nvs, cw, sbyte);
+          else quantize_block32(z, cw, sbyte);
           const int blk = b0 + h * 4 + bb;
           if (row < M && blk < nblocks)
             *reinterpret_cast<uint4*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
-          sc_word |= sbyte << (8 * bb);
+          if constexpr (FMT == FMT_NVFP4) {
+            if (blk >= nblocks) sbyte = 0;               // padding blocks decode to zero
+            if (bb < 2) sc_word |= sbyte << (16 * bb);
+            else sc_word2 |= sbyte << (16 * (bb - 2));
+          } else {
+            sc_word |= sbyte << (8 * bb);
+          }
         }
-        if (chunk < kb4 && mt < m_tiles)                 // the pair's second row tile may not exist
-          *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4 + chunk) * 512 + lane * 16 + q * 4) = sc_word;
+        if constexpr (FMT == FMT_NVFP4) {
+          const int kb4n = (2 * nblocks + 3) / 4;        // 4-byte groups of 16-block scales per row
+          if (mt < m_tiles) {
+            if (2 * chunk < kb4n)
+              *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4n + 2 * chunk) * 512 + lane * 16 + q * 4) = sc_word;
+            if (2 * chunk + 1 < kb4n)
+              *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4n + 2 * chunk + 1) * 512 + lane * 16 + q * 4) = sc_word2;
+          }
+        } else {
+          if (chunk < kb4 && mt < m_tiles)               // the pair's second row tile may not exist
+            *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4 + chunk) * 512 + lane * 16 + q * 4) = sc_word;
+        }
         continue;
       }
       // ---- accumulator fragment layout (16 rows at a time): thread t holds rows t/4 and t/4 + 8,

@@ -9,6 +9,7 @@
 #include "mxfp4_gemm.cuh"
 #include "mxfp4_gemm_pair.cuh"
 #include "quantize.cuh"
+#include "nvfp4_quantize.cuh"
 #include "rotate_quantize.cuh"
 #include "rotate_quantize_pair.cuh"
 #include "rotate_splitk.cuh"
@@ -92,17 +93,22 @@ static DeviceState* device_state() {
     }
     bool ok = opt_in_smem(mxfp4_gemm_kernel<256, 1>, GemmCfg<256, 1>::SMEM_BYTES) &&
               opt_in_smem(mxfp4_gemm_kernel<128, 2>, GemmCfg<128, 2>::SMEM_BYTES) &&
+              opt_in_smem(mxfp4_gemm_kernel<256, 1, FMT_NVFP4>, GemmCfg<256, 1, FMT_NVFP4>::SMEM_BYTES) &&
+              opt_in_smem(mxfp4_gemm_kernel<128, 2, FMT_NVFP4>, GemmCfg<128, 2, FMT_NVFP4>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_kernel<256>, RotCfg<256>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_kernel<128>, RotCfg<128>::SMEM_BYTES) &&
-              opt_in_smem(rotate_quantize_pair_kernel, RotPairCfg::SMEM_BYTES) &&
+              opt_in_smem(rotate_quantize_kernel<256, FMT_NVFP4>, RotCfg<256>::SMEM_BYTES) &&
+              opt_in_smem(rotate_quantize_pair_kernel<FMT_MXFP4>, RotPairCfg::SMEM_BYTES) &&
+              opt_in_smem(rotate_quantize_pair_kernel<FMT_NVFP4>, RotPairCfg::SMEM_BYTES) &&
               opt_in_smem(rotate_splitk_kernel, RotSplitCfg::SMEM_BYTES) &&
               opt_in_smem(rotate_structured_kernel, RotStructCfg::SMEM_BYTES) &&
-              opt_in_smem(mxfp4_gemm_pair_kernel, GemmPairCfg::SMEM_BYTES);
+              opt_in_smem(mxfp4_gemm_pair_kernel<FMT_MXFP4>, GemmPairCfg::SMEM_BYTES) &&
+              opt_in_smem(mxfp4_gemm_pair_kernel<FMT_NVFP4>, GemmPairCfgT<FMT_NVFP4>::SMEM_BYTES);
     if (!ok) return nullptr;
-    st.rot_pairs = max_active_pairs(rotate_quantize_pair_kernel, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
-                                    st.sm_count);
-    st.gemm_pairs = max_active_pairs(mxfp4_gemm_pair_kernel, GemmPairCfg::THREADS, GemmPairCfg::SMEM_BYTES,
-                                     st.sm_count);
+    st.rot_pairs = max_active_pairs(rotate_quantize_pair_kernel<FMT_MXFP4>, RotPairCfg::THREADS,
+                                    RotPairCfg::SMEM_BYTES, st.sm_count);
+    st.gemm_pairs = max_active_pairs(mxfp4_gemm_pair_kernel<FMT_NVFP4>, GemmPairCfg::THREADS,
+                                     GemmPairCfgT<FMT_NVFP4>::SMEM_BYTES, st.sm_count);
     if (st.rot_pairs < 1 || st.gemm_pairs < 1) return nullptr;
   }
   st.ready = true;
@@ -266,11 +272,14 @@ torq_status torq_quantize_mxfp4(const void* Z, torq_dtype z_dtype, int64_t M, in
 }
 
 // Steps 1-4.  `scratch` (may be NULL) is fp32 room for the split-K partials of the few-token path;
-// without enough of it the single-pass kernels run.
+// without enough of it the single-pass kernels run.  `fmt` FMT_NVFP4 (with its tensor scale) takes
+// the single-pass kernels always and needs R_inter.
 static torq_status rotate_quantize_impl(const void* X, const void* R_inter, const void* R_intra, int64_t M,
                                         int64_t d, void* out_codes, void* out_scales, void* scratch,
-                                        size_t scratch_bytes, void* stream) {
+                                        size_t scratch_bytes, void* stream, int fmt = FMT_MXFP4,
+                                        float tensor_scale = 0.0f) {
   if (!X || !out_codes || !out_scales) return TORQ_ERR_NULL;
+  if (fmt == FMT_NVFP4 && !R_inter) return TORQ_ERR_NULL;
   if (M < 1 || d < 32 || d % 32 != 0 || M > (1 << 30) || d > (1 << 24)) return TORQ_ERR_SHAPE;
   if (!aligned16(X) || !aligned16(out_codes) || !aligned16(out_scales) ||
       (R_inter && !aligned16(R_inter)) || (R_intra && !aligned16(R_intra)))
@@ -293,7 +302,7 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
   if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d, 128, 64) ||
       !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
     return TORQ_ERR_LAUNCH;
-  const int splits = rotation_splits(M, d, st->sm_count);
+  const int splits = fmt == FMT_NVFP4 ? 1 : rotation_splits(M, d, st->sm_count);
   if (splits >= 2 && scratch && scratch_bytes >= splitk_scratch_bytes(M, d, splits) &&
       (reinterpret_cast<uintptr_t>(scratch) & 15u) == 0) {
     // Few tokens: split K over the SMs, partial tiles to scratch, then reduce + intra + quantize.
@@ -315,15 +324,26 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
     const int ptiles = (int)((M + 255) / 256) * (int)((d + 255) / 256);
     const int max_pairs = st->rot_pairs;
     const int pairs = ptiles < max_pairs ? ptiles : max_pairs;
-    launch_tc(rotate_quantize_pair_kernel, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES, s, tmX,
-                tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, st->err_word);
+    if (fmt == FMT_NVFP4)
+      launch_tc(rotate_quantize_pair_kernel<FMT_NVFP4>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
+                s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d,
+                tensor_scale, st->err_word);
+    else
+      launch_tc(rotate_quantize_pair_kernel<FMT_MXFP4>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
+                s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
+                st->err_word);
     return launch_status();
   }
   const int m_tiles = (int)((M + 127) / 128);
   const int tiles = m_tiles * (int)((d + 255) / 256);
   const int grid = tiles < st->sm_count ? tiles : st->sm_count;
-  launch_tc(rotate_quantize_kernel<256>, 1, grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s, tmX, tmR,
-            static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, st->err_word);
+  if (fmt == FMT_NVFP4)
+    launch_tc(rotate_quantize_kernel<256, FMT_NVFP4>, 1, grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s,
+              tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, tensor_scale,
+              st->err_word);
+  else
+    launch_tc(rotate_quantize_kernel<256>, 1, grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s, tmX, tmR,
+              static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f, st->err_word);
   return launch_status();
 }
 
@@ -363,8 +383,12 @@ torq_status torq_rotate_quantize_structured(const void* X, const void* R_B, cons
   return TORQ_OK;
 }
 
-torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, const void* Ws, int64_t M,
-                            int64_t N, int64_t K, void* Y, torq_dtype y_dtype, void* stream) {
+}  // extern "C"
+
+// Step 5 for either format; `alpha` multiplies the NVFP4 result (product of the tensor scales).
+template <int FMT>
+static torq_status gemm_impl(const void* Aq, const void* As, const void* Wq, const void* Ws, int64_t M,
+                             int64_t N, int64_t K, void* Y, torq_dtype y_dtype, float alpha, void* stream) {
   if (!Aq || !As || !Wq || !Ws || !Y) return TORQ_ERR_NULL;
   if (M < 1 || N < 8 || K < 128 || K % 128 != 0 || N % 8 != 0 || M > (1 << 30) || N > (1 << 30) ||
       K > (1 << 24))
@@ -380,7 +404,7 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
   CUtensorMap tmA, tmB;
   if (M > 128) {
     CUtensorMap tmSFA, tmSFB;
-    const uint64_t kb4 = (uint64_t)(K / 128);
+    const uint64_t kb4 = (uint64_t)(K / (FMT == FMT_NVFP4 ? 64 : 128));   // 512-byte scale chunks per row
     if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, (uint64_t)(K / 2), 128, 128) ||
         !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)(K / 2), BN / 2, 128) ||
         !encode_2d(&tmSFA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, As, (uint64_t)((M + 127) / 128), kb4 * 128, 1, 256,
@@ -396,8 +420,8 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
     const int ptiles = (int)((M + 255) / 256) * (int)((N + BN - 1) / BN);
     const int max_pairs = st->gemm_pairs;
     const int pairs = ptiles < max_pairs ? ptiles : max_pairs;
-    launch_tc(mxfp4_gemm_pair_kernel, 2, 2 * pairs, GemmPairCfg::THREADS, GemmPairCfg::SMEM_BYTES, s, tmA, tmB,
-                tmSFA, tmSFB, tmY, ybf ? 1 : 0, (int)M, (int)N, (int)K, st->err_word);
+    launch_tc(mxfp4_gemm_pair_kernel<FMT>, 2, 2 * pairs, GemmPairCfgT<FMT>::THREADS, GemmPairCfgT<FMT>::SMEM_BYTES, s,
+              tmA, tmB, tmSFA, tmSFB, tmY, ybf ? 1 : 0, (int)M, (int)N, (int)K, alpha, st->err_word);
     return launch_status();
   }
   // One row tile: the work is streaming W once, so prefer the narrower tile while it still leaves
@@ -410,14 +434,116 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
   const int tiles = (int)((M + 127) / 128) * (int)((N + bn - 1) / bn);
   const int grid = tiles < st->sm_count ? tiles : st->sm_count;
   if (narrow)
-    launch_tc(mxfp4_gemm_kernel<128, 2>, 1, grid, GemmCfg<128, 2>::THREADS, GemmCfg<128, 2>::SMEM_BYTES, s, tmA,
-              tmB, static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y,
-              y_dtype == TORQ_BF16 ? 1 : 0, (int)M, (int)N, (int)K, st->err_word);
+    launch_tc(mxfp4_gemm_kernel<128, 2, FMT>, 1, grid, GemmCfg<128, 2, FMT>::THREADS, GemmCfg<128, 2, FMT>::SMEM_BYTES,
+              s, tmA, tmB, static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y,
+              y_dtype == TORQ_BF16 ? 1 : 0, (int)M, (int)N, (int)K, alpha, st->err_word);
   else
-    launch_tc(mxfp4_gemm_kernel<BN, 1>, 1, grid, GemmCfg<BN, 1>::THREADS, GemmCfg<BN, 1>::SMEM_BYTES, s, tmA, tmB,
-              static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y, y_dtype == TORQ_BF16 ? 1 : 0,
-              (int)M, (int)N, (int)K, st->err_word);
+    launch_tc(mxfp4_gemm_kernel<BN, 1, FMT>, 1, grid, GemmCfg<BN, 1, FMT>::THREADS, GemmCfg<BN, 1, FMT>::SMEM_BYTES, s,
+              tmA, tmB, static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y,
+              y_dtype == TORQ_BF16 ? 1 : 0, (int)M, (int)N, (int)K, alpha, st->err_word);
   return launch_status();
+}
+
+extern "C" {
+
+torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, const void* Ws, int64_t M,
+                            int64_t N, int64_t K, void* Y, torq_dtype y_dtype, void* stream) {
+  return gemm_impl<FMT_MXFP4>(Aq, As, Wq, Ws, M, N, K, Y, y_dtype, 1.0f, stream);
+}
+
+static inline bool scale_ok(float s) { return s > 0.0f && s <= 3.0e38f; }   // positive, finite
+
+torq_status torq_nvfp4_gemm(const void* Aq, const void* As, float a_tensor_scale, const void* Wq, const void* Ws,
+                            float w_tensor_scale, int64_t M, int64_t N, int64_t K, void* Y, torq_dtype y_dtype,
+                            void* stream) {
+  if (!scale_ok(a_tensor_scale) || !scale_ok(w_tensor_scale)) return TORQ_ERR_SHAPE;
+  return gemm_impl<FMT_NVFP4>(Aq, As, Wq, Ws, M, N, K, Y, y_dtype, a_tensor_scale * w_tensor_scale, stream);
+}
+
+size_t torq_nvfp4_scales_bytes(int64_t rows, int64_t k) {
+  if (rows <= 0 || k <= 0) return 0;
+  return (size_t)((rows + 127) / 128) * (size_t)((k / 16 + 3) / 4) * 512;
+}
+
+static size_t nvfp4_quantized_bytes(int64_t M, int64_t d) {
+  return ((size_t)M * (size_t)(d / 2) + 255) / 256 * 256 + torq_nvfp4_scales_bytes(M, d);
+}
+
+size_t torq_nvfp4_workspace_bytes(int64_t M, int64_t d, int64_t N) {
+  (void)N;
+  if (M <= 0 || d <= 0) return 0;
+  return nvfp4_quantized_bytes(M, d);
+}
+
+torq_status torq_expand_intra16(const void* R_intra16, int64_t d, void* R_intra32, void* stream) {
+  if (!R_intra16 || !R_intra32) return TORQ_ERR_NULL;
+  if (d < 32 || d % 32 != 0 || d > (1 << 24)) return TORQ_ERR_SHAPE;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  expand_intra16_kernel<<<ew_grid(d * 32, 256, st->sm_count), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(R_intra16), d / 32, static_cast<__nv_bfloat16*>(R_intra32));
+  return launch_status();
+}
+
+torq_status torq_quantize_nvfp4(const void* Z, torq_dtype z_dtype, int64_t M, int64_t d, float tensor_scale,
+                                void* out_codes, void* out_scales, void* stream) {
+  if (!Z || !out_codes || !out_scales) return TORQ_ERR_NULL;
+  if (M < 1 || d < 16 || d % 16 != 0 || M > (1 << 30) || d > (1 << 30) || !scale_ok(tensor_scale))
+    return TORQ_ERR_SHAPE;
+  if (z_dtype != TORQ_F32 && z_dtype != TORQ_BF16) return TORQ_ERR_SHAPE;
+  if (!aligned16(Z) || !aligned16(out_codes) || !aligned16(out_scales)) return TORQ_ERR_ALIGN;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t kb4 = (d / 16 + 3) / 4;
+  const int64_t items = ((M + 127) / 128 * 128) * ((kb4 * 64 + 255) / 256);   // warps
+  const int grid = ew_grid(items, 8, st->sm_count);
+  if (z_dtype == TORQ_F32)
+    nv_quantize_kernel<float><<<grid, 256, 0, s>>>(static_cast<const float*>(Z), M, d, tensor_scale,
+                                                   static_cast<uint8_t*>(out_codes), static_cast<uint8_t*>(out_scales));
+  else
+    nv_quantize_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(Z), M, d, tensor_scale,
+                                                           static_cast<uint8_t*>(out_codes),
+                                                           static_cast<uint8_t*>(out_scales));
+  return launch_status();
+}
+
+torq_status torq_rotate_quantize_nvfp4(const void* X, const void* R_inter, const void* R_intra32, int64_t M,
+                                       int64_t d, float tensor_scale, void* out_codes, void* out_scales,
+                                       void* stream) {
+  if (!scale_ok(tensor_scale)) return TORQ_ERR_SHAPE;
+  return rotate_quantize_impl(X, R_inter, R_intra32, M, d, out_codes, out_scales, nullptr, 0, stream, FMT_NVFP4,
+                              tensor_scale);
+}
+
+torq_status torq_rotated_linear_nvfp4(const void* X, const void* R_inter, const void* R_intra32, float x_tensor_scale,
+                                      const void* Wq, const void* Ws, float w_tensor_scale, int64_t M, int64_t d,
+                                      int64_t N, void* Y, torq_dtype y_dtype, void* workspace, size_t workspace_bytes,
+                                      void* dbg_codes, void* dbg_scales, void* stream) {
+  if (!X || !R_inter || !Wq || !Ws || !Y) return TORQ_ERR_NULL;
+  if (M < 1 || d < 128 || d % 128 != 0 || N < 8 || N % 8 != 0 || M > (1 << 30) || d > (1 << 24) ||
+      !scale_ok(x_tensor_scale) || !scale_ok(w_tensor_scale))
+    return TORQ_ERR_SHAPE;
+  if (!workspace || workspace_bytes < nvfp4_quantized_bytes(M, d)) return TORQ_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return TORQ_ERR_ALIGN;
+  uint8_t* codes = static_cast<uint8_t*>(workspace);
+  const size_t codes_bytes = (size_t)M * (size_t)(d / 2);
+  uint8_t* scales = codes + (codes_bytes + 255) / 256 * 256;
+  torq_status rc = rotate_quantize_impl(X, R_inter, R_intra32, M, d, codes, scales, nullptr, 0, stream, FMT_NVFP4,
+                                        x_tensor_scale);
+  if (rc != TORQ_OK) return rc;
+  rc = torq_nvfp4_gemm(codes, scales, x_tensor_scale, Wq, Ws, w_tensor_scale, M, N, d, Y, y_dtype, stream);
+  if (rc != TORQ_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dbg_codes &&
+      cudaMemcpyAsync(dbg_codes, codes, codes_bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return TORQ_ERR_LAUNCH;
+  if (dbg_scales && cudaMemcpyAsync(dbg_scales, scales, torq_nvfp4_scales_bytes(M, d),
+                                    cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return TORQ_ERR_LAUNCH;
+  return TORQ_OK;
 }
 
 // Steps 1-5 with `workspace_bytes` >= quantized_bytes(M, d) already checked by the caller: codes,

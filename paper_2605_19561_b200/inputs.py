@@ -100,6 +100,13 @@ def rotations(cfg: LayerConfig, d: int | None = None, device: str = "cpu"):
     return to_bf16_bits(r_inter), to_bf16_bits(r_intra), r_inter, r_intra
 
 
+def intra_rotations16(cfg: LayerConfig, d: int | None = None) -> np.ndarray:
+    """R_intra [d/16,16,16] as bfloat16 bit patterns: the intra-block rotations of a format whose
+    quantization block has 16 elements (stream 5 of the configuration)."""
+    d = cfg.d if d is None else d
+    return to_bf16_bits(orthogonal(16, _rng(cfg.cfg_id, 5), batch=d // 16))
+
+
 def weights(cfg: LayerConfig, d: int | None = None, N: int | None = None) -> np.ndarray:
     """W [d,N] ~ N(0, 0.02^2), float32 (the un-rotated weight of out = x W)."""
     d = cfg.d if d is None else d

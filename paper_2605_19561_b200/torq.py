@@ -58,6 +58,21 @@ def lib() -> ctypes.CDLL:
     L.torq_swizzle_scales.restype = ci
     L.torq_merge_rotations.argtypes = [vp, vp, i64, vp, vp]
     L.torq_merge_rotations.restype = ci
+    f32 = ctypes.c_float
+    L.torq_nvfp4_scales_bytes.argtypes = [i64, i64]
+    L.torq_nvfp4_scales_bytes.restype = sz
+    L.torq_nvfp4_workspace_bytes.argtypes = [i64, i64, i64]
+    L.torq_nvfp4_workspace_bytes.restype = sz
+    L.torq_expand_intra16.argtypes = [vp, i64, vp, vp]
+    L.torq_expand_intra16.restype = ci
+    L.torq_quantize_nvfp4.argtypes = [vp, ci, i64, i64, f32, vp, vp, vp]
+    L.torq_quantize_nvfp4.restype = ci
+    L.torq_rotate_quantize_nvfp4.argtypes = [vp, vp, vp, i64, i64, f32, vp, vp, vp]
+    L.torq_rotate_quantize_nvfp4.restype = ci
+    L.torq_nvfp4_gemm.argtypes = [vp, vp, f32, vp, vp, f32, i64, i64, i64, vp, ci, vp]
+    L.torq_nvfp4_gemm.restype = ci
+    L.torq_rotated_linear_nvfp4.argtypes = [vp, vp, vp, f32, vp, vp, f32, i64, i64, i64, vp, ci, vp, sz, vp, vp, vp]
+    L.torq_rotated_linear_nvfp4.restype = ci
     L.torq_probe_fp4_peak.argtypes = [ci, ctypes.POINTER(ctypes.c_double), vp]
     L.torq_probe_fp4_peak.restype = ci
     L.torq_status_string.argtypes = [ci]
@@ -273,3 +288,105 @@ def prepare_weights(R_inter, R_intra, W):
     finally:
         torch.backends.cuda.matmul.allow_tf32 = prev
     return torq_quantize_mxfp4(Wp)
+
+
+# ---- NVFP4 variant (16-element blocks, E4M3 block scales, float32 tensor scale) -----------------------
+def torq_nvfp4_scales_bytes(rows: int, k: int) -> int:
+    return lib().torq_nvfp4_scales_bytes(rows, k)
+
+
+def torq_nvfp4_workspace_bytes(M: int, d: int, N: int) -> int:
+    return lib().torq_nvfp4_workspace_bytes(M, d, N)
+
+
+def torq_expand_intra16(R_intra16, out=None, stream=None):
+    """[d/16,16,16] bf16 -> the 32-wide block-diagonal form [d/32,32,32] the rotation kernels take."""
+    _check(R_intra16, torch.bfloat16, "R_intra16")
+    d = R_intra16.shape[0] * 16
+    if out is None:
+        out = torch.empty((d // 32, 32, 32), dtype=torch.bfloat16, device=R_intra16.device)
+    _raise(lib().torq_expand_intra16(_ptr(R_intra16), d, _ptr(out), _stream(stream)), "torq_expand_intra16")
+    return out
+
+
+def torq_quantize_nvfp4(Z, tensor_scale: float, out_codes=None, out_scales=None, stream=None):
+    """Z [M,d] float32 or bfloat16 -> (codes [M,d/2] uint8, tiled E4M3 scale bytes uint8)."""
+    M, d = Z.shape
+    dt = TORQ_F32 if Z.dtype == torch.float32 else TORQ_BF16
+    _check(Z, torch.float32 if dt == TORQ_F32 else torch.bfloat16, "Z")
+    if out_codes is None:
+        out_codes = torch.empty((M, d // 2), dtype=torch.uint8, device=Z.device)
+    if out_scales is None:
+        out_scales = torch.empty(torq_nvfp4_scales_bytes(M, d), dtype=torch.uint8, device=Z.device)
+    _raise(lib().torq_quantize_nvfp4(_ptr(Z), dt, M, d, tensor_scale, _ptr(out_codes), _ptr(out_scales),
+                                     _stream(stream)), "torq_quantize_nvfp4")
+    return out_codes, out_scales
+
+
+def torq_rotate_quantize_nvfp4(X, R_inter, R_intra32, tensor_scale: float, out_codes=None, out_scales=None,
+                               stream=None):
+    """X [M,d] bf16, R_inter [d,d] bf16, R_intra32 [d/32,32,32] bf16 or None (see torq_expand_intra16)."""
+    M, d = X.shape
+    for t, n in ((X, "X"), (R_inter, "R_inter"), (R_intra32, "R_intra32")):
+        _check(t, torch.bfloat16, n)
+    if out_codes is None:
+        out_codes = torch.empty((M, d // 2), dtype=torch.uint8, device=X.device)
+    if out_scales is None:
+        out_scales = torch.empty(torq_nvfp4_scales_bytes(M, d), dtype=torch.uint8, device=X.device)
+    _raise(lib().torq_rotate_quantize_nvfp4(_ptr(X), _ptr(R_inter), _ptr(R_intra32), M, d, tensor_scale,
+                                            _ptr(out_codes), _ptr(out_scales), _stream(stream)),
+           "torq_rotate_quantize_nvfp4")
+    return out_codes, out_scales
+
+
+def torq_nvfp4_gemm(Aq, As, a_tensor_scale: float, Wq, Ws, w_tensor_scale: float, out_dtype=torch.bfloat16, Y=None,
+                    stream=None):
+    """Aq [M,K/2], Wq [N,K/2] uint8 codes; As, Ws tiled E4M3 scale bytes -> Y [M,N]."""
+    M, K2 = Aq.shape
+    N = Wq.shape[0]
+    for t, n in ((Aq, "Aq"), (As, "As"), (Wq, "Wq"), (Ws, "Ws")):
+        _check(t, torch.uint8, n)
+    if Y is None:
+        Y = torch.empty((M, N), dtype=out_dtype, device=Aq.device)
+    _check(Y, Y.dtype, "Y")
+    dt = TORQ_F32 if Y.dtype == torch.float32 else TORQ_BF16
+    _raise(lib().torq_nvfp4_gemm(_ptr(Aq), _ptr(As), a_tensor_scale, _ptr(Wq), _ptr(Ws), w_tensor_scale, M, N,
+                                 2 * K2, _ptr(Y), dt, _stream(stream)), "torq_nvfp4_gemm")
+    return Y
+
+
+def torq_rotated_linear_nvfp4(X, R_inter, R_intra32, x_tensor_scale: float, Wq, Ws, w_tensor_scale: float,
+                              out_dtype=torch.bfloat16, Y=None, workspace=None, dbg_codes=None, dbg_scales=None,
+                              stream=None):
+    """Rotate, quantize to NVFP4 and multiply in one call.  Returns Y [M,N]."""
+    M, d = X.shape
+    N = Wq.shape[0]
+    for t, n in ((X, "X"), (R_inter, "R_inter"), (R_intra32, "R_intra32")):
+        _check(t, torch.bfloat16, n)
+    for t, n in ((Wq, "Wq"), (Ws, "Ws"), (dbg_codes, "dbg_codes"), (dbg_scales, "dbg_scales")):
+        _check(t, torch.uint8, n)
+    if Y is None:
+        Y = torch.empty((M, N), dtype=out_dtype, device=X.device)
+    if workspace is None:
+        workspace = torch.empty(torq_nvfp4_workspace_bytes(M, d, N), dtype=torch.uint8, device=X.device)
+    dt = TORQ_F32 if Y.dtype == torch.float32 else TORQ_BF16
+    _raise(lib().torq_rotated_linear_nvfp4(_ptr(X), _ptr(R_inter), _ptr(R_intra32), x_tensor_scale, _ptr(Wq),
+                                           _ptr(Ws), w_tensor_scale, M, d, N, _ptr(Y), dt, _ptr(workspace),
+                                           workspace.numel(), _ptr(dbg_codes), _ptr(dbg_scales), _stream(stream)),
+           "torq_rotated_linear_nvfp4")
+    return Y
+
+
+def prepare_weights_nvfp4(R_inter, R_intra32, W):
+    """Offline weight side in NVFP4: W' = R~^T W (as prepare_weights), tensor scale amax / (6 * 448),
+    quantized along K by torq_quantize_nvfp4.  Returns (Wq [N,d/2], Ws tiled, tensor_scale)."""
+    Rm = torq_merge_rotations(R_inter, R_intra32)
+    prev = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = False
+    try:
+        Wp = torch.matmul(W.t().contiguous().to(torch.float32), Rm).contiguous()
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = prev
+    ts = float(Wp.abs().max().item()) / (6.0 * 448.0)
+    Wq, Ws = torq_quantize_nvfp4(Wp, ts)
+    return Wq, Ws, ts
