@@ -69,6 +69,31 @@ __device__ __forceinline__ void nv_quantize_2x16(const float (&z)[32], const NvS
   sbytes = b0 | (b1 << 8);
 }
 
+// One row of 32 columns spread over the four lanes that share it in the warp-MMA accumulator layout
+// (lane p = lane % 4 holds v[2 nt + e] = element 8 nt + 2 p + e): the first block is nt 0..1, the
+// second nt 2..3.  Returns both scale bytes (first block in the low byte) and, in `word`, the four
+// code bytes 4p .. 4p+3 of the 32 columns.
+__device__ __forceinline__ void nv_quantize_row_fragment(const float (&v)[8], int p, const NvScale& s,
+                                                         uint32_t& word, uint32_t& sbytes) {
+  float a0 = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
+  float a1 = fmaxf(fmaxf(fabsf(v[4]), fabsf(v[5])), fmaxf(fabsf(v[6]), fabsf(v[7])));
+  a0 = fmaxf(a0, __shfl_xor_sync(0xFFFFFFFFu, a0, 1));
+  a1 = fmaxf(a1, __shfl_xor_sync(0xFFFFFFFFu, a1, 1));
+  a0 = fmaxf(a0, __shfl_xor_sync(0xFFFFFFFFu, a0, 2));
+  a1 = fmaxf(a1, __shfl_xor_sync(0xFFFFFFFFu, a1, 2));
+  uint32_t b0, b1;
+  float r0, r1;
+  nv_block_scale(a0, s, b0, r0);
+  nv_block_scale(a1, s, b1, r1);
+  sbytes = b0 | (b1 << 8);
+  const uint32_t w = pack8_e2m1(__fmul_rn(v[0], r0), __fmul_rn(v[1], r0), __fmul_rn(v[2], r0), __fmul_rn(v[3], r0),
+                                __fmul_rn(v[4], r1), __fmul_rn(v[5], r1), __fmul_rn(v[6], r1), __fmul_rn(v[7], r1));
+  const uint32_t w1 = __shfl_xor_sync(0xFFFFFFFFu, w, 1);                   // 4 x 4 byte transpose across the lanes
+  const uint32_t x = (p & 1) ? __byte_perm(w, w1, 0x3715) : __byte_perm(w, w1, 0x6240);
+  const uint32_t x2 = __shfl_xor_sync(0xFFFFFFFFu, x, 2);
+  word = (p & 2) ? __byte_perm(x, x2, 0x3276) : __byte_perm(x, x2, 0x5410);
+}
+
 // Quantize-only.  One warp handles 256 consecutive elements of a row (16 blocks): lane l owns
 // elements 8l..8l+7, two lanes share a block.  Rows M..Mpad-1 and blocks beyond d only get their
 // padding scale byte (0, which decodes to 0.0) written.

@@ -39,8 +39,7 @@ struct RotPairCfg {
 
 // FMT_NVFP4: the same kernel with the NVFP4 quantizer in the epilogue (two 16-element blocks per
 // 32 columns, E4M3 scales, `tensor_scale` the tensor's float32 scale; unused for MXFP4).  R_intra
-// is still [d/32, 32, 32]; 16-wide rotations arrive as its block-diagonal form.  Every tile takes
-// the FMA form of the intra-block rotation.
+// is still [d/32, 32, 32]; 16-wide rotations arrive as its block-diagonal form.
 template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(320, 1)
 rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
@@ -196,7 +195,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
       const int mt = 2 * mp + (int)rank;
       const int a = tcount % C::NACC;
       const int b0 = nt * (BN / 32);
-      const bool last = FMT == FMT_MXFP4 && tile + npairs >= total_tiles;
+      const bool last = tile + npairs >= total_tiles;
       if (R_intra != nullptr) {
         // Executed by every epilogue thread for every tile, also after a wait has given up.
         named_barrier_sync(1, 256);
@@ -283,6 +282,9 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
       //      eight columns of each per block
       const int64_t row_base = (int64_t)mt * C::BM + q * 32 + r8;     // + 16 mh + 8 rh
       uint32_t sc_word[4] = {0u, 0u, 0u, 0u};            // rows r8 + 16 mh + 8 rh -> index 2 mh + rh
+      uint32_t sc_hi[4] = {0u, 0u, 0u, 0u};              // NVFP4: second group of four 16-blocks
+      NvScale nvs = {};
+      if constexpr (FMT == FMT_NVFP4) nvs = nv_scale(tensor_scale);
 #pragma unroll 1
       for (int bb = 0; bb < 4; ++bb) {
         const int blk = b0 + h * 4 + bb;
@@ -340,15 +342,34 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
             const float v[8] = {acc[0][2 * rh], acc[0][2 * rh + 1], acc[1][2 * rh], acc[1][2 * rh + 1],
                                 acc[2][2 * rh], acc[2][2 * rh + 1], acc[3][2 * rh], acc[3][2 * rh + 1]};
             uint32_t word, sbyte;
-            quantize_row_fragment(v, p, word, sbyte);
+            if constexpr (FMT == FMT_NVFP4) nv_quantize_row_fragment(v, p, nvs, word, sbyte);
+            else quantize_row_fragment(v, p, word, sbyte);
             const int64_t row = row_base + 16 * mh + 8 * rh;
             if (row < M && blk < nblocks)
               *reinterpret_cast<uint32_t*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16 + 4 * p) = word;
-            sc_word[2 * mh + rh] |= sbyte << (8 * bb);
+            if constexpr (FMT == FMT_NVFP4) {
+              if (blk >= nblocks) sbyte = 0;
+              if (bb < 2) sc_word[2 * mh + rh] |= sbyte << (16 * bb);
+              else sc_hi[2 * mh + rh] |= sbyte << (16 * (bb - 2));
+            } else {
+              sc_word[2 * mh + rh] |= sbyte << (8 * bb);
+            }
           }
         }
       }
-      if (p == 0 && chunk < kb4 && mt < m_tiles) {       // the pair's second row tile may not exist
+      if constexpr (FMT == FMT_NVFP4) {
+        const int kb4n = (2 * nblocks + 3) / 4;
+        if (p == 0 && mt < m_tiles) {
+#pragma unroll
+          for (int rs = 0; rs < 4; ++rs) {
+            const size_t in_tile = (size_t)(r8 + 16 * (rs >> 1) + 8 * (rs & 1)) * 16 + q * 4;
+            if (2 * chunk < kb4n)
+              *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4n + 2 * chunk) * 512 + in_tile) = sc_word[rs];
+            if (2 * chunk + 1 < kb4n)
+              *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4n + 2 * chunk + 1) * 512 + in_tile) = sc_hi[rs];
+          }
+        }
+      } else if (p == 0 && chunk < kb4 && mt < m_tiles) {  // the pair's second row tile may not exist
 #pragma unroll
         for (int rs = 0; rs < 4; ++rs)
           *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4 + chunk) * 512 +
