@@ -204,6 +204,14 @@ def main():
     X0 = I.bf16_bits_to_tensor(xb, "cuda")
     R0, Ri0 = I.bf16_bits_to_tensor(rb, "cuda"), I.bf16_bits_to_tensor(rib, "cuda")
     Wq0, Ws0 = torq.prepare_weights(R0, Ri0, torch.from_numpy(w).cuda())
+    # the NVFP4 variant of the same layer (16-element blocks): its own intra rotations and weights
+    Ri32_nv = torq.torq_expand_intra16(I.bf16_bits_to_tensor(I.intra_rotations16(cfg), "cuda"))
+    torch.cuda.synchronize()
+    Wq_nv, Ws_nv, w_ts_nv = torq.prepare_weights_nvfp4(R0, Ri32_nv, torch.from_numpy(w).cuda())
+    # activation tensor scale, fixed ahead of time as a calibrated one would be: no rotated element
+    # exceeds its token's 2-norm, so the largest norm over the top of the E4M3 range never saturates
+    x_ts_nv = float(X0.float().norm(dim=1).max().item()) / (6.0 * 448.0)
+    ws_nv = [torch.empty(torq.torq_nvfp4_workspace_bytes(M, d, N), dtype=torch.uint8, device="cuda") for _ in range(2)]
     del w
     set_bytes = X0.numel() * 2 + R0.numel() * 2 + Wq0.numel() + M * N * 2
     n_sets = max(2, min(N_BUFFER_SETS, int(8e9 // set_bytes)))     # bounded device memory
@@ -301,6 +309,29 @@ def main():
             torq.torq_rotated_linear_structured(b["X"], RB, Ri1, b["Wq"], b["Ws"], Y=b["Y"], workspace=b["ws"])
 
         t_struct_layer = timed_loop(struct_layer)
+    # the NVFP4 variant: rotation + quantizer, GEMM, and the whole layer
+    def nv_codes_scales(k):
+        return (ws_nv[k][: M * d // 2].view(M, d // 2),
+                ws_nv[k][(M * d // 2 + 255) // 256 * 256:][: torq.torq_nvfp4_scales_bytes(M, d)])
+
+    nv_i = [0]
+
+    def nv_rot(b):
+        nv_i[0] ^= 1
+        c, sc = nv_codes_scales(nv_i[0])
+        torq.torq_rotate_quantize_nvfp4(b["X"], b["R"], Ri32_nv, x_ts_nv, out_codes=c, out_scales=sc)
+
+    def nv_gemm(b):
+        nv_i[0] ^= 1
+        c, sc = nv_codes_scales(nv_i[0])
+        torq.torq_nvfp4_gemm(c, sc, x_ts_nv, Wq_nv, Ws_nv, w_ts_nv, Y=b["Y"])
+
+    def nv_layer(b):
+        nv_i[0] ^= 1
+        torq.torq_rotated_linear_nvfp4(b["X"], b["R"], Ri32_nv, x_ts_nv, Wq_nv, Ws_nv, w_ts_nv, Y=b["Y"],
+                                       workspace=ws_nv[nv_i[0]])
+
+    t_nv_rot, t_nv_gemm, t_nv_layer = timed_loop(nv_rot), timed_loop(nv_gemm), timed_loop(nv_layer)
     barrier()
     clocks = sampler.stop()
     assert torq.torq_last_device_error() == 0
@@ -410,6 +441,14 @@ def main():
                 "speedup_over_dense_rotation": t_rot / t_struct,
                 "whole_layer_ms_per_step": t_struct_layer * 1e3, "whole_layer_tokens_per_s": world * M / t_struct_layer})(
                     2.0 * M * d + 2.0 * (d // 32) ** 2 + 2048.0 + M * d / 2 + M * d / 32),
+            "nvfp4_variant": {
+                "what": "the same layer in NVFP4 (16-element blocks, E4M3 block scales, float32 tensor scales; "
+                        "kind::mxf4nvf4 GEMM), single-pass rotation kernels",
+                "rotate_quant_ms": t_nv_rot * 1e3, "rotate_quant_TFLOPs": rot_flop / t_nv_rot / 1e12,
+                "rotate_quant_frac": rot_flop / t_nv_rot / 1e12 / bf16_peak,
+                "gemm_ms": t_nv_gemm * 1e3, "gemm_TFLOPs": gemm_flop / t_nv_gemm / 1e12,
+                "gemm_frac": gemm_flop / t_nv_gemm / 1e12 / fp4_peak,
+                "whole_layer_ms_per_step": t_nv_layer * 1e3, "whole_layer_tokens_per_s": world * M / t_nv_layer},
             "e2e": {"value": world * M / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": Xh.numel() * 2,
                     "d2h_bytes_per_step": Yh.numel() * 2},
             "gpu_launches": int(launches), "clocks": clocks,
