@@ -224,6 +224,28 @@ torq_status torq_rotated_linear_nvfp4(const void* X, const void* R_inter, const 
                                       torq_dtype y_dtype, void* workspace, size_t workspace_bytes,
                                       void* dbg_codes, void* dbg_scales, void* stream);
 
+/* ---- calibration of the inter-block rotation (Section 5.1; offline, not on the inference path) ----
+ * Covariance across the blocks of a token, pooled over the T calibration tokens and the 32
+ * positions of a block (block means taken as zero, as Section 5.1 assumes):
+ *   Sigma[b, b'] = (1 / (32 T)) sum_t sum_k x[t, 32 b + k] x[t, 32 b' + k]
+ * X [T, d] bf16, Sigma_f64 [d/32, d/32] float64 (written whole); d % 32 == 0.  float64 accumulation. */
+torq_status torq_block_covariance(const void* X, int64_t T, int64_t d, void* Sigma_f64, void* stream);
+
+/* Algorithm 1 (Givens rotations for variance equalisation): an orthogonal Q with
+ * diag(Q Sigma Q^T) = (tr Sigma / B) 1 up to the absolute threshold eps -- the matrix R_B that
+ * torq_rotate_quantize_structured applies across the blocks of a token.  Departures from the
+ * listing, which cannot reach its own stated output as printed: the rotation angle is the one that
+ * sets sigma_ii to the target exactly (the printed angle zeroes sigma_ij instead and spreads the two
+ * variances); the pair is (largest deviation, smallest deviation), ties to the lowest index; the
+ * matrix returned is the transpose of the listing's accumulated product, so that the output line
+ * holds as written.  At most B - 1 rotations.
+ *   Sigma_f64 [B, B] float64: in Sigma, out Q Sigma Q^T;  Q_f64 [B, B] float64;
+ *   Q_bf16 [B, B] bf16 or NULL (Q rounded through float32);  n_rotations: device int32 or NULL.
+ * One CTA; float64, one rounding per operation (no fused multiply-add), so the result is defined
+ * bit for bit.  1 <= B <= 32768, eps >= 0. */
+torq_status torq_givens_equalize(void* Sigma_f64, int64_t B, double eps, void* Q_f64, void* Q_bf16,
+                                 void* n_rotations, void* stream);
+
 /* Measurement tool (no counterpart in the paper): runs `groups` groups of four block-scaled FP4
  * tensor-core instructions (256 x 256 x 64 each, the GEMM's own instruction) per CTA pair on operands
  * that already sit in shared memory, with no loads and no epilogue, times them with CUDA events on

@@ -15,6 +15,7 @@
 #include "rotate_splitk.cuh"
 #include "rotate_structured.cuh"
 #include "fp4_peak_probe.cuh"
+#include "calibrate.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -670,6 +671,33 @@ torq_status torq_probe_fp4_peak(int groups, double* tflops, void* stream) {
   if (!ok) return TORQ_ERR_LAUNCH;
   *tflops = (double)pairs * groups * 4.0 * 2.0 * 256.0 * 256.0 * 64.0 / ((double)ms * 1e-3) / 1e12;
   return TORQ_OK;
+}
+
+torq_status torq_block_covariance(const void* X, int64_t T, int64_t d, void* Sigma_f64, void* stream) {
+  if (!X || !Sigma_f64) return TORQ_ERR_NULL;
+  if (T < 1 || d < 32 || d % 32 != 0 || T > (1 << 30) || d > (1 << 20)) return TORQ_ERR_SHAPE;
+  if (!aligned16(X) || !aligned16(Sigma_f64)) return TORQ_ERR_ALIGN;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  const unsigned tiles = (unsigned)((d / 32 + 15) / 16);
+  block_covariance_kernel<<<dim3(tiles, tiles, 1), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(X), T, d, static_cast<double*>(Sigma_f64));
+  return launch_status();
+}
+
+torq_status torq_givens_equalize(void* Sigma_f64, int64_t B, double eps, void* Q_f64, void* Q_bf16,
+                                 void* n_rotations, void* stream) {
+  if (!Sigma_f64 || !Q_f64) return TORQ_ERR_NULL;
+  if (B < 1 || B > 32768 || !(eps >= 0.0)) return TORQ_ERR_SHAPE;
+  if (!aligned16(Sigma_f64) || !aligned16(Q_f64) || (Q_bf16 && !aligned16(Q_bf16))) return TORQ_ERR_ALIGN;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  givens_equalize_kernel<<<1, 512, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<double*>(Sigma_f64), (int)B, eps, static_cast<double*>(Q_f64), static_cast<__nv_bfloat16*>(Q_bf16),
+      static_cast<int*>(n_rotations), (int)(4 * B));
+  return launch_status();
 }
 
 torq_status torq_swizzle_scales(const void* linear_scales, int64_t rows, int64_t k, void* out,

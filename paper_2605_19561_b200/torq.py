@@ -73,6 +73,10 @@ def lib() -> ctypes.CDLL:
     L.torq_nvfp4_gemm.restype = ci
     L.torq_rotated_linear_nvfp4.argtypes = [vp, vp, vp, f32, vp, vp, f32, i64, i64, i64, vp, ci, vp, sz, vp, vp, vp]
     L.torq_rotated_linear_nvfp4.restype = ci
+    L.torq_block_covariance.argtypes = [vp, i64, i64, vp, vp]
+    L.torq_block_covariance.restype = ci
+    L.torq_givens_equalize.argtypes = [vp, i64, ctypes.c_double, vp, vp, vp, vp]
+    L.torq_givens_equalize.restype = ci
     L.torq_probe_fp4_peak.argtypes = [ci, ctypes.POINTER(ctypes.c_double), vp]
     L.torq_probe_fp4_peak.restype = ci
     L.torq_status_string.argtypes = [ci]
@@ -390,3 +394,28 @@ def prepare_weights_nvfp4(R_inter, R_intra32, W):
     ts = float(Wp.abs().max().item()) / (6.0 * 448.0)
     Wq, Ws = torq_quantize_nvfp4(Wp, ts)
     return Wq, Ws, ts
+
+
+# ---- calibration of the inter-block rotation (Section 5.1, Algorithm 1; offline) -----------------------
+def torq_block_covariance(X, out=None, stream=None):
+    """X [T,d] bf16 -> Sigma [d/32,d/32] float64: covariance across blocks, pooled over tokens and positions."""
+    _check(X, torch.bfloat16, "X")
+    T, d = X.shape
+    if out is None:
+        out = torch.empty((d // 32, d // 32), dtype=torch.float64, device=X.device)
+    _check(out, torch.float64, "out")
+    _raise(lib().torq_block_covariance(_ptr(X), T, d, _ptr(out), _stream(stream)), "torq_block_covariance")
+    return out
+
+
+def torq_givens_equalize(Sigma, eps: float, stream=None):
+    """Algorithm 1 on Sigma [B,B] float64 (overwritten with Q Sigma Q^T).
+    Returns (Q float64 [B,B], Q bf16 [B,B], number of rotations as a device int32 tensor)."""
+    _check(Sigma, torch.float64, "Sigma")
+    B = Sigma.shape[0]
+    Q = torch.empty((B, B), dtype=torch.float64, device=Sigma.device)
+    Qb = torch.empty((B, B), dtype=torch.bfloat16, device=Sigma.device)
+    n = torch.zeros(4, dtype=torch.int32, device=Sigma.device)
+    _raise(lib().torq_givens_equalize(_ptr(Sigma), B, float(eps), _ptr(Q), _ptr(Qb), _ptr(n), _stream(stream)),
+           "torq_givens_equalize")
+    return Q, Qb, n[:1]
