@@ -98,6 +98,21 @@ __device__ __forceinline__ void split3_bf16x2(uint32_t x0, uint32_t x1, uint32_t
   f1 -= __uint_as_float(mid & 0xFFFF0000u);
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo) : "f"(f1), "f"(f0));
 }
+// The same split by truncation, with integer and add instructions only (no conversion unit): hi =
+// the top 16 bits of y, mid = the top 16 bits of y - hi, lo = what is left, which has at most eight
+// significant bits: y = hi + mid + lo exactly (subnormal leftovers aside).
+__device__ __forceinline__ void split3_trunc_bf16x2(uint32_t x0, uint32_t x1, uint32_t& hi, uint32_t& mid,
+                                                    uint32_t& lo) {
+  const uint32_t h0 = x0 & 0xFFFF0000u, h1 = x1 & 0xFFFF0000u;
+  const uint32_t r0 = __float_as_uint(__uint_as_float(x0) - __uint_as_float(h0));
+  const uint32_t r1 = __float_as_uint(__uint_as_float(x1) - __uint_as_float(h1));
+  const uint32_t m0 = r0 & 0xFFFF0000u, m1 = r1 & 0xFFFF0000u;
+  const uint32_t l0 = __float_as_uint(__uint_as_float(r0) - __uint_as_float(m0));
+  const uint32_t l1 = __float_as_uint(__uint_as_float(r1) - __uint_as_float(m1));
+  hi = __byte_perm(x0, x1, 0x7632);                      // high halves: element 0 in the low half
+  mid = __byte_perm(r0, r1, 0x7632);
+  lo = __byte_perm(l0, l1, 0x7632);
+}
 // D[16x8] += A[16x16] . B[16x8], bf16 inputs, fp32 accumulate (fragment layouts of the PTX ISA).
 __device__ __forceinline__ void mma_16816_bf16(float (&c)[4], const uint32_t* a, const uint32_t* b) {
   asm volatile(

@@ -21,8 +21,9 @@
 //
 // Persistent, warp-specialised: warp 0 TMA producer, warp 1 issues both kinds of MMA, warps 2..9
 // epilogue in two groups of four (lane quarter w % 4; group g = (w - 2) / 4 owns tokens 2g, 2g + 1
-// of the tile's four).  Per tile a group splits token 0, hands it to the MMA warp, splits token 1
-// while those MMAs run, then quantizes both.
+// of the tile's four).  The epilogue is software-pipelined across tiles: a group takes the step-3
+// result of a token of tile t out of tensor memory, splits the same token of tile t + 1 and hands it
+// to the MMA warp, and quantizes the values it took out while those MMAs run.
 #pragma once
 #include <cuda_bf16.h>
 #include "quantize.cuh"
@@ -204,27 +205,19 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
     }
     const int row = q * 32 + lane;                       // b' within the tile = tensor-memory lane
     const uint32_t row_sw = (uint32_t)((row >> 1) & 3);
-    uint32_t tcount = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-      const int bt = tile % b_tiles, tg = tile / b_tiles;
-      const int a = tcount & 1;
-      ok = mbar_wait(acc1f_bar(a), (tcount >> 1) & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
-      ok = __all_sync(0xFFFFFFFFu, ok);
-      if (!ok) break;
-      tc_fence_after_sync();
-      const uint32_t t1 = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
-      const int blk = bt * C::BM + row;
-      auto emit = [&](const float (&z)[32], int64_t token) {
-        uint4 cw;
-        uint32_t sbyte;
-        quantize_block32(z, cw, sbyte);
-        if (token < M && blk < nblocks) {
-          *reinterpret_cast<uint4*>(codes + token * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
-          scales[scale_offset(token, blk, kb4)] = (uint8_t)sbyte;
-        }
-      };
-      if (!intra) {
+    if (!intra) {
+      // no step 3: D1 is the result
+      uint32_t tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+        const int bt = tile % b_tiles, tg = tile / b_tiles;
+        const int a = tcount & 1;
+        ok = mbar_wait(acc1f_bar(a), (tcount >> 1) & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t t1 = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
+        const int blk = bt * C::BM + row;
 #pragma unroll 1
         for (int j = 0; j < 2; ++j) {
           uint32_t y[32];
@@ -238,18 +231,25 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
           float z[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(y[i]);
-          emit(z, (int64_t)tg * C::TOK + 2 * g + j);
+          uint4 cw;
+          uint32_t sbyte;
+          quantize_block32(z, cw, sbyte);
+          const int64_t token = (int64_t)tg * C::TOK + 2 * g + j;
+          if (token < M && blk < nblocks) {
+            *reinterpret_cast<uint4*>(codes + token * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+            scales[scale_offset(token, blk, kb4)] = (uint8_t)sbyte;
+          }
         }
-        continue;
       }
-      // ---- split y into three bf16 terms, one A tile row (64 B) per term and token
-#pragma unroll 1
-      for (int j = 0; j < 2; ++j) {
-        const int tok = 2 * g + j;
+    }
+    if (intra) {
+      // Splits one token of the tile whose D1 sits in buffer `a`: y -> hi + mid + lo bf16, one A tile row
+      // (64 B) per term, then hands the token to the MMA warp.  `last` = this warp's share of D1 is read.
+      auto split_token = [&](int a, int tok, bool last) {
         uint32_t y[32];
-        tmem_ld_32x32(t1 + tok * 32, y);
+        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + tok * 32, y);
         tmem_ld_wait();
-        if (j == 1) {                                    // this warp's share of D1 is read
+        if (last) {
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive(acc1e_bar(a));
@@ -259,7 +259,7 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
         for (int c = 0; c < 4; ++c) {                    // 8 values = one 16-byte piece per term
           uint32_t hi[4], mid[4], lo[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) split3_bf16x2(y[8 * c + 2 * e], y[8 * c + 2 * e + 1], hi[e], mid[e], lo[e]);
+          for (int e = 0; e < 4; ++e) split3_trunc_bf16x2(y[8 * c + 2 * e], y[8 * c + 2 * e + 1], hi[e], mid[e], lo[e]);
           const uint32_t off = (uint32_t)((c ^ row_sw) << 4);
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
                        ::"r"(dst + off), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
@@ -271,23 +271,59 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(a2f_bar(tok));        // four warps (the lane quarters) per token
-      }
-      // ---- D2 -> Eq. 1 -> codes and scales
-#pragma unroll 1
-      for (int j = 0; j < 2; ++j) {
-        const int tok = 2 * g + j;
-        ok = mbar_wait(a2d_bar(tok), tcount & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
+      };
+      // Software pipeline over this CTA's tiles: while the step-3 MMAs of a token run, the group
+      // quantizes the same token of the tile before.  Iteration t: for each of the group's two tokens,
+      // take D2 of tile t out of tensor memory (which frees D2 and the split tile of that token), split
+      // the token of tile t + 1 and hand it to the MMA warp, then run Eq. 1 on the values taken out.
+      uint32_t tcount = 0;
+      bool ok = true;
+      if ((int)blockIdx.x < total_tiles) {
+        ok = mbar_wait(acc1f_bar(0), 0, cta_abort, err_word, SITE_EPI_ACC_FULL);
         ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) break;
-        tc_fence_after_sync();
-        uint32_t y[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + C::ACC2_COL + tok * 32, y);
-        tmem_ld_wait();
-        tc_fence_before_sync();
-        float z[32];
+        if (ok) {
+          tc_fence_after_sync();
+          split_token(0, 2 * g, false);
+          split_token(0, 2 * g + 1, true);
+        }
+      }
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+        const int bt = tile % b_tiles, tg = tile / b_tiles;
+        const int blk = bt * C::BM + row;
+        const bool has_next = tile + (int)gridDim.x < total_tiles;
+        const int an = (tcount + 1) & 1;
+#pragma unroll 1
+        for (int j = 0; j < 2; ++j) {
+          const int tok = 2 * g + j;
+          ok = mbar_wait(a2d_bar(tok), tcount & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) break;
+          tc_fence_after_sync();
+          uint32_t zr[32];
+          tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + C::ACC2_COL + tok * 32, zr);
+          tmem_ld_wait();
+          tc_fence_before_sync();
+          if (has_next) {
+            if (j == 0) {
+              ok = mbar_wait(acc1f_bar(an), ((tcount + 1) >> 1) & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
+              ok = __all_sync(0xFFFFFFFFu, ok);
+              if (!ok) break;
+              tc_fence_after_sync();
+            }
+            split_token(an, tok, j == 1);
+          }
+          float z[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(y[i]);
-        emit(z, (int64_t)tg * C::TOK + tok);
+          for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(zr[i]);
+          uint4 cw;
+          uint32_t sbyte;
+          quantize_block32(z, cw, sbyte);
+          const int64_t token = (int64_t)tg * C::TOK + tok;
+          if (token < M && blk < nblocks) {
+            *reinterpret_cast<uint4*>(codes + token * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+            scales[scale_offset(token, blk, kb4)] = (uint8_t)sbyte;
+          }
+        }
       }
     }
   }
