@@ -40,13 +40,11 @@ struct RotStructCfg {
   static constexpr int B_BOX_BYTES = 32 * BK * 2;      // one token x 64 blocks = 4 KiB
   static constexpr int B_BYTES = TOK * B_BOX_BYTES;    // 16 KiB
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 32 KiB
-  static constexpr int STAGES = 3;
-  static constexpr int A2_TERM_BYTES = BM * 64;        // 128 rows x 32 bf16 = 8 KiB
-  static constexpr int A2_TOKEN_BYTES = 3 * A2_TERM_BYTES;
-  static constexpr int A2_BYTES = TOK * A2_TOKEN_BYTES;   // 96 KiB
+  static constexpr int STAGES = 6;
   static constexpr int RI_BYTES = 32 * 64;             // R_intra, 64-byte swizzle
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + A2_BYTES + RI_BYTES + 256 + 1024;
-  static constexpr int ACC2_COL = 2 * BN;              // D1 double-buffered in columns [0, 256)
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + RI_BYTES + 256 + 1024;
+  static constexpr int ACC2_COL = 2 * BN;              // D1 double-buffered in columns [0, 256); D2 in [256, 384)
+  static constexpr int LO_COL = ACC2_COL + BN;         // third split term: 16 columns per token, [384, 448)
   static constexpr int TMEM_COLS = 512;
   static constexpr int THREADS = 320;
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
@@ -63,9 +61,8 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t a2_base = smem_base + C::STAGES * C::STAGE_BYTES;
-  const uint32_t ri_base = a2_base + C::A2_BYTES;
-  const uint32_t bar_off = C::STAGES * C::STAGE_BYTES + C::A2_BYTES + C::RI_BYTES;
+  const uint32_t ri_base = smem_base + C::STAGES * C::STAGE_BYTES;
+  const uint32_t bar_off = C::STAGES * C::STAGE_BYTES + C::RI_BYTES;
   const uint32_t bar_base = smem_base + bar_off;
   // barrier map (8 bytes each)
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
@@ -152,8 +149,8 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
         const uint64_t bdesc = make_desc(st + C::A_BYTES, C::B_BOX_BYTES, 512, kSwizzle64);
         if (elect_one()) {
 #pragma unroll
-          for (int j = 0; j < C::BK / 16; ++j)          // 16 k-rows = 1 KiB
-            mma_bf16(acc, adesc + 2 * j, bdesc + 64 * j, idesc1, (kt | j) != 0);
+          for (int j = 0; j < C::BK / 16; ++j)          // 16 k-rows = 1 KiB; steps past the last block are skipped
+            if (kt * C::BK + j * 16 < nblocks) mma_bf16(acc, adesc + 2 * j, bdesc + 64 * j, idesc1, (kt | j) != 0);
           tc_commit(empty_bar(s));
         }
         __syncwarp();
@@ -173,13 +170,14 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
           tc_fence_after_sync();
           if (elect_one()) {
             const uint32_t d2 = tmem_base + C::ACC2_COL + tq * 32;
-#pragma unroll
-            for (int term = 0; term < 3; ++term) {
-              const uint64_t adesc = make_desc(a2_base + tq * C::A2_TOKEN_BYTES + term * C::A2_TERM_BYTES, 16, 512,
-                                               kSwizzle64);
-              mma_bf16(d2, adesc, rdesc, idesc2, term != 0);
-              mma_bf16(d2, adesc + 2, rdesc + 64, idesc2, 1);        // k 16..31: +32 B in A rows, +16 rows of R
-            }
+            const uint32_t d1 = tmem_base + (tcount & 1) * BN + tq * 32;      // hi, mid: over the token's y
+            const uint32_t lo = tmem_base + C::LO_COL + tq * 16;
+            mma_bf16_tmem_a(d2, d1, rdesc, idesc2, 0);
+            mma_bf16_tmem_a(d2, d1 + 8, rdesc + 64, idesc2, 1);              // k 16..31: +8 columns of A, +16 rows of R
+            mma_bf16_tmem_a(d2, d1 + 16, rdesc, idesc2, 1);
+            mma_bf16_tmem_a(d2, d1 + 24, rdesc + 64, idesc2, 1);
+            mma_bf16_tmem_a(d2, lo, rdesc, idesc2, 1);
+            mma_bf16_tmem_a(d2, lo + 8, rdesc + 64, idesc2, 1);
             tc_commit(a2d_bar(tq));
           }
           __syncwarp();
@@ -204,7 +202,6 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
       named_barrier_sync(1, 256);
     }
     const int row = q * 32 + lane;                       // b' within the tile = tensor-memory lane
-    const uint32_t row_sw = (uint32_t)((row >> 1) & 3);
     if (!intra) {
       // no step 3: D1 is the result
       uint32_t tcount = 0;
@@ -243,8 +240,9 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
       }
     }
     if (intra) {
-      // Splits one token of the tile whose D1 sits in buffer `a`: y -> hi + mid + lo bf16, one A tile row
-      // (64 B) per term, then hands the token to the MMA warp.  `last` = this warp's share of D1 is read.
+      // Splits one token of the tile whose D1 sits in buffer `a`: y -> hi + mid + lo bf16, written back to
+      // tensor memory as the A operand of step 3 (row b' = lane, two K-elements per column), then hands
+      // the token to the MMA warp.  `last` = this warp's share of D1 is read.
       auto split_token = [&](int a, int tok, bool last) {
         uint32_t y[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + tok * 32, y);
@@ -254,21 +252,15 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
           __syncwarp();
           if (lane == 0) mbar_arrive(acc1e_bar(a));
         }
-        const uint32_t dst = a2_base + tok * C::A2_TOKEN_BYTES + (uint32_t)row * 64;
+        uint32_t hi[16], mid[16], lo[16];                // packed pairs: column e = elements 2e, 2e + 1
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {                    // 8 values = one 16-byte piece per term
-          uint32_t hi[4], mid[4], lo[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) split3_trunc_bf16x2(y[8 * c + 2 * e], y[8 * c + 2 * e + 1], hi[e], mid[e], lo[e]);
-          const uint32_t off = (uint32_t)((c ^ row_sw) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(dst + off), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(dst + C::A2_TERM_BYTES + off), "r"(mid[0]), "r"(mid[1]), "r"(mid[2]), "r"(mid[3]) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(dst + 2 * C::A2_TERM_BYTES + off), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
-        }
-        fence_proxy_async_smem();
+        for (int e = 0; e < 16; ++e) split3_trunc_bf16x2(y[2 * e], y[2 * e + 1], hi[e], mid[e], lo[e]);
+        const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
+        tmem_st_32x32_x16(tq + a * BN + tok * 32, hi);   // hi and mid take the place of the token's y
+        tmem_st_32x32_x16(tq + a * BN + tok * 32 + 16, mid);
+        tmem_st_32x32_x16(tq + C::LO_COL + tok * 16, lo);
+        tmem_st_wait();
+        tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(a2f_bar(tok));        // four warps (the lane quarters) per token
       };
