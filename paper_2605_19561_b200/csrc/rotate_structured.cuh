@@ -19,11 +19,10 @@
 //   R_intra (bf16, exact) as the N-major B tile.  Six small MMAs (M 128, N 32, K 16) per token.
 //   D2 has lanes = b', 32 columns per token: one thread reads one (token, block) row and runs Eq. 1.
 //
-// Persistent, warp-specialised: warp 0 TMA producer, warp 1 issues both kinds of MMA, warps 2..9
-// epilogue in two groups of four (lane quarter w % 4; group g = (w - 2) / 4 owns tokens 2g, 2g + 1
-// of the tile's four).  The epilogue is software-pipelined across tiles: a group takes the step-3
-// result of a token of tile t out of tensor memory, splits the same token of tile t + 1 and hands it
-// to the MMA warp, and quantizes the values it took out while those MMAs run.
+// Persistent, warp-specialised: warp 0 TMA producer, warp 1 issues both kinds of MMA, warps 2..17
+// epilogue in four groups of four (lane quarter w % 4; group (w - 2) / 4 owns that token of the
+// tile's four): read y from tensor memory, split it, write the terms back to tensor memory as the A
+// operand of step 3, wait for the token's six MMAs, read D2, quantize, store.
 #pragma once
 #include <cuda_bf16.h>
 #include "quantize.cuh"
@@ -46,13 +45,13 @@ struct RotStructCfg {
   static constexpr int ACC2_COL = 2 * BN;              // D1 double-buffered in columns [0, 256); D2 in [256, 384)
   static constexpr int LO_COL = ACC2_COL + BN;         // third split term: 16 columns per token, [384, 448)
   static constexpr int TMEM_COLS = 512;
-  static constexpr int THREADS = 320;
+  static constexpr int THREADS = 576;                  // producer, MMA issuer, 16 epilogue warps
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
 
 // tmRB: R_B [B, B] bf16, box [128 x 64], 128-byte swizzle.  tmX3: X as (k, token, block), box (32, 1, 64),
 // 64-byte swizzle.
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(576, 1)
 rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_constant__ CUtensorMap tmX3,
                          const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
                          uint8_t* __restrict__ scales, int M, int d, int* err_word) {
@@ -85,7 +84,7 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(acc1f_bar(a), 1); mbar_init(acc1e_bar(a), 8); }
+    for (int a = 0; a < 2; ++a) { mbar_init(acc1f_bar(a), 1); mbar_init(acc1e_bar(a), 16); }
     for (int t = 0; t < C::TOK; ++t) { mbar_init(a2f_bar(t), 4); mbar_init(a2d_bar(t), 1); }
     *cta_abort = 0;
     fence_mbar_init();
@@ -165,7 +164,7 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
       if (!ok) break;
       if (intra) {
         for (int tok = 0; tok < C::TOK && ok; ++tok) {
-          const int tq = (tok & 1) * 2 + (tok >> 1);     // order: group 0 token 0, group 1 token 0, then tokens 1
+          const int tq = tok;
           if (!mbar_wait_warp(a2f_bar(tq), tcount & 1, cta_abort, err_word, SITE_MMA_FULL)) { ok = false; break; }
           tc_fence_after_sync();
           if (elect_one()) {
@@ -185,9 +184,13 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (two groups of 4 warps)
+    // ------------------------------------------------------------------ epilogue (four groups of 4 warps)
+    // Group g owns token g of every tile; inside a group warp q reads lane quarter q (32 output
+    // blocks).  Sixteen warps = four per scheduler: while one group waits for its step-3 MMAs the
+    // others split or quantize.  A warp whose 32 rows lie wholly beyond the last block (the second
+    // strip of a 160-block layer has 32 real rows of 128) only makes its barrier arrivals.
     const int q = warp & 3;
-    const int g = (warp - 2) >> 2;
+    const int tok = (warp - 2) >> 2;
     const int et = (warp - 2) * 32 + lane;
     if (intra) {
       // R_intra -> shared memory once: row k = 64 bytes, 16-byte piece c stored at c ^ ((k >> 1) & 3)
@@ -199,122 +202,68 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
                        "r"(v.z), "r"(v.w) : "memory");
       }
       fence_proxy_async_smem();                          // visible to the tensor core's reads
-      named_barrier_sync(1, 256);
+      named_barrier_sync(1, 512);
     }
     const int row = q * 32 + lane;                       // b' within the tile = tensor-memory lane
-    if (!intra) {
-      // no step 3: D1 is the result
-      uint32_t tcount = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-        const int bt = tile % b_tiles, tg = tile / b_tiles;
-        const int a = tcount & 1;
-        ok = mbar_wait(acc1f_bar(a), (tcount >> 1) & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
+    const uint32_t tlane = tmem_base + ((uint32_t)(q * 32) << 16);
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      const int bt = tile % b_tiles, tg = tile / b_tiles;
+      const int a = tcount & 1;
+      const int blk = bt * C::BM + row;
+      const bool live = bt * C::BM + q * 32 < nblocks;   // warp-uniform
+      const int64_t token = (int64_t)tg * C::TOK + tok;
+      ok = mbar_wait(acc1f_bar(a), (tcount >> 1) & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+      uint32_t y[32];
+      if (live) {
+        tmem_ld_32x32(tlane + a * BN + tok * 32, y);
+        tmem_ld_wait();
+      }
+      if (!intra) {                                      // no step 3: D1 is the result
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc1e_bar(a));
+      } else {
+        // y -> hi + mid + lo bf16, written back to tensor memory as the A operand of step 3 (row b' =
+        // lane, two K-elements per column): hi and mid over the token's y, lo in its own columns.  The
+        // MMA warp issues step 2 of the tile after next only after this tile's step 3, so D1 is free
+        // for it by the order of the tensor pipe; acc1e just counts the warps.
+        if (live) {
+          uint32_t hi[16], mid[16], lo[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) split3_trunc_bf16x2(y[2 * e], y[2 * e + 1], hi[e], mid[e], lo[e]);
+          tmem_st_32x32_x16(tlane + a * BN + tok * 32, hi);
+          tmem_st_32x32_x16(tlane + a * BN + tok * 32 + 16, mid);
+          tmem_st_32x32_x16(tlane + C::LO_COL + tok * 16, lo);
+          tmem_st_wait();
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) { mbar_arrive(acc1e_bar(a)); mbar_arrive(a2f_bar(tok)); }
+        ok = mbar_wait(a2d_bar(tok), tcount & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t t1 = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
-        const int blk = bt * C::BM + row;
-#pragma unroll 1
-        for (int j = 0; j < 2; ++j) {
-          uint32_t y[32];
-          tmem_ld_32x32(t1 + (2 * g + j) * 32, y);
+        if (live) {
+          tmem_ld_32x32(tlane + C::ACC2_COL + tok * 32, y);
           tmem_ld_wait();
-          if (j == 1) {
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc1e_bar(a));
-          }
-          float z[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(y[i]);
-          uint4 cw;
-          uint32_t sbyte;
-          quantize_block32(z, cw, sbyte);
-          const int64_t token = (int64_t)tg * C::TOK + 2 * g + j;
-          if (token < M && blk < nblocks) {
-            *reinterpret_cast<uint4*>(codes + token * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
-            scales[scale_offset(token, blk, kb4)] = (uint8_t)sbyte;
-          }
         }
-      }
-    }
-    if (intra) {
-      // Splits one token of the tile whose D1 sits in buffer `a`: y -> hi + mid + lo bf16, written back to
-      // tensor memory as the A operand of step 3 (row b' = lane, two K-elements per column), then hands
-      // the token to the MMA warp.  `last` = this warp's share of D1 is read.
-      auto split_token = [&](int a, int tok, bool last) {
-        uint32_t y[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + tok * 32, y);
-        tmem_ld_wait();
-        if (last) {
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(acc1e_bar(a));
-        }
-        uint32_t hi[16], mid[16], lo[16];                // packed pairs: column e = elements 2e, 2e + 1
-#pragma unroll
-        for (int e = 0; e < 16; ++e) split3_trunc_bf16x2(y[2 * e], y[2 * e + 1], hi[e], mid[e], lo[e]);
-        const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
-        tmem_st_32x32_x16(tq + a * BN + tok * 32, hi);   // hi and mid take the place of the token's y
-        tmem_st_32x32_x16(tq + a * BN + tok * 32 + 16, mid);
-        tmem_st_32x32_x16(tq + C::LO_COL + tok * 16, lo);
-        tmem_st_wait();
         tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(a2f_bar(tok));        // four warps (the lane quarters) per token
-      };
-      // Software pipeline over this CTA's tiles: while the step-3 MMAs of a token run, the group
-      // quantizes the same token of the tile before.  Iteration t: for each of the group's two tokens,
-      // take D2 of tile t out of tensor memory (which frees D2 and the split tile of that token), split
-      // the token of tile t + 1 and hand it to the MMA warp, then run Eq. 1 on the values taken out.
-      uint32_t tcount = 0;
-      bool ok = true;
-      if ((int)blockIdx.x < total_tiles) {
-        ok = mbar_wait(acc1f_bar(0), 0, cta_abort, err_word, SITE_EPI_ACC_FULL);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (ok) {
-          tc_fence_after_sync();
-          split_token(0, 2 * g, false);
-          split_token(0, 2 * g + 1, true);
-        }
       }
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-        const int bt = tile % b_tiles, tg = tile / b_tiles;
-        const int blk = bt * C::BM + row;
-        const bool has_next = tile + (int)gridDim.x < total_tiles;
-        const int an = (tcount + 1) & 1;
-#pragma unroll 1
-        for (int j = 0; j < 2; ++j) {
-          const int tok = 2 * g + j;
-          ok = mbar_wait(a2d_bar(tok), tcount & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
-          ok = __all_sync(0xFFFFFFFFu, ok);
-          if (!ok) break;
-          tc_fence_after_sync();
-          uint32_t zr[32];
-          tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + C::ACC2_COL + tok * 32, zr);
-          tmem_ld_wait();
-          tc_fence_before_sync();
-          if (has_next) {
-            if (j == 0) {
-              ok = mbar_wait(acc1f_bar(an), ((tcount + 1) >> 1) & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
-              ok = __all_sync(0xFFFFFFFFu, ok);
-              if (!ok) break;
-              tc_fence_after_sync();
-            }
-            split_token(an, tok, j == 1);
-          }
-          float z[32];
+      if (live) {
+        float z[32];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(zr[i]);
-          uint4 cw;
-          uint32_t sbyte;
-          quantize_block32(z, cw, sbyte);
-          const int64_t token = (int64_t)tg * C::TOK + tok;
-          if (token < M && blk < nblocks) {
-            *reinterpret_cast<uint4*>(codes + token * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
-            scales[scale_offset(token, blk, kb4)] = (uint8_t)sbyte;
-          }
+        for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(y[i]);
+        uint4 cw;
+        uint32_t sbyte;
+        quantize_block32(z, cw, sbyte);
+        if (token < M && blk < nblocks) {
+          *reinterpret_cast<uint4*>(codes + token * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+          scales[scale_offset(token, blk, kb4)] = (uint8_t)sbyte;
         }
       }
     }
