@@ -403,7 +403,12 @@ static torq_status gemm_impl(const void* Aq, const void* As, const void* Wq, con
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   constexpr int BN = 256;
   CUtensorMap tmA, tmB;
-  if (M > 128) {
+  // CTA pairs from two row tiles on -- except for exactly two row tiles with so few 256-column tiles
+  // that the pairs would leave more than half of the SMs idle: 128 x 128 tiles on single CTAs then
+  // put four times as many SMs to work on streaming W.
+  const int64_t pair_tiles = ((M + 255) / 256) * ((N + BN - 1) / BN);
+  const bool use_pairs = M > 128 && !(M <= 256 && 4 * pair_tiles <= st->sm_count);
+  if (use_pairs) {
     CUtensorMap tmSFA, tmSFB;
     const uint64_t kb4 = (uint64_t)(K / (FMT == FMT_NVFP4 ? 64 : 128));   // 512-byte scale chunks per row
     if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, (uint64_t)(K / 2), 128, 128) ||
@@ -425,9 +430,9 @@ static torq_status gemm_impl(const void* Aq, const void* As, const void* Wq, con
               tmA, tmB, tmSFA, tmSFB, tmY, ybf ? 1 : 0, (int)M, (int)N, (int)K, alpha, st->err_word);
     return launch_status();
   }
-  // One row tile: the work is streaming W once, so prefer the narrower tile while it still leaves
+  // One or two row tiles: the work is streaming W once, so prefer the narrower tile while it still leaves
   // SMs idle (128-column tiles double the number of CTAs pulling on memory).
-  const bool narrow = 2 * (int)((N + BN - 1) / BN) <= st->sm_count;
+  const bool narrow = 2 * (int)((M + 127) / 128) * (int)((N + BN - 1) / BN) <= st->sm_count;
   const uint32_t bn = narrow ? 128 : BN;
   if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, (uint64_t)(K / 2), 128, 128) ||
       !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)(K / 2), bn, 128))
