@@ -216,8 +216,9 @@ torq_status torq_nvfp4_gemm(const void* Aq, const void* As, float a_tensor_scale
                             void* Y, torq_dtype y_dtype, void* stream);
 
 /* Steps 1-5 in NVFP4: torq_rotate_quantize_nvfp4 into `workspace` (at least
- * torq_nvfp4_workspace_bytes(M, d, N) bytes, 256-byte aligned), then torq_nvfp4_gemm.
- * d % 128 == 0, N % 8 == 0. */
+ * torq_nvfp4_workspace_bytes(M, d, N) bytes, 256-byte aligned), then torq_nvfp4_gemm.  As in
+ * torq_rotated_linear, for few tokens the workspace also holds the fp32 partial tiles of the
+ * rotation split along its contraction.  d % 128 == 0, N % 8 == 0. */
 torq_status torq_rotated_linear_nvfp4(const void* X, const void* R_inter, const void* R_intra32,
                                       float x_tensor_scale, const void* Wq, const void* Ws,
                                       float w_tensor_scale, int64_t M, int64_t d, int64_t N, void* Y,

@@ -11,7 +11,7 @@
 // token are written as zeros; 32-row groups without any token are not written and not read).
 #pragma once
 #include <cuda_bf16.h>
-#include "quantize.cuh"
+#include "nvfp4_quantize.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -192,9 +192,12 @@ rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 //     block maximum over the four threads by two shuffles, Eq. 1, and one 4-byte code store per
 //     thread (the four threads of a row write its 16 bytes contiguously).
 // Rows M .. (group end) and K-blocks d/32 .. (padded to 4) only get their padding scale byte (0).
+// FMT_NVFP4: the 32 columns are two 16-element blocks (two threads each), E4M3 scales at twice the
+// block index, `tensor_scale` the tensor's float32 scale; the grid covers the padded 16-blocks in pairs.
+template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(256)
 splitk_reduce_quantize_kernel(const float* __restrict__ P, const __nv_bfloat16* __restrict__ R_intra,
-                              int M, int d, int splits, uint8_t* __restrict__ codes,
+                              int M, int d, int splits, float tensor_scale, uint8_t* __restrict__ codes,
                               uint8_t* __restrict__ scales) {
   __shared__ float y_s[32 * 33];                         // row stride 33: conflict-free by row and by column
   __shared__ __align__(16) float r_s[1024];
@@ -202,14 +205,21 @@ splitk_reduce_quantize_kernel(const float* __restrict__ P, const __nv_bfloat16* 
   griddep_wait();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int nb = d / 32;
-  const int kb4 = (nb + 3) / 4;
-  const int nbp = kb4 * 4;
+  const int kb4 = FMT == FMT_NVFP4 ? (2 * nb + 3) / 4 : (nb + 3) / 4;   // 4-byte scale groups per row
+  const int nbp = FMT == FMT_NVFP4 ? kb4 * 2 : kb4 * 4;                  // padded count of 32-column blocks
   const int b = blockIdx.x % nbp, rg = blockIdx.x / nbp;  // row group: rows 32 rg .. 32 rg + 31
   const int m_tiles = (M + 127) / 128;
   const int row0 = rg * 32;
   const int rows = max(0, min(32, M - row0));            // real rows of this group
   if (b >= nb || rows == 0) {                            // padding only: zero scale bytes
-    if (threadIdx.x < 32) scales[scale_offset(row0 + threadIdx.x, b, kb4)] = 0;
+    if (threadIdx.x < 32) {
+      if constexpr (FMT == FMT_NVFP4) {
+        scales[scale_offset(row0 + threadIdx.x, 2 * b, kb4)] = 0;
+        scales[scale_offset(row0 + threadIdx.x, 2 * b + 1, kb4)] = 0;
+      } else {
+        scales[scale_offset(row0 + threadIdx.x, b, kb4)] = 0;
+      }
+    }
     return;
   }
   const size_t split_stride = (size_t)m_tiles * 128 * d;
@@ -261,6 +271,18 @@ splitk_reduce_quantize_kernel(const float* __restrict__ P, const __nv_bfloat16* 
 #pragma unroll
   for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fabsf(z[j]));
   amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+  if constexpr (FMT == FMT_NVFP4) {                      // a 16-element block = two threads
+    uint32_t sb;
+    float rr;
+    nv_block_scale(amax, nv_scale(tensor_scale), sb, rr);
+    if (r < rows) {
+      const uint32_t w = pack8_e2m1(__fmul_rn(z[0], rr), __fmul_rn(z[1], rr), __fmul_rn(z[2], rr), __fmul_rn(z[3], rr),
+                                    __fmul_rn(z[4], rr), __fmul_rn(z[5], rr), __fmul_rn(z[6], rr), __fmul_rn(z[7], rr));
+      *reinterpret_cast<uint32_t*>(codes + (size_t)row * (d / 2) + b * 16 + 4 * p) = w;
+    }
+    if ((p & 1) == 0) scales[scale_offset(row, 2 * b + (p >> 1), kb4)] = r < rows ? (uint8_t)sb : (uint8_t)0;
+    return;
+  }
   amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
   uint32_t sbyte;
   float inv;

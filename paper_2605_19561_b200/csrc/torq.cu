@@ -273,8 +273,7 @@ torq_status torq_quantize_mxfp4(const void* Z, torq_dtype z_dtype, int64_t M, in
 }
 
 // Steps 1-4.  `scratch` (may be NULL) is fp32 room for the split-K partials of the few-token path;
-// without enough of it the single-pass kernels run.  `fmt` FMT_NVFP4 (with its tensor scale) takes
-// the single-pass kernels always and needs R_inter.
+// without enough of it the single-pass kernels run.  `fmt` FMT_NVFP4 (with its tensor scale) needs R_inter.
 static torq_status rotate_quantize_impl(const void* X, const void* R_inter, const void* R_intra, int64_t M,
                                         int64_t d, void* out_codes, void* out_scales, void* scratch,
                                         size_t scratch_bytes, void* stream, int fmt = FMT_MXFP4,
@@ -303,7 +302,7 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
   if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d, 128, 64) ||
       !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
     return TORQ_ERR_LAUNCH;
-  const int splits = fmt == FMT_NVFP4 ? 1 : rotation_splits(M, d, st->sm_count);
+  const int splits = rotation_splits(M, d, st->sm_count);
   if (splits >= 2 && scratch && scratch_bytes >= splitk_scratch_bytes(M, d, splits) &&
       (reinterpret_cast<uintptr_t>(scratch) & 15u) == 0) {
     // Few tokens: split K over the SMs, partial tiles to scratch, then reduce + intra + quantize.
@@ -316,8 +315,14 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
     launch_tc(rotate_splitk_kernel, 1, m_tiles * n_tiles * splits, RotSplitCfg::THREADS, RotSplitCfg::SMEM_BYTES, s, tmX, tmR,
               tmP, (int)M, (int)d, splits, st->err_word);
     if (launch_status() != TORQ_OK) return TORQ_ERR_LAUNCH;
-    launch_tc(splitk_reduce_quantize_kernel, 1, (int)(((d / 32 + 3) / 4) * 4) * m_tiles * 4, 256, 0, s, static_cast<const float*>(scratch),
-              static_cast<const __nv_bfloat16*>(R_intra), (int)M, (int)d, splits, codes, scales);
+    if (fmt == FMT_NVFP4)
+      launch_tc(splitk_reduce_quantize_kernel<FMT_NVFP4>, 1, (int)(((d / 16 + 3) / 4) * 2) * m_tiles * 4, 256, 0, s,
+                static_cast<const float*>(scratch), static_cast<const __nv_bfloat16*>(R_intra), (int)M, (int)d, splits,
+                tensor_scale, codes, scales);
+    else
+      launch_tc(splitk_reduce_quantize_kernel<FMT_MXFP4>, 1, (int)(((d / 32 + 3) / 4) * 4) * m_tiles * 4, 256, 0, s,
+                static_cast<const float*>(scratch), static_cast<const __nv_bfloat16*>(R_intra), (int)M, (int)d, splits,
+                0.0f, codes, scales);
     return launch_status();
   }
   if (M > 128) {
@@ -478,7 +483,7 @@ static size_t nvfp4_quantized_bytes(int64_t M, int64_t d) {
 size_t torq_nvfp4_workspace_bytes(int64_t M, int64_t d, int64_t N) {
   (void)N;
   if (M <= 0 || d <= 0) return 0;
-  return nvfp4_quantized_bytes(M, d);
+  return nvfp4_quantized_bytes(M, d) + splitk_scratch_bytes(M, d, rotation_splits(M, d, 0));
 }
 
 torq_status torq_expand_intra16(const void* R_intra16, int64_t d, void* R_intra32, void* stream) {
@@ -532,13 +537,14 @@ torq_status torq_rotated_linear_nvfp4(const void* X, const void* R_inter, const 
   if (M < 1 || d < 128 || d % 128 != 0 || N < 8 || N % 8 != 0 || M > (1 << 30) || d > (1 << 24) ||
       !scale_ok(x_tensor_scale) || !scale_ok(w_tensor_scale))
     return TORQ_ERR_SHAPE;
-  if (!workspace || workspace_bytes < nvfp4_quantized_bytes(M, d)) return TORQ_ERR_WORKSPACE;
+  if (!workspace || workspace_bytes < torq_nvfp4_workspace_bytes(M, d, N)) return TORQ_ERR_WORKSPACE;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return TORQ_ERR_ALIGN;
   uint8_t* codes = static_cast<uint8_t*>(workspace);
   const size_t codes_bytes = (size_t)M * (size_t)(d / 2);
   uint8_t* scales = codes + (codes_bytes + 255) / 256 * 256;
-  torq_status rc = rotate_quantize_impl(X, R_inter, R_intra32, M, d, codes, scales, nullptr, 0, stream, FMT_NVFP4,
-                                        x_tensor_scale);
+  const size_t used = nvfp4_quantized_bytes(M, d);
+  torq_status rc = rotate_quantize_impl(X, R_inter, R_intra32, M, d, codes, scales, codes + used,
+                                        workspace_bytes - used, stream, FMT_NVFP4, x_tensor_scale);
   if (rc != TORQ_OK) return rc;
   rc = torq_nvfp4_gemm(codes, scales, x_tensor_scale, Wq, Ws, w_tensor_scale, M, N, d, Y, y_dtype, stream);
   if (rc != TORQ_OK) return rc;

@@ -128,11 +128,11 @@ def test_gemm_exact_regime_is_bit_exact():
     assert (got == ref).all()
 
 
-@pytest.mark.parametrize("M", [128, 256])
+@pytest.mark.parametrize("M", [128, 256, 384])
 def test_gemm_one_hot_rows_pin_the_scale_assignment(M):
     """A one-hot activation row with value 1.0 returns one dequantized weight element times the row's
     own block scale: any mix-up of row <-> scale or 16-block <-> scale byte on either side, in either
-    kernel (one CTA: M <= 128; CTA pair: M > 128), shows up exactly.  Scales over the whole E4M3 range,
+    kernel (one CTA: M <= 128, and M = 256 with this few column tiles; CTA pair: M = 384), shows up exactly.  Scales over the whole E4M3 range,
     subnormals and zero included."""
     N, K = 256, 1024
     g = np.random.default_rng(5 + M)
@@ -271,6 +271,46 @@ def test_rotated_linear_end_to_end_tiny_config():
     # the layer approximates x W (two 4-bit operands)
     exact = O.decode_bf16(xb) @ w
     assert np.linalg.norm(got - exact) / np.linalg.norm(exact) < 0.25
+
+
+@pytest.mark.parametrize("M", [1, 33, 128])
+def test_rotated_linear_few_tokens_takes_the_split_rotation(M):
+    """Few tokens with a workspace: the rotation is split along its contraction over the SMs and a second
+    kernel adds the partials, rotates inside the blocks and quantizes (three launches instead of two)."""
+    cfg = I.CONFIGS["tiny"]
+    d, N = 1024, 256
+    xb = I.activations(cfg, M=M, d=d)
+    rb, _, _, _ = I.rotations(cfg, d=d)
+    ri16 = I.intra_rotations16(cfg, d=d)
+    z = O.rotate_blocks(xb, rb, ri16)
+    x_ts = O.tensor_scale_from_amax(np.abs(z).max())
+    g = np.random.default_rng(3)
+    wc = g.integers(0, 16, (N, d), dtype=np.uint8)
+    wsb = g.integers(0x30, 0x40, (N, d // 16), dtype=np.uint8)
+    ri32 = torq.torq_expand_intra16(dev_bf16(ri16))
+    dbg_c = torch.empty((M, d // 2), dtype=torch.uint8, device="cuda")
+    dbg_s = torch.empty(torq.torq_nvfp4_scales_bytes(M, d), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    n0 = torq.torq_launch_count()
+    y = torq.torq_rotated_linear_nvfp4(dev_bf16(xb), dev_bf16(rb), ri32, float(x_ts), dev_u8(O.pack_codes(wc)),
+                                       dev_u8(O.nv_swizzle_scales(wsb, d)), 0.01, out_dtype=torch.float32,
+                                       dbg_codes=dbg_c, dbg_scales=dbg_s)
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    assert torq.torq_launch_count() - n0 == 3
+    g_codes, g_sb = _to_numpy(dbg_c, dbg_s, M, d)
+    o_codes, o_sb = O.quantize_nvfp4(z.astype(np.float32), x_ts)
+    rep = _mismatch(g_codes, g_sb, o_codes, o_sb, x_ts)
+    assert rep["non_adjacent"] == 0 and rep["scale_off_by_more_than_one"] == 0, rep
+    assert rep["elem"] * M * d <= max(2, 1e-4 * M * d) and rep["blocks"] * M * (d // 16) <= max(1, 1e-4 * M * (d // 16)), rep
+    # padding of the scale tiles is zero
+    buf = dbg_s.cpu().numpy().copy()
+    rr, cc = np.meshgrid(np.arange(M), np.arange(d // 16), indexing="ij")
+    buf[O.nv_scale_layout_offset(rr, cc, d)] = 0
+    assert not buf.any()
+    ref = O.gemm_nvfp4(g_codes, g_sb, x_ts, wc, wsb, np.float32(0.01))
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
 
 
 def test_llama3_qkv_shape_sampled_rows():
