@@ -66,3 +66,35 @@ def test_argument_errors_are_status_codes():
     import ctypes as _c
     assert L.torq_probe_fp4_peak(0, _c.byref(_c.c_double()), None) == 2
     assert L.torq_status_string(0) == b"ok" and L.torq_status_string(6)
+
+
+def test_nvfp4_and_calibration_argument_errors_and_sizes():
+    L = torq.lib()
+    one = ctypes.c_void_p(16)
+    odd = ctypes.c_void_p(24)
+    # sizes: 16-element blocks -> twice the scale bytes of the 32-element layout for the same K
+    for rows, k in [(1, 64), (64, 256), (129, 4096), (200, 96)]:
+        assert torq.torq_nvfp4_scales_bytes(rows, k) == O.nv_scale_layout_bytes(rows, k)
+    assert torq.torq_nvfp4_scales_bytes(128, 4096) == 2 * torq.torq_scales_bytes(128, 4096)
+    assert torq.torq_nvfp4_workspace_bytes(2048, 4096, 6144) >= 2048 * 2048 + torq.torq_nvfp4_scales_bytes(2048, 4096)
+    # few tokens: room for the fp32 partials of the split rotation as well
+    assert torq.torq_nvfp4_workspace_bytes(16, 4096, 6144) > 16 * 2048 + torq.torq_nvfp4_scales_bytes(16, 4096) + 4 * 128 * 4096
+    assert L.torq_quantize_nvfp4(one, 0, 4, 64, 1.0, None, one, None) == 1
+    assert L.torq_quantize_nvfp4(one, 0, 4, 24, 1.0, one, one, None) == 2            # d % 16 != 0
+    assert L.torq_quantize_nvfp4(one, 0, 4, 64, 0.0, one, one, None) == 2            # tensor scale must be > 0
+    assert L.torq_quantize_nvfp4(one, 0, 4, 64, float("inf"), one, one, None) == 2
+    assert L.torq_quantize_nvfp4(odd, 0, 4, 64, 1.0, one, one, None) == 3
+    assert L.torq_rotate_quantize_nvfp4(one, None, None, 4, 64, 1.0, one, one, None) == 1    # R_inter is required
+    assert L.torq_rotate_quantize_nvfp4(one, one, None, 4, 64, -1.0, one, one, None) == 2
+    assert L.torq_nvfp4_gemm(one, one, 1.0, one, one, 1.0, 4, 8, 96, one, 0, None) == 2     # K % 128 != 0
+    assert L.torq_nvfp4_gemm(one, one, 0.0, one, one, 1.0, 4, 8, 128, one, 0, None) == 2
+    assert L.torq_nvfp4_gemm(one, None, 1.0, one, one, 1.0, 4, 8, 128, one, 0, None) == 1
+    assert L.torq_rotated_linear_nvfp4(one, one, one, 1.0, one, one, 1.0, 4, 128, 8, one, 0, one, 16, None, None,
+                                       None) == 7
+    assert L.torq_expand_intra16(None, 64, one, None) == 1
+    assert L.torq_expand_intra16(one, 48, one, None) == 2
+    assert L.torq_block_covariance(one, 4, 48, one, None) == 2
+    assert L.torq_block_covariance(None, 4, 64, one, None) == 1
+    assert L.torq_givens_equalize(one, 0, 1e-9, one, None, None, None) == 2
+    assert L.torq_givens_equalize(one, 8, -1.0, one, None, None, None) == 2
+    assert L.torq_givens_equalize(None, 8, 1e-9, one, None, None, None) == 1
