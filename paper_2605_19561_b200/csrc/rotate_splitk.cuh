@@ -187,10 +187,12 @@ rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 //  1. All warps add the partials P[s][row][32 b + j] in split order into a shared-memory tile
 //     (a warp reads one row's 128 bytes per split; all loads of the CTA are in flight together, so
 //     the phase costs one memory latency).
-//  2. Four threads per row, thread p of a row owning columns 8p .. 8p+7: the intra-block rotation
-//     z_j = sum_i y_i R[i][j] in fp32 FMAs in index order (y and R_intra[b] from shared memory),
-//     block maximum over the four threads by two shuffles, Eq. 1, and one 4-byte code store per
-//     thread (the four threads of a row write its 16 bytes contiguously).
+//  2. The intra-block rotation z = y R_intra[b] of the 32 x 32 tile on the warp-level tensor-core
+//     path (two warps, 16 rows each): y split into three bf16 terms, R_intra exact in bf16, fp32
+//     accumulation -- 48 MMAs instead of a thousand FMA instructions per warp, which is what the
+//     kernel's time was.  Then Eq. 1 on the accumulator fragments (four lanes share a row: block
+//     maximum by two shuffles, a 4 x 4 byte transpose so that each lane stores 4 contiguous code
+//     bytes).  Without R_intra: four threads per row on the sums themselves.
 // Rows M .. (group end) and K-blocks d/32 .. (padded to 4) only get their padding scale byte (0).
 // FMT_NVFP4: the 32 columns are two 16-element blocks (two threads each), E4M3 scales at twice the
 // block index, `tensor_scale` the tensor's float32 scale; the grid covers the padded 16-blocks in pairs.
@@ -200,7 +202,7 @@ splitk_reduce_quantize_kernel(const float* __restrict__ P, const __nv_bfloat16* 
                               int M, int d, int splits, float tensor_scale, uint8_t* __restrict__ codes,
                               uint8_t* __restrict__ scales) {
   __shared__ float y_s[32 * 33];                         // row stride 33: conflict-free by row and by column
-  __shared__ __align__(16) float r_s[1024];
+  __shared__ __align__(16) uint8_t r_s[32 * 80];         // R_intra[b], bf16, 80-byte rows: conflict-free ldmatrix
   griddep_launch_dependents();
   griddep_wait();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -235,38 +237,76 @@ splitk_reduce_quantize_kernel(const float* __restrict__ P, const __nv_bfloat16* 
     for (int s = 0; s < 8; ++s) if (s < splits) y += part[s];
     y_s[r * 33 + lane] = y;
   }
+  for (int r = rows + warp; r < 32; r += nwarps) y_s[r * 33 + lane] = 0.f;     // rows past M: zeros
   if (R_intra != nullptr && threadIdx.x < 128) {
-    float v[8];
-    load8(R_intra + (size_t)b * 1024 + threadIdx.x * 8, v);
-    *reinterpret_cast<float4*>(r_s + threadIdx.x * 8) = make_float4(v[0], v[1], v[2], v[3]);
-    *reinterpret_cast<float4*>(r_s + threadIdx.x * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+    const int i = threadIdx.x >> 2, c = (threadIdx.x & 3) * 8;
+    *reinterpret_cast<uint4*>(r_s + i * 80 + c * 2) =
+        __ldg(reinterpret_cast<const uint4*>(R_intra + (size_t)b * 1024 + threadIdx.x * 8));
   }
   __syncthreads();
-  // ---- 2. four threads per row
+  if (R_intra != nullptr) {
+    // ---- 2a. two warps, 16 rows each, on the warp-level tensor cores
+    if (warp >= 2) return;
+    const int p = lane & 3, r8 = lane >> 2;
+    uint32_t bfrag[2][4][2];                             // [k chunk][n tile][2]
+    {
+      // lane l: row l % 8 of matrix l / 8; matrices (k 0-7, n), (k 8-15, n), (k 0-7, n+8), (k 8-15, n+8)
+      const uint32_t rb = smem_u32(r_s) + (uint32_t)(((lane >> 3) & 1) * 8 + (lane & 7)) * 80 + (uint32_t)(lane >> 4) * 16;
+#pragma unroll
+      for (int kc = 0; kc < 2; ++kc)
+#pragma unroll
+        for (int np = 0; np < 2; ++np)
+          ldmatrix_x4_trans(rb + kc * 16 * 80 + np * 32, bfrag[kc][2 * np][0], bfrag[kc][2 * np][1],
+                            bfrag[kc][2 * np + 1][0], bfrag[kc][2 * np + 1][1]);
+    }
+    uint32_t ah[8], am[8], al[8];                        // A fragments: [k chunk * 4 + (n & 1) * 2 + row half]
+#pragma unroll
+    for (int n = 0; n < 4; ++n)
+#pragma unroll
+      for (int rh = 0; rh < 2; ++rh) {
+        const float* yp = y_s + (16 * warp + r8 + 8 * rh) * 33 + 8 * n + 2 * p;
+        const int ai = (n >> 1) * 4 + (n & 1) * 2 + rh;
+        split3_bf16x2(__float_as_uint(yp[0]), __float_as_uint(yp[1]), ah[ai], am[ai], al[ai]);
+      }
+    float acc[4][4];
+#pragma unroll
+    for (int n = 0; n < 4; ++n) { acc[n][0] = 0.f; acc[n][1] = 0.f; acc[n][2] = 0.f; acc[n][3] = 0.f; }
+#pragma unroll
+    for (int kc = 0; kc < 2; ++kc)
+#pragma unroll
+      for (int n = 0; n < 4; ++n) {
+        mma_16816_bf16(acc[n], al + 4 * kc, bfrag[kc][n]);
+        mma_16816_bf16(acc[n], am + 4 * kc, bfrag[kc][n]);
+        mma_16816_bf16(acc[n], ah + 4 * kc, bfrag[kc][n]);
+      }
+#pragma unroll
+    for (int rh = 0; rh < 2; ++rh) {
+      const float v[8] = {acc[0][2 * rh], acc[0][2 * rh + 1], acc[1][2 * rh], acc[1][2 * rh + 1],
+                          acc[2][2 * rh], acc[2][2 * rh + 1], acc[3][2 * rh], acc[3][2 * rh + 1]};
+      const int r = 16 * warp + r8 + 8 * rh;
+      const int row = row0 + r;
+      uint32_t word, sb;
+      if constexpr (FMT == FMT_NVFP4) nv_quantize_row_fragment(v, p, nv_scale(tensor_scale), word, sb);
+      else quantize_row_fragment(v, p, word, sb);
+      if (r < rows) *reinterpret_cast<uint32_t*>(codes + (size_t)row * (d / 2) + b * 16 + 4 * p) = word;
+      if (p == 0) {
+        if constexpr (FMT == FMT_NVFP4) {
+          scales[scale_offset(row, 2 * b, kb4)] = r < rows ? (uint8_t)(sb & 0xFF) : (uint8_t)0;
+          scales[scale_offset(row, 2 * b + 1, kb4)] = r < rows ? (uint8_t)(sb >> 8) : (uint8_t)0;
+        } else {
+          scales[scale_offset(row, b, kb4)] = r < rows ? (uint8_t)sb : (uint8_t)0;
+        }
+      }
+    }
+    return;
+  }
+  // ---- 2b. no intra rotation: four threads per row on the sums
   if (threadIdx.x >= 128) return;
   const int r = threadIdx.x >> 2, p = threadIdx.x & 3;
   const int row = row0 + r;
   float z[8];
-  if (r < rows) {
-    if (R_intra != nullptr) {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) z[j] = 0.f;
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const float yi = y_s[r * 33 + i];
-        const float4 ra = *reinterpret_cast<const float4*>(r_s + i * 32 + 8 * p);
-        const float4 rb = *reinterpret_cast<const float4*>(r_s + i * 32 + 8 * p + 4);
-        z[0] = fmaf(yi, ra.x, z[0]); z[1] = fmaf(yi, ra.y, z[1]); z[2] = fmaf(yi, ra.z, z[2]); z[3] = fmaf(yi, ra.w, z[3]);
-        z[4] = fmaf(yi, rb.x, z[4]); z[5] = fmaf(yi, rb.y, z[5]); z[6] = fmaf(yi, rb.z, z[6]); z[7] = fmaf(yi, rb.w, z[7]);
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) z[j] = y_s[r * 33 + 8 * p + j];
-    }
-  } else {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) z[j] = 0.f;
-  }
+  for (int j = 0; j < 8; ++j) z[j] = y_s[r * 33 + 8 * p + j];
   float amax = 0.f;
 #pragma unroll
   for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fabsf(z[j]));
