@@ -438,6 +438,7 @@ def main():
                 "R_intra (the paper's structure, 2d(B+32) flop per token) on the same activations", "bound": "hbm",
                 "ms_per_launch": t_struct * 1e3, "achieved": nbytes / t_struct / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": nbytes / t_struct / 1e9 / pk["hbm_gbs"], "algorithmic_bytes": nbytes,
+                "traffic": profiled_traffic("rotate_structured_kernel", args.workload),
                 "speedup_over_dense_rotation": t_rot / t_struct,
                 "whole_layer_ms_per_step": t_struct_layer * 1e3, "whole_layer_tokens_per_s": world * M / t_struct_layer})(
                     2.0 * M * d + 2.0 * (d // 32) ** 2 + 2048.0 + M * d / 2 + M * d / 32),
