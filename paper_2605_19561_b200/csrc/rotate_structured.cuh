@@ -19,10 +19,10 @@
 //   R_intra (bf16, exact) as the N-major B tile.  Six small MMAs (M 128, N 32, K 16) per token.
 //   D2 has lanes = b', 32 columns per token: one thread reads one (token, block) row and runs Eq. 1.
 //
-// Persistent, warp-specialised: warp 0 TMA producer, warp 1 issues both kinds of MMA, warps 2..17
-// epilogue in four groups of four (lane quarter w % 4; group (w - 2) / 4 owns that token of the
-// tile's four): read y from tensor memory, split it, write the terms back to tensor memory as the A
-// operand of step 3, wait for the token's six MMAs, read D2, quantize, store.
+// Persistent, warp-specialised: warp 0 TMA producer, warp 1 issues the step-2 MMAs, warp 18 the step-3
+// MMAs, warps 2..17 epilogue in four groups of four (lane quarter w % 4; group (w - 2) / 4 owns that
+// token of the tile's four): read y from tensor memory, split it, write the terms back to tensor
+// memory as the A operand of step 3, wait for the token's six MMAs, read D2, quantize, store.
 #pragma once
 #include <cuda_bf16.h>
 #include "quantize.cuh"
@@ -45,13 +45,13 @@ struct RotStructCfg {
   static constexpr int ACC2_COL = 2 * BN;              // D1 double-buffered in columns [0, 256); D2 in [256, 384)
   static constexpr int LO_COL = ACC2_COL + BN;         // third split term: 16 columns per token, [384, 448)
   static constexpr int TMEM_COLS = 512;
-  static constexpr int THREADS = 576;                  // producer, MMA issuer, 16 epilogue warps
+  static constexpr int THREADS = 608;                  // producer, step-2 issuer, 16 epilogue warps, step-3 issuer
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
 
 // tmRB: R_B [B, B] bf16, box [128 x 64], 128-byte swizzle.  tmX3: X as (k, token, block), box (32, 1, 64),
 // 64-byte swizzle.
-__global__ void __launch_bounds__(576, 1)
+__global__ void __launch_bounds__(608, 1)
 rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_constant__ CUtensorMap tmX3,
                          const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
                          uint8_t* __restrict__ scales, int M, int d, int* err_word) {
@@ -70,8 +70,9 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
   auto acc1e_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + 2 + a); };
   auto a2f_bar = [&](int tok) { return bar_base + 8u * (2 * C::STAGES + 4 + tok); };   // epilogue -> MMA
   auto a2d_bar = [&](int tok) { return bar_base + 8u * (2 * C::STAGES + 8 + tok); };   // MMA -> epilogue
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + bar_off + 192);
-  volatile int* cta_abort = reinterpret_cast<volatile int*>(smem_gen + bar_off + 200);
+  auto d1free_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + 12 + a); };   // step 3 of a tile done -> its D1 buffer
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + bar_off + 240);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(smem_gen + bar_off + 248);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nblocks = d / 32;                          // B
@@ -86,6 +87,7 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(acc1f_bar(a), 1); mbar_init(acc1e_bar(a), 16); }
     for (int t = 0; t < C::TOK; ++t) { mbar_init(a2f_bar(t), 4); mbar_init(a2d_bar(t), 1); }
+    for (int a = 0; a < 2; ++a) mbar_init(d1free_bar(a), 1);
     *cta_abort = 0;
     fence_mbar_init();
   }
@@ -121,16 +123,19 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer (both steps)
+    // ------------------------------------------------------------------ step-2 issuer
     constexpr uint32_t idesc1 = idesc_bf16(128, BN, /*A MN-major*/ false, /*B MN-major*/ true);
-    constexpr uint32_t idesc2 = idesc_bf16(128, 32, /*A MN-major*/ false, /*B MN-major*/ true);
-    const uint64_t rdesc = make_desc(ri_base, 2048, 512, kSwizzle64);
     uint32_t it = 0;
     bool ok = true;
     // step 2 of tile number `tc` (this CTA's count) into D1 buffer tc % 2
     auto step2 = [&](uint32_t tc) {
       const int a = tc & 1;
       if (!mbar_wait_warp(acc1e_bar(a), ((tc >> 1) & 1) ^ 1, cta_abort, err_word, SITE_MMA_ACC_EMPTY)) {
+        ok = false; return;
+      }
+      // with step 3, the split terms of the tile two back sit in this buffer until its step-3 MMAs
+      // (issued by another warp, so not ordered against these by the pipe) have completed
+      if (intra && !mbar_wait_warp(d1free_bar(a), ((tc >> 1) & 1) ^ 1, cta_abort, err_word, SITE_MMA_ACC_EMPTY)) {
         ok = false; return;
       }
       tc_fence_after_sync();
@@ -162,25 +167,33 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
       if (tile + (int)gridDim.x < total_tiles) step2(tcount + 1);    // next tile's step 2 runs beside this tile's step 3
       if (!ok) break;
-      if (intra) {
-        for (int tok = 0; tok < C::TOK && ok; ++tok) {
-          const int tq = tok;
-          if (!mbar_wait_warp(a2f_bar(tq), tcount & 1, cta_abort, err_word, SITE_MMA_FULL)) { ok = false; break; }
-          tc_fence_after_sync();
-          if (elect_one()) {
-            const uint32_t d2 = tmem_base + C::ACC2_COL + tq * 32;
-            const uint32_t d1 = tmem_base + (tcount & 1) * BN + tq * 32;      // hi, mid: over the token's y
-            const uint32_t lo = tmem_base + C::LO_COL + tq * 16;
-            mma_bf16_tmem_a(d2, d1, rdesc, idesc2, 0);
-            mma_bf16_tmem_a(d2, d1 + 8, rdesc + 64, idesc2, 1);              // k 16..31: +8 columns of A, +16 rows of R
-            mma_bf16_tmem_a(d2, d1 + 16, rdesc, idesc2, 1);
-            mma_bf16_tmem_a(d2, d1 + 24, rdesc + 64, idesc2, 1);
-            mma_bf16_tmem_a(d2, lo, rdesc, idesc2, 1);
-            mma_bf16_tmem_a(d2, lo + 8, rdesc + 64, idesc2, 1);
-            tc_commit(a2d_bar(tq));
-          }
-          __syncwarp();
+    }
+  } else if (warp == 18) {
+    // ------------------------------------------------------------------ step-3 issuer
+    // Its own warp: issuing step 2 of the next tile and step 3 of this one from one thread made that
+    // thread's loop the kernel's critical path.
+    constexpr uint32_t idesc2 = idesc_bf16(128, 32, /*A MN-major*/ false, /*B MN-major*/ true);
+    const uint64_t rdesc = make_desc(ri_base, 2048, 512, kSwizzle64);
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; intra && tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      for (int tok = 0; tok < C::TOK && ok; ++tok) {
+        if (!mbar_wait_warp(a2f_bar(tok), tcount & 1, cta_abort, err_word, SITE_MMA_FULL)) { ok = false; break; }
+        tc_fence_after_sync();
+        if (elect_one()) {
+          const uint32_t d2 = tmem_base + C::ACC2_COL + tok * 32;
+          const uint32_t d1 = tmem_base + (tcount & 1) * BN + tok * 32;       // hi, mid: over the token's y
+          const uint32_t lo = tmem_base + C::LO_COL + tok * 16;
+          mma_bf16_tmem_a(d2, d1, rdesc, idesc2, 0);
+          mma_bf16_tmem_a(d2, d1 + 8, rdesc + 64, idesc2, 1);                // k 16..31: +8 columns of A, +16 rows of R
+          mma_bf16_tmem_a(d2, d1 + 16, rdesc, idesc2, 1);
+          mma_bf16_tmem_a(d2, d1 + 24, rdesc + 64, idesc2, 1);
+          mma_bf16_tmem_a(d2, lo, rdesc, idesc2, 1);
+          mma_bf16_tmem_a(d2, lo + 8, rdesc + 64, idesc2, 1);
+          tc_commit(a2d_bar(tok));
+          if (tok == C::TOK - 1) tc_commit(d1free_bar(tcount & 1));
         }
+        __syncwarp();
       }
     }
   } else {
