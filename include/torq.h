@@ -77,8 +77,9 @@ torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void*
  * 2 d^2 flop per token.
  *   X [M, d] bf16;  R_B [d/32, d/32] bf16 (required);  R_intra [32, 32] bf16 or NULL = identity
  * Requires d % 256 == 0, 16-byte aligned pointers.  fp32 accumulation: step 2 on the tensor cores
- * with exact bf16 products, step 3 with y split into three bf16 terms (y to 2^-24) against the
- * bf16 R_intra on the warp-level tensor-core path. */
+ * with exact bf16 products, step 3 on the tensor cores as well, with y split exactly into three
+ * bf16 terms against the bf16 R_intra.  R_B is a constant of the layer like R_inter (see the
+ * conventions above). */
 torq_status torq_rotate_quantize_structured(const void* X, const void* R_B, const void* R_intra,
                                             int64_t M, int64_t d, void* out_codes, void* out_scales,
                                             void* stream);
@@ -206,6 +207,13 @@ torq_status torq_quantize_nvfp4(const void* Z, torq_dtype z_dtype, int64_t M, in
 torq_status torq_rotate_quantize_nvfp4(const void* X, const void* R_inter, const void* R_intra32,
                                        int64_t M, int64_t d, float tensor_scale, void* out_codes,
                                        void* out_scales, void* stream);
+
+/* torq_rotate_quantize_structured with the NVFP4 quantizer at its end: the rotation in the paper's own
+ * structure (R_B across blocks, one shared R_intra [32, 32] -- for a 16-wide intra rotation its two
+ * 16 x 16 blocks on the diagonal -- or NULL) and 16-element blocks with E4M3 scales.  d % 256 == 0. */
+torq_status torq_rotate_quantize_structured_nvfp4(const void* X, const void* R_B, const void* R_intra,
+                                                  int64_t M, int64_t d, float tensor_scale,
+                                                  void* out_codes, void* out_scales, void* stream);
 
 /* Algorithm 3 step 5 on NVFP4 operands: Y[m,n] = a_tensor_scale * w_tensor_scale *
  * sum_k (code * e4m3 scale)_a[m,k] (code * e4m3 scale)_w[n,k], fp32 accumulation on the tensor

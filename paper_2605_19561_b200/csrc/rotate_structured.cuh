@@ -25,7 +25,7 @@
 // memory as the A operand of step 3, wait for the token's six MMAs, read D2, quantize, store.
 #pragma once
 #include <cuda_bf16.h>
-#include "quantize.cuh"
+#include "nvfp4_quantize.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -51,10 +51,14 @@ struct RotStructCfg {
 
 // tmRB: R_B [B, B] bf16, box [128 x 64], 128-byte swizzle.  tmX3: X as (k, token, block), box (32, 1, 64),
 // 64-byte swizzle.
+// FMT_NVFP4: the NVFP4 quantizer at the end (two 16-element blocks per row of 32, E4M3 scales,
+// `tensor_scale` the tensor's float32 scale; unused for MXFP4); R_intra stays a 32 x 32 matrix (two
+// 16 x 16 blocks on its diagonal for a 16-wide intra rotation).
+template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(608, 1)
 rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_constant__ CUtensorMap tmX3,
                          const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
-                         uint8_t* __restrict__ scales, int M, int d, int* err_word) {
+                         uint8_t* __restrict__ scales, int M, int d, float tensor_scale, int* err_word) {
   using C = RotStructCfg;
   constexpr int BN = C::BN;
   extern __shared__ uint8_t smem_raw[];
@@ -273,10 +277,15 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
         for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(y[i]);
         uint4 cw;
         uint32_t sbyte;
-        quantize_block32(z, cw, sbyte);
+        if constexpr (FMT == FMT_NVFP4) nv_quantize_2x16(z, nv_scale(tensor_scale), cw, sbyte);
+        else quantize_block32(z, cw, sbyte);
         if (token < M && blk < nblocks) {
           *reinterpret_cast<uint4*>(codes + token * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
-          scales[scale_offset(token, blk, kb4)] = (uint8_t)sbyte;
+          if constexpr (FMT == FMT_NVFP4) {              // two scale bytes, adjacent in the tiled layout
+            *reinterpret_cast<uint16_t*>(scales + scale_offset(token, 2 * blk, (2 * nblocks + 3) / 4)) = (uint16_t)sbyte;
+          } else {
+            scales[scale_offset(token, blk, kb4)] = (uint8_t)sbyte;
+          }
         }
       }
     }

@@ -102,7 +102,8 @@ static DeviceState* device_state() {
               opt_in_smem(rotate_quantize_pair_kernel<FMT_MXFP4>, RotPairCfg::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_pair_kernel<FMT_NVFP4>, RotPairCfg::SMEM_BYTES) &&
               opt_in_smem(rotate_splitk_kernel, RotSplitCfg::SMEM_BYTES) &&
-              opt_in_smem(rotate_structured_kernel, RotStructCfg::SMEM_BYTES) &&
+              opt_in_smem(rotate_structured_kernel<FMT_MXFP4>, RotStructCfg::SMEM_BYTES) &&
+              opt_in_smem(rotate_structured_kernel<FMT_NVFP4>, RotStructCfg::SMEM_BYTES) &&
               opt_in_smem(mxfp4_gemm_pair_kernel<FMT_MXFP4>, GemmPairCfg::SMEM_BYTES) &&
               opt_in_smem(mxfp4_gemm_pair_kernel<FMT_NVFP4>, GemmPairCfgT<FMT_NVFP4>::SMEM_BYTES);
     if (!ok) return nullptr;
@@ -358,8 +359,9 @@ torq_status torq_rotate_quantize(const void* X, const void* R_inter, const void*
   return rotate_quantize_impl(X, R_inter, R_intra, M, d, out_codes, out_scales, nullptr, 0, stream);
 }
 
-torq_status torq_rotate_quantize_structured(const void* X, const void* R_B, const void* R_intra, int64_t M,
-                                            int64_t d, void* out_codes, void* out_scales, void* stream) {
+static torq_status rotate_structured_impl(const void* X, const void* R_B, const void* R_intra, int64_t M, int64_t d,
+                                          void* out_codes, void* out_scales, void* stream, int fmt,
+                                          float tensor_scale) {
   if (!X || !R_B || !out_codes || !out_scales) return TORQ_ERR_NULL;
   if (M < 1 || d < 256 || d % 256 != 0 || M > (1 << 30) || d > (1 << 24)) return TORQ_ERR_SHAPE;
   if (!aligned16(X) || !aligned16(R_B) || !aligned16(out_codes) || !aligned16(out_scales) ||
@@ -376,17 +378,35 @@ torq_status torq_rotate_quantize_structured(const void* X, const void* R_B, cons
     return TORQ_ERR_LAUNCH;
   const int64_t tiles = ((nb + 127) / 128) * ((M + RotStructCfg::TOK - 1) / RotStructCfg::TOK);
   const int grid = (int)(tiles < st->sm_count ? tiles : st->sm_count);
-  launch_tc(rotate_structured_kernel, 1, grid, RotStructCfg::THREADS, RotStructCfg::SMEM_BYTES, s, tmRB, tmX3,
-            static_cast<const __nv_bfloat16*>(R_intra), static_cast<uint8_t*>(out_codes),
-            static_cast<uint8_t*>(out_scales), (int)M, (int)d, st->err_word);
+  if (fmt == FMT_NVFP4)
+    launch_tc(rotate_structured_kernel<FMT_NVFP4>, 1, grid, RotStructCfg::THREADS, RotStructCfg::SMEM_BYTES, s, tmRB,
+              tmX3, static_cast<const __nv_bfloat16*>(R_intra), static_cast<uint8_t*>(out_codes),
+              static_cast<uint8_t*>(out_scales), (int)M, (int)d, tensor_scale, st->err_word);
+  else
+    launch_tc(rotate_structured_kernel<FMT_MXFP4>, 1, grid, RotStructCfg::THREADS, RotStructCfg::SMEM_BYTES, s, tmRB,
+              tmX3, static_cast<const __nv_bfloat16*>(R_intra), static_cast<uint8_t*>(out_codes),
+              static_cast<uint8_t*>(out_scales), (int)M, (int)d, 0.0f, st->err_word);
   if (launch_status() != TORQ_OK) return TORQ_ERR_LAUNCH;
-  const int64_t kc = (nb + 3) / 4 * 4, mpad = (M + 127) / 128 * 128;
-  const int64_t pad = (mpad - M) * kc + M * (kc - nb);
+  const int64_t ns = fmt == FMT_NVFP4 ? 2 * nb : nb;     // scale bytes per row
+  const int64_t kc = (ns + 3) / 4 * 4, mpad = (M + 127) / 128 * 128;
+  const int64_t pad = (mpad - M) * kc + M * (kc - ns);
   if (pad > 0) {
-    scale_padding_kernel<<<ew_grid(pad, 256, st->sm_count), 256, 0, s>>>(static_cast<uint8_t*>(out_scales), M, nb);
+    scale_padding_kernel<<<ew_grid(pad, 256, st->sm_count), 256, 0, s>>>(static_cast<uint8_t*>(out_scales), M, ns);
     return launch_status();
   }
   return TORQ_OK;
+}
+
+torq_status torq_rotate_quantize_structured(const void* X, const void* R_B, const void* R_intra, int64_t M,
+                                            int64_t d, void* out_codes, void* out_scales, void* stream) {
+  return rotate_structured_impl(X, R_B, R_intra, M, d, out_codes, out_scales, stream, FMT_MXFP4, 0.0f);
+}
+
+torq_status torq_rotate_quantize_structured_nvfp4(const void* X, const void* R_B, const void* R_intra, int64_t M,
+                                                  int64_t d, float tensor_scale, void* out_codes, void* out_scales,
+                                                  void* stream) {
+  if (!(tensor_scale > 0.0f && tensor_scale <= 3.0e38f)) return TORQ_ERR_SHAPE;
+  return rotate_structured_impl(X, R_B, R_intra, M, d, out_codes, out_scales, stream, FMT_NVFP4, tensor_scale);
 }
 
 }  // extern "C"

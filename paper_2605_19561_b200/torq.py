@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
     L.torq_quantize_nvfp4.restype = ci
     L.torq_rotate_quantize_nvfp4.argtypes = [vp, vp, vp, i64, i64, f32, vp, vp, vp]
     L.torq_rotate_quantize_nvfp4.restype = ci
+    L.torq_rotate_quantize_structured_nvfp4.argtypes = [vp, vp, vp, i64, i64, f32, vp, vp, vp]
+    L.torq_rotate_quantize_structured_nvfp4.restype = ci
     L.torq_nvfp4_gemm.argtypes = [vp, vp, f32, vp, vp, f32, i64, i64, i64, vp, ci, vp]
     L.torq_nvfp4_gemm.restype = ci
     L.torq_rotated_linear_nvfp4.argtypes = [vp, vp, vp, f32, vp, vp, f32, i64, i64, i64, vp, ci, vp, sz, vp, vp, vp]
@@ -419,3 +421,19 @@ def torq_givens_equalize(Sigma, eps: float, stream=None):
     _raise(lib().torq_givens_equalize(_ptr(Sigma), B, float(eps), _ptr(Q), _ptr(Qb), _ptr(n), _stream(stream)),
            "torq_givens_equalize")
     return Q, Qb, n[:1]
+
+
+def torq_rotate_quantize_structured_nvfp4(X, R_B, R_intra, tensor_scale: float, out_codes=None, out_scales=None,
+                                          stream=None):
+    """The structured rotation (R_B [d/32,d/32], shared R_intra [32,32] or None) followed by the NVFP4 quantizer."""
+    M, d = X.shape
+    for t, n in ((X, "X"), (R_B, "R_B"), (R_intra, "R_intra")):
+        _check(t, torch.bfloat16, n)
+    if out_codes is None:
+        out_codes = torch.empty((M, d // 2), dtype=torch.uint8, device=X.device)
+    if out_scales is None:
+        out_scales = torch.empty(torq_nvfp4_scales_bytes(M, d), dtype=torch.uint8, device=X.device)
+    _raise(lib().torq_rotate_quantize_structured_nvfp4(_ptr(X), _ptr(R_B), _ptr(R_intra), M, d, tensor_scale,
+                                                       _ptr(out_codes), _ptr(out_scales), _stream(stream)),
+           "torq_rotate_quantize_structured_nvfp4")
+    return out_codes, out_scales

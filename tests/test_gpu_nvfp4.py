@@ -361,3 +361,29 @@ def test_weight_preparation_on_device_matches_the_oracle():
     dg = O.dequantize_nvfp4(g_codes, g_sb, ts)
     do = O.dequantize_nvfp4(o_codes, o_sb, o_ts)
     assert np.linalg.norm(dg - do) / np.linalg.norm(do) < 2e-3        # fp32 vs fp64 product, a few flipped codes
+
+
+@pytest.mark.parametrize("M,d", [(64, 256), (130, 512), (2048, 4096)])
+def test_structured_rotation_with_the_nvfp4_quantizer(M, d):
+    """The rotation in the paper's own structure (one matrix across blocks, one shared matrix inside them,
+    here two 16 x 16 blocks on the diagonal of a 32 x 32) followed by the NVFP4 quantizer."""
+    cfg = I.CONFIGS["tiny"]
+    xb = I.activations(cfg, M=M, d=d)
+    g = np.random.Generator(np.random.PCG64(I.BASE_SEED + 77))
+    rbb = I.to_bf16_bits(I.orthogonal(d // 32, g))
+    ri32 = O.expand_intra16(I.intra_rotations16(cfg, d=32))[0]           # [32, 32] bit patterns
+    rows = np.arange(M) if M <= 256 else np.array([0, 1, 3, 4, 127, 128, 1000, 2046, 2047])
+    z = O.rotate_structured(xb[rows], rbb, ri32)
+    ts = np.float32(np.abs(z).max() / (6 * 448) * (1 if M <= 256 else 2))
+    codes_t, scales_t = torq.torq_rotate_quantize_structured_nvfp4(dev_bf16(xb), dev_bf16(rbb), dev_bf16(ri32), float(ts))
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    g_codes, g_sb = _to_numpy(codes_t, scales_t, M, d)
+    o_codes, o_sb = O.quantize_nvfp4(z.astype(np.float32), ts)
+    rep = _mismatch(g_codes[rows], g_sb[rows], o_codes, o_sb, ts)
+    assert rep["non_adjacent"] == 0 and rep["scale_off_by_more_than_one"] == 0, rep
+    assert rep["elem"] <= 2e-4 and rep["blocks"] <= 2e-4, rep
+    buf = scales_t.cpu().numpy().copy()                                  # padding of the scale tiles is zero
+    rr, cc = np.meshgrid(np.arange(M), np.arange(d // 16), indexing="ij")
+    buf[O.nv_scale_layout_offset(rr, cc, d)] = 0
+    assert not buf.any()
