@@ -100,6 +100,10 @@ __device__ __forceinline__ bool elect_one() {
 }
 
 // ---- proxies / fences -------------------------------------------------------------------------
+// Orders this thread's generic-proxy accesses (all state spaces) against its later async-proxy ones.
+__device__ __forceinline__ void fence_proxy_async_all() {
+  asm volatile("fence.proxy.async;" ::: "memory");
+}
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
