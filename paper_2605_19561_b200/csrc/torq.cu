@@ -607,8 +607,14 @@ static torq_status fused_layer(const void* X, const void* R_inter, const void* R
       !aligned16(Y))
     return TORQ_OK;                                      // let the two-kernel path report it
   const int64_t rot_tiles = mp_tiles * ((d + 255) / 256), gemm_tiles = mp_tiles * ((N + 255) / 256);
-  // worth it only when a pair that runs out of rotation tiles finds GEMM tiles to do
-  if (rot_tiles % st->fused_pairs == 0 && gemm_tiles % st->fused_pairs == 0) return TORQ_OK;
+  // Worth it only from three rotation waves on.  The epilogue of a rotation tile that is not its
+  // pair's last runs beside the next mainloop and takes most of it, so a row tile is complete about
+  // one tile time after its last mainloop: with two waves (2048 x 4096: measured 77 us against 72.5 us
+  // for the two kernels) the pairs that skip the second wave would still find no finished row.
+  if (rot_tiles < 3 * (int64_t)st->fused_pairs) return TORQ_OK;
+  // ... and while the GEMM is not the bulk of the work: its tiles are dealt out row tile by row tile
+  // here, which re-streams W for every row tile (8192 x 5120 -> 25600: 759 us against 689 us).
+  if (N > 2 * d) return TORQ_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   CUtensorMap tmX, tmR, tmA, tmB, tmSFA, tmSFB, tmY;
   const uint64_t kb4 = (uint64_t)(d / 128);

@@ -183,3 +183,38 @@ def test_ragged_shapes_on_the_cta_pair_rotation(M, d):
     rb, rib, _, _ = I.rotations(cfg, d=d)
     _rotate_quantize_case(xb, rb, rib)
     _rotate_quantize_case(xb, rb, None)
+
+
+@pytest.mark.parametrize("M,out_dtype", [(3072, torch.bfloat16), (3001, torch.float32)])
+def test_one_kernel_layer_agrees_with_the_two_kernels(M, out_dtype):
+    """From three rotation waves on (and N <= 2 d) the fused call runs rotation and GEMM as one persistent
+    kernel whose GEMM tiles wait on per-row-tile counters.  Same tiles, same arithmetic: its codes, scales and
+    output must agree with the two separate calls (the tile that takes the warp-MMA form of the intra step
+    differs between the two, so codes may differ where the oracle tests allow it: <= 1e-4, adjacent)."""
+    cfg = I.CONFIGS["qwen3_32b_sweep"]
+    d, N = cfg.d, 5120
+    xb = I.activations(cfg, M=M)
+    rb, rib, _, _ = I.rotations(cfg, device="cuda")
+    X, R, Ri = dev_bf16(xb), dev_bf16(rb), dev_bf16(rib)
+    g = np.random.default_rng(12)
+    Wq = dev_u8(g.integers(0, 256, (N, d // 2), dtype=np.uint8))
+    Ws = dev_u8(O.swizzle_scales(g.integers(120, 131, (N, d // 32), dtype=np.uint8), d, fill=0))
+    dbg_c = torch.empty((M, d // 2), dtype=torch.uint8, device="cuda")
+    dbg_s = torch.empty(torq.torq_scales_bytes(M, d), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    before = torq.torq_launch_count()
+    y1 = torq.torq_rotated_linear(X, R, Ri, Wq, Ws, out_dtype=out_dtype, dbg_codes=dbg_c, dbg_scales=dbg_s)
+    torch.cuda.synchronize()
+    assert torq.torq_launch_count() - before == 1
+    assert torq.torq_last_device_error() == 0
+    c2, s2 = torq.torq_rotate_quantize(X, R, Ri)
+    y2 = torq.torq_mxfp4_gemm(dbg_c, dbg_s, Wq, Ws, out_dtype=out_dtype)      # the GEMM alone on the fused call's codes
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y2)                            # same tiles, same instruction order per tile
+    assert torch.equal(dbg_s, s2) or float((dbg_s != s2).float().mean()) <= 1e-4
+    diff = (dbg_c != c2)
+    assert float(diff.float().mean()) <= 1e-4
+    # twice in a row on the same workspace-free call: the counters start from zero each time
+    y3 = torq.torq_rotated_linear(X, R, Ri, Wq, Ws, out_dtype=out_dtype)
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y3)
