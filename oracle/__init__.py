@@ -6,3 +6,4 @@ the benchmark's cpu_baseline / reference legs do.
 from .torq_oracle import *  # noqa: F401,F403
 from .nvfp4_oracle import *  # noqa: F401,F403,E402
 from .givens_oracle import *  # noqa: F401,F403,E402
+from .mxint4_oracle import *  # noqa: F401,F403,E402
