@@ -236,6 +236,49 @@ torq_status torq_rotated_linear_nvfp4(const void* X, const void* R_inter, const 
                                       torq_dtype y_dtype, void* workspace, size_t workspace_bytes,
                                       void* dbg_codes, void* dbg_scales, void* stream);
 
+/* ---- MXINT4 variant (the paper's format study, Section 6 "Generalizability to Other Formats") ----
+ * The same layer with integer elements: blocks of 32 along K, one E8M0 scale byte per block by
+ * the same rule and in the same tiled layout as MXFP4 (torq_scales_bytes / torq_scale_offset),
+ * elements q = clamp(rint(z / 2^e), -7, 7) (rint = round half to even; z / 2^e is exact, so the
+ * quantizer is bit-exact by definition); decoding x^ = q * 2^e.
+ * Two forms of the codes:
+ *   stored form   [rows, k/2] bytes: two's-complement nibbles, even element in the low nibble;
+ *   operand form  [rows, k]   bytes: the FP8 E4M3 byte whose value is q (a zero may carry a sign
+ *                 bit).  The tensor cores of this GPU have no 4-bit integer path; the GEMM runs
+ *                 as tcgen05.mma kind::mxf8f6f4 on E4M3 operands with the E8M0 block scales.
+ *                 Integer products and their power-of-two scales are exact in it; accumulation
+ *                 is fp32.
+ * The rotation entry points write the operand form directly.  All pointers device, 16-byte
+ * aligned; errors as elsewhere in this header.  The paper has no worked example of this format. */
+size_t torq_mxint4_workspace_bytes(int64_t M, int64_t d, int64_t N);
+
+/* Quantize Z [M, d] (fp32 or bf16), d % 32 == 0.  packed != 0: stored form, out_codes [M, d/2];
+ * packed == 0: operand form, out_codes [M, d].  out_scales: torq_scales_bytes(M, d) bytes. */
+torq_status torq_quantize_mxint4(const void* Z, torq_dtype z_dtype, int64_t M, int64_t d, int packed,
+                                 void* out_codes, void* out_scales, void* stream);
+
+/* Stored form [rows, k/2] -> operand form [rows, k] (nibble -8 becomes the E4M3 byte of -8). */
+torq_status torq_mxint4_expand(const void* packed, int64_t rows, int64_t k, void* out_bytes, void* stream);
+
+/* Algorithm 3 steps 1-4 with the MXINT4 quantizer.  X [M, d] bf16; R_inter [d, d] bf16 (required);
+ * R_intra [d/32, 32, 32] bf16 or NULL = identity; d % 32 == 0.  out_bytes [M, d] operand form. */
+torq_status torq_rotate_quantize_mxint4(const void* X, const void* R_inter, const void* R_intra, int64_t M,
+                                        int64_t d, void* out_bytes, void* out_scales, void* stream);
+
+/* Algorithm 3 step 5 on MXINT4 operands: Y[m,n] = sum_k a^[m,k] w^[n,k].  A8 [M, K], W8 [N, K]
+ * operand form; As, Ws tiled E8M0 scales; K % 128 == 0, N % 8 == 0; Y [M, N] fp32 or bf16. */
+torq_status torq_mxint4_gemm(const void* A8, const void* As, const void* W8, const void* Ws, int64_t M,
+                             int64_t N, int64_t K, void* Y, torq_dtype y_dtype, void* stream);
+
+/* Steps 1-5 in MXINT4: torq_rotate_quantize_mxint4 into `workspace` (at least
+ * torq_mxint4_workspace_bytes(M, d, N) bytes, 256-byte aligned), then torq_mxint4_gemm.  dbg_bytes
+ * [M, d] / dbg_scales, when not NULL, receive copies of the quantized activations.
+ * d % 128 == 0, N % 8 == 0. */
+torq_status torq_rotated_linear_mxint4(const void* X, const void* R_inter, const void* R_intra, const void* W8,
+                                       const void* Ws, int64_t M, int64_t d, int64_t N, void* Y,
+                                       torq_dtype y_dtype, void* workspace, size_t workspace_bytes,
+                                       void* dbg_bytes, void* dbg_scales, void* stream);
+
 /* ---- calibration of the inter-block rotation (Section 5.1; offline, not on the inference path) ----
  * Covariance across the blocks of a token, pooled over the T calibration tokens and the 32
  * positions of a block (block means taken as zero, as Section 5.1 assumes):

@@ -14,6 +14,10 @@
 // elements of K, the product of the two tensor scales applied in the epilogue).  Scale bytes come
 // in 512-byte chunks of 128 rows x 4 bytes; one chunk covers 128 elements of K in MXFP4 and 64 in
 // NVFP4, so a stage holds CH = 2 or 4 chunks per 128 rows, four tensor-memory columns each.
+//
+// FMT_MXINT4: the integer codes arrive as E4M3 operand bytes, one per element (kind::mxf8f6f4, E8M0
+// scale per 32 elements of K).  A stage is still 128 bytes of K per row, now 128 elements: one
+// scale chunk, four instructions of K = 32 that take bytes 0..3 of the chunk's 4-byte cells.
 #pragma once
 #include <cuda_bf16.h>
 #include "sm100_ptx.cuh"
@@ -23,13 +27,13 @@ namespace torq {
 template <int BN, int NACC, int FMT = FMT_MXFP4>
 struct GemmCfg {
   static constexpr int BM = 128;
-  static constexpr int BK = 256;                       // elements of K per stage
-  static constexpr int A_BYTES = BM * BK / 2;          // 16 KiB
-  static constexpr int B_BYTES = BN * BK / 2;
-  static constexpr int CH = FMT == FMT_NVFP4 ? 4 : 2;  // scale chunks per stage and 128 rows
+  static constexpr int BK = FMT == FMT_MXINT4 ? 128 : 256;   // elements of K per stage (128 bytes per row)
+  static constexpr int A_BYTES = BM * 128;             // 16 KiB
+  static constexpr int B_BYTES = BN * 128;
+  static constexpr int CH = FMT == FMT_NVFP4 ? 4 : (FMT == FMT_MXINT4 ? 1 : 2);   // scale chunks per stage and 128 rows
   static constexpr int SFA_BYTES = CH * 512;
   static constexpr int SFB_BYTES = (BN / 128) * SFA_BYTES;
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
+  static constexpr int STAGE_BYTES = (A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES + 1023) / 1024 * 1024;   // swizzle atoms need 1 KiB
   static constexpr int STAGES = (BN == 256) ? 4 : 6;
   static constexpr int BAR_BYTES = 256;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + align slack
@@ -68,7 +72,7 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int n_tiles = (N + BN - 1) / BN;
   const int total_tiles = m_tiles * n_tiles;
   const int k_tiles = (K + C::BK - 1) / C::BK;          // K % 128 == 0: last stage may be half
-  const int kb4 = K / (256 / CH);                       // scale chunks (4 K-blocks each) per row
+  const int kb4 = K / (C::BK / CH);                     // scale chunks (4 K-blocks each) per row
   const int n_rowtiles = (N + 127) / 128;
 
   if (threadIdx.x == 0) {
@@ -177,7 +181,12 @@ mxfp4_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 tmem_cp_32x128b_warpx4(sfb_t + c * (BN / 32) + 4 * t, sfb_d + (C::SFA_BYTES / 16) * t + 32 * c);
             }
           }
-          if constexpr (FMT == FMT_NVFP4) {                // one chunk per instruction
+          if constexpr (FMT == FMT_MXINT4) {               // a quarter chunk (one scale byte) per instruction
+            mma_mxf8(acc, adesc, bdesc, idesc_mxf8(128, BN, 0), sfa_t, sfb_t, kt != 0);
+            mma_mxf8(acc, adesc + 2, bdesc + 2, idesc_mxf8(128, BN, 1), sfa_t, sfb_t, 1);
+            mma_mxf8(acc, adesc + 4, bdesc + 4, idesc_mxf8(128, BN, 2), sfa_t, sfb_t, 1);
+            mma_mxf8(acc, adesc + 6, bdesc + 6, idesc_mxf8(128, BN, 3), sfa_t, sfb_t, 1);
+          } else if constexpr (FMT == FMT_NVFP4) {         // one chunk per instruction
 #pragma unroll
             for (int j = 0; j < 4; ++j)
               if (j < 2 || two)

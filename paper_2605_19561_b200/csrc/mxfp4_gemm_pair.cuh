@@ -19,6 +19,10 @@
 // FMT_NVFP4 runs the same pipeline with kind::mxf4nvf4 (one E4M3 scale per 16 elements of K:
 // four 512-byte scale chunks per stage and 128 rows instead of two) and multiplies the result by
 // the product of the two tensor scales in the epilogue.
+//
+// FMT_MXINT4: integer codes as E4M3 operand bytes (kind::mxf8f6f4, E8M0 scale per 32 elements of K):
+// a stage is 128 elements of K, one scale chunk, four instructions of K = 32 taking bytes 0..3 of
+// the chunk's 4-byte cells.
 #pragma once
 #include <cuda_bf16.h>
 #include "sm100_ptx.cuh"
@@ -29,13 +33,16 @@ template <int FMT = FMT_MXFP4>
 struct GemmPairCfgT {
   static constexpr int BN = 256;
   static constexpr int BM = 128;                       // rows per CTA
-  static constexpr int BK = 256;
-  static constexpr int A_BYTES = BM * BK / 2;          // 16 KiB
-  static constexpr int B_BYTES = (BN / 2) * BK / 2;    // 16 KiB
-  static constexpr int CH = FMT == FMT_NVFP4 ? 4 : 2;  // scale chunks per stage and 128 rows
+  static constexpr int BK = FMT == FMT_MXINT4 ? 128 : 256;   // elements of K per stage (128 bytes per row)
+  static constexpr int A_BYTES = BM * 128;             // 16 KiB
+  static constexpr int B_BYTES = (BN / 2) * 128;       // 16 KiB
+  static constexpr int CH = FMT == FMT_NVFP4 ? 4 : (FMT == FMT_MXINT4 ? 1 : 2);   // scale chunks per stage and 128 rows
+  static constexpr int SF_BOXES = CH == 1 ? 1 : CH / 2;       // scale loads per stage and 128 rows:
+  static constexpr int SF_BOX_WORDS = CH == 1 ? 128 : 256;    // 1 KiB (two chunks), or the single chunk
   static constexpr int SFA_BYTES = CH * 512;
   static constexpr int SFB_BYTES = 2 * SFA_BYTES;      // both 128-row tiles of the W scales
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;   // 35 / 38 KiB
+  static constexpr int STAGE_TX = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;      // bytes one CTA loads per stage
+  static constexpr int STAGE_BYTES = (STAGE_TX + 1023) / 1024 * 1024;             // 35 / 38 / 34 KiB (swizzle atoms need 1 KiB)
   static constexpr int STAGES = 5;
   static constexpr int OUT_WARP_BYTES = 32 * 128;      // per epilogue warp: 32 rows x 128 B, swizzled
   static constexpr int OUT_BYTES = 8 * OUT_WARP_BYTES;
@@ -77,7 +84,7 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   const int n_tiles = (N + BN - 1) / BN;
   const int total_tiles = mp_tiles * n_tiles;
   const int k_tiles = (K + C::BK - 1) / C::BK;
-  const int kb4 = K / (256 / CH);                      // scale chunks per row
+  const int kb4 = K / (C::BK / CH);                    // scale chunks per row
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -108,14 +115,14 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       for (int kt = 0; kt < pre; ++kt) {
         const uint32_t st = smem_base + kt * C::STAGE_BYTES;
         const uint32_t leader_full = map_to_cta(full_bar(kt), 0);
-        if (rank == 0) mbar_arrive_expect_tx(full_bar(kt), 2 * C::STAGE_BYTES);
+        if (rank == 0) mbar_arrive_expect_tx(full_bar(kt), 2 * C::STAGE_TX);
         tma_load_2d_pair(st + C::A_BYTES, &tmB, kt * 128, nt * BN + (int)rank * (BN / 2), leader_full);
 #pragma unroll
         for (int t = 0; t < 2; ++t)                      // one 1 KiB box = two chunks
 #pragma unroll
-          for (int b = 0; b < CH / 2; ++b)
+          for (int b = 0; b < C::SF_BOXES; ++b)
             tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * C::SFA_BYTES + b * 1024, &tmSFB,
-                             (kt * (CH / 2) + b) * 256, 2 * nt + t, leader_full);
+                             kt * CH * 128 + b * 256, 2 * nt + t, leader_full);
       }
     }
     __syncwarp();
@@ -138,7 +145,7 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         const uint32_t leader_full = map_to_cta(full_bar(s), 0);
         if (elect_one()) {
           const bool w_issued = it < (uint32_t)pre;      // W side of this stage went out before the wait above
-          if (rank == 0 && !w_issued) mbar_arrive_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
+          if (rank == 0 && !w_issued) mbar_arrive_expect_tx(full_bar(s), 2 * C::STAGE_TX);
           tma_load_2d_pair(st, &tmA, kt * 128, mt * C::BM, leader_full);
           if (!w_issued)
             tma_load_2d_pair(st + C::A_BYTES, &tmB, kt * 128, nt * BN + (int)rank * (BN / 2), leader_full);
@@ -146,16 +153,16 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           // 1 KiB (two chunks); anything outside the buffer arrives as zeros (scale 2^-127 or 0,
           // multiplying operand data that is zero there as well).
 #pragma unroll
-          for (int b = 0; b < CH / 2; ++b)
-            tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + b * 1024, &tmSFA, (kt * (CH / 2) + b) * 256, mt,
+          for (int b = 0; b < C::SF_BOXES; ++b)
+            tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + b * 1024, &tmSFA, kt * CH * 128 + b * 256, mt,
                              leader_full);
           if (!w_issued) {
 #pragma unroll
             for (int t = 0; t < 2; ++t)
 #pragma unroll
-              for (int b = 0; b < CH / 2; ++b)
+              for (int b = 0; b < C::SF_BOXES; ++b)
                 tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * C::SFA_BYTES + b * 1024, &tmSFB,
-                                 (kt * (CH / 2) + b) * 256, 2 * nt + t, leader_full);
+                                 kt * CH * 128 + b * 256, 2 * nt + t, leader_full);
           }
         }
         __syncwarp();
@@ -197,7 +204,12 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                 tmem_cp_32x128b_warpx4_pair(sfb_t + 8 * c + 4, sfb_d + 32 * c + C::SFA_BYTES / 16);
               }
             }
-            if constexpr (FMT == FMT_NVFP4) {              // one chunk per instruction
+            if constexpr (FMT == FMT_MXINT4) {             // a quarter chunk (one scale byte) per instruction
+              mma_mxf8_pair(tmem_base, adesc, bdesc, idesc_mxf8(256, BN, 0), sfa_t, sfb_t, kt != 0);
+              mma_mxf8_pair(tmem_base, adesc + 2, bdesc + 2, idesc_mxf8(256, BN, 1), sfa_t, sfb_t, 1);
+              mma_mxf8_pair(tmem_base, adesc + 4, bdesc + 4, idesc_mxf8(256, BN, 2), sfa_t, sfb_t, 1);
+              mma_mxf8_pair(tmem_base, adesc + 6, bdesc + 6, idesc_mxf8(256, BN, 3), sfa_t, sfb_t, 1);
+            } else if constexpr (FMT == FMT_NVFP4) {       // one chunk per instruction
 #pragma unroll
               for (int j = 0; j < 4; ++j)
                 if (j < 2 || two)

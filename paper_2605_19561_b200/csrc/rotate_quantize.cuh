@@ -15,6 +15,7 @@
 #pragma once
 #include <cuda_bf16.h>
 #include "nvfp4_quantize.cuh"
+#include "mxint4_quantize.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -38,7 +39,8 @@ struct RotCfg {
 };
 
 // FMT_NVFP4: NVFP4 quantizer in the epilogue (two 16-element blocks per 32 columns, E4M3 scales,
-// `tensor_scale` the tensor's float32 scale; unused for MXFP4).
+// `tensor_scale` the tensor's float32 scale; unused for MXFP4).  FMT_MXINT4: integer codes as one
+// E4M3 operand byte per element (`codes` is [M, d] bytes), scale bytes as for MXFP4.
 template <int BN, int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(192, 1)
 rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
@@ -210,11 +212,21 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
         }
         uint4 cw;
         uint32_t sbyte;
-        if constexpr (FMT == FMT_NVFP4) nv_quantize_2x16(z, nvs, cw, sbyte);
-        else quantize_block32(z, cw, sbyte);
         const int blk = b0 + bb;
-        if (row < M && blk < nblocks)
-          *reinterpret_cast<uint4*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+        if constexpr (FMT == FMT_MXINT4) {                 // one operand byte per element
+          uint4 cw2;
+          mxint4_quantize_block32(z, cw, cw2, sbyte);
+          if (row < M && blk < nblocks) {
+            uint4* dst = reinterpret_cast<uint4*>(codes + row * (int64_t)d + (int64_t)blk * 32);
+            dst[0] = cw;
+            dst[1] = cw2;
+          }
+        } else {
+          if constexpr (FMT == FMT_NVFP4) nv_quantize_2x16(z, nvs, cw, sbyte);
+          else quantize_block32(z, cw, sbyte);
+          if (row < M && blk < nblocks)
+            *reinterpret_cast<uint4*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+        }
         if constexpr (FMT == FMT_NVFP4) {                  // two 16-blocks = half a 4-byte group
           sc_word |= sbyte << (16 * (bb & 1));
           if (bb & 1) {

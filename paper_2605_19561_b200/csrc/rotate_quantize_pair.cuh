@@ -14,6 +14,7 @@
 #pragma once
 #include <cuda_bf16.h>
 #include "nvfp4_quantize.cuh"
+#include "mxint4_quantize.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -40,6 +41,8 @@ struct RotPairCfg {
 // FMT_NVFP4: the same kernel with the NVFP4 quantizer in the epilogue (two 16-element blocks per
 // 32 columns, E4M3 scales, `tensor_scale` the tensor's float32 scale; unused for MXFP4).  R_intra
 // is still [d/32, 32, 32]; 16-wide rotations arrive as its block-diagonal form.
+// FMT_MXINT4: integer codes written as one E4M3 operand byte per element (`codes` is [M, d] bytes),
+// the scale bytes as for MXFP4.
 template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(320, 1)
 rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
@@ -251,11 +254,21 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
           }
           uint4 cw;
           uint32_t sbyte;
-          if constexpr (FMT == FMT_NVFP4) nv_quantize_2x16(z, nvs, cw, sbyte);
-          else quantize_block32(z, cw, sbyte);
           const int blk = b0 + h * 4 + bb;
-          if (row < M && blk < nblocks)
-            *reinterpret_cast<uint4*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+          if constexpr (FMT == FMT_MXINT4) {               // one operand byte per element
+            uint4 cw2;
+            mxint4_quantize_block32(z, cw, cw2, sbyte);
+            if (row < M && blk < nblocks) {
+              uint4* dst = reinterpret_cast<uint4*>(codes + row * (int64_t)d + (int64_t)blk * 32);
+              dst[0] = cw;
+              dst[1] = cw2;
+            }
+          } else {
+            if constexpr (FMT == FMT_NVFP4) nv_quantize_2x16(z, nvs, cw, sbyte);
+            else quantize_block32(z, cw, sbyte);
+            if (row < M && blk < nblocks)
+              *reinterpret_cast<uint4*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+          }
           if constexpr (FMT == FMT_NVFP4) {
             if (blk >= nblocks) sbyte = 0;               // padding blocks decode to zero
             if (bb < 2) sc_word |= sbyte << (16 * bb);
@@ -342,11 +355,21 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
             const float v[8] = {acc[0][2 * rh], acc[0][2 * rh + 1], acc[1][2 * rh], acc[1][2 * rh + 1],
                                 acc[2][2 * rh], acc[2][2 * rh + 1], acc[3][2 * rh], acc[3][2 * rh + 1]};
             uint32_t word, sbyte;
-            if constexpr (FMT == FMT_NVFP4) nv_quantize_row_fragment(v, p, nvs, word, sbyte);
-            else quantize_row_fragment(v, p, word, sbyte);
             const int64_t row = row_base + 16 * mh + 8 * rh;
-            if (row < M && blk < nblocks)
-              *reinterpret_cast<uint32_t*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16 + 4 * p) = word;
+            if constexpr (FMT == FMT_MXINT4) {             // two operand bytes per 8 columns and lane
+              uint32_t pr[4];
+              mxint4_quantize_row_fragment(v, pr, sbyte);
+              if (row < M && blk < nblocks) {
+                uint8_t* dst = codes + row * (int64_t)d + (int64_t)blk * 32 + 2 * p;
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) *reinterpret_cast<uint16_t*>(dst + 8 * nt) = (uint16_t)pr[nt];
+              }
+            } else {
+              if constexpr (FMT == FMT_NVFP4) nv_quantize_row_fragment(v, p, nvs, word, sbyte);
+              else quantize_row_fragment(v, p, word, sbyte);
+              if (row < M && blk < nblocks)
+                *reinterpret_cast<uint32_t*>(codes + row * (int64_t)(d / 2) + (int64_t)blk * 16 + 4 * p) = word;
+            }
             if constexpr (FMT == FMT_NVFP4) {
               if (blk >= nblocks) sbyte = 0;
               if (bb < 2) sc_word[2 * mh + rh] |= sbyte << (16 * bb);

@@ -10,6 +10,7 @@
 #include "mxfp4_gemm_pair.cuh"
 #include "quantize.cuh"
 #include "nvfp4_quantize.cuh"
+#include "mxint4_quantize.cuh"
 #include "rotate_quantize.cuh"
 #include "rotate_quantize_pair.cuh"
 #include "rotate_splitk.cuh"
@@ -107,7 +108,12 @@ static DeviceState* device_state() {
               opt_in_smem(rotate_structured_kernel<FMT_MXFP4>, RotStructCfg::SMEM_BYTES) &&
               opt_in_smem(rotate_structured_kernel<FMT_NVFP4>, RotStructCfg::SMEM_BYTES) &&
               opt_in_smem(mxfp4_gemm_pair_kernel<FMT_MXFP4>, GemmPairCfg::SMEM_BYTES) &&
-              opt_in_smem(mxfp4_gemm_pair_kernel<FMT_NVFP4>, GemmPairCfgT<FMT_NVFP4>::SMEM_BYTES);
+              opt_in_smem(mxfp4_gemm_pair_kernel<FMT_NVFP4>, GemmPairCfgT<FMT_NVFP4>::SMEM_BYTES) &&
+              opt_in_smem(mxfp4_gemm_kernel<256, 1, FMT_MXINT4>, GemmCfg<256, 1, FMT_MXINT4>::SMEM_BYTES) &&
+              opt_in_smem(mxfp4_gemm_kernel<128, 2, FMT_MXINT4>, GemmCfg<128, 2, FMT_MXINT4>::SMEM_BYTES) &&
+              opt_in_smem(mxfp4_gemm_pair_kernel<FMT_MXINT4>, GemmPairCfgT<FMT_MXINT4>::SMEM_BYTES) &&
+              opt_in_smem(rotate_quantize_kernel<256, FMT_MXINT4>, RotCfg<256>::SMEM_BYTES) &&
+              opt_in_smem(rotate_quantize_pair_kernel<FMT_MXINT4>, RotPairCfg::SMEM_BYTES);
     if (!ok) return nullptr;
     st.rot_pairs = max_active_pairs(rotate_quantize_pair_kernel<FMT_MXFP4>, RotPairCfg::THREADS,
                                     RotPairCfg::SMEM_BYTES, st.sm_count);
@@ -289,7 +295,7 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
                                         size_t scratch_bytes, void* stream, int fmt = FMT_MXFP4,
                                         float tensor_scale = 0.0f) {
   if (!X || !out_codes || !out_scales) return TORQ_ERR_NULL;
-  if (fmt == FMT_NVFP4 && !R_inter) return TORQ_ERR_NULL;
+  if (fmt != FMT_MXFP4 && !R_inter) return TORQ_ERR_NULL;
   if (M < 1 || d < 32 || d % 32 != 0 || M > (1 << 30) || d > (1 << 24)) return TORQ_ERR_SHAPE;
   if (!aligned16(X) || !aligned16(out_codes) || !aligned16(out_scales) ||
       (R_inter && !aligned16(R_inter)) || (R_intra && !aligned16(R_intra)))
@@ -312,7 +318,7 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
   if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d, 128, 64) ||
       !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
     return TORQ_ERR_LAUNCH;
-  const int splits = rotation_splits(M, d, st->sm_count);
+  const int splits = fmt == FMT_MXINT4 ? 1 : rotation_splits(M, d, st->sm_count);   // MXINT4: single pass only
   if (splits >= 2 && scratch && scratch_bytes >= splitk_scratch_bytes(M, d, splits) &&
       (reinterpret_cast<uintptr_t>(scratch) & 15u) == 0) {
     // Few tokens: split K over the SMs, partial tiles to scratch, then reduce + intra + quantize.
@@ -340,7 +346,11 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
     const int ptiles = (int)((M + 255) / 256) * (int)((d + 255) / 256);
     const int max_pairs = st->rot_pairs;
     const int pairs = ptiles < max_pairs ? ptiles : max_pairs;
-    if (fmt == FMT_NVFP4)
+    if (fmt == FMT_MXINT4)
+      launch_tc(rotate_quantize_pair_kernel<FMT_MXINT4>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
+                s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
+                st->err_word);
+    else if (fmt == FMT_NVFP4)
       launch_tc(rotate_quantize_pair_kernel<FMT_NVFP4>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
                 s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d,
                 tensor_scale, st->err_word);
@@ -353,7 +363,11 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
   const int m_tiles = (int)((M + 127) / 128);
   const int tiles = m_tiles * (int)((d + 255) / 256);
   const int grid = tiles < st->sm_count ? tiles : st->sm_count;
-  if (fmt == FMT_NVFP4)
+  if (fmt == FMT_MXINT4)
+    launch_tc(rotate_quantize_kernel<256, FMT_MXINT4>, 1, grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s,
+              tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
+              st->err_word);
+  else if (fmt == FMT_NVFP4)
     launch_tc(rotate_quantize_kernel<256, FMT_NVFP4>, 1, grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s,
               tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, tensor_scale,
               st->err_word);
@@ -436,6 +450,7 @@ static torq_status gemm_impl(const void* Aq, const void* As, const void* Wq, con
   if (!st->arch_ok) return TORQ_ERR_ARCH;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   constexpr int BN = 256;
+  const uint64_t krow = (uint64_t)(FMT == FMT_MXINT4 ? K : K / 2);   // operand bytes per row
   CUtensorMap tmA, tmB;
   // CTA pairs from two row tiles on -- except for exactly two row tiles with so few 256-column tiles
   // that the pairs would leave more than half of the SMs idle: 128 x 128 tiles on single CTAs then
@@ -445,11 +460,12 @@ static torq_status gemm_impl(const void* Aq, const void* As, const void* Wq, con
   if (use_pairs) {
     CUtensorMap tmSFA, tmSFB;
     const uint64_t kb4 = (uint64_t)(K / (FMT == FMT_NVFP4 ? 64 : 128));   // 512-byte scale chunks per row
-    if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, (uint64_t)(K / 2), 128, 128) ||
-        !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)(K / 2), BN / 2, 128) ||
-        !encode_2d(&tmSFA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, As, (uint64_t)((M + 127) / 128), kb4 * 128, 1, 256,
+    constexpr uint32_t sf_box = GemmPairCfgT<FMT>::SF_BOX_WORDS;
+    if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, krow, 128, 128) ||
+        !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, krow, BN / 2, 128) ||
+        !encode_2d(&tmSFA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, As, (uint64_t)((M + 127) / 128), kb4 * 128, 1, sf_box,
                    CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !encode_2d(&tmSFB, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, Ws, (uint64_t)((N + 127) / 128), kb4 * 128, 1, 256,
+        !encode_2d(&tmSFB, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, Ws, (uint64_t)((N + 127) / 128), kb4 * 128, 1, sf_box,
                    CU_TENSOR_MAP_SWIZZLE_NONE))
       return TORQ_ERR_LAUNCH;
     CUtensorMap tmY;
@@ -468,8 +484,8 @@ static torq_status gemm_impl(const void* Aq, const void* As, const void* Wq, con
   // SMs idle (128-column tiles double the number of CTAs pulling on memory).
   const bool narrow = 2 * (int)((M + 127) / 128) * (int)((N + BN - 1) / BN) <= st->sm_count;
   const uint32_t bn = narrow ? 128 : BN;
-  if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, (uint64_t)(K / 2), 128, 128) ||
-      !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)(K / 2), bn, 128))
+  if (!encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, krow, 128, 128) ||
+      !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, krow, bn, 128))
     return TORQ_ERR_LAUNCH;
   const int tiles = (int)((M + 127) / 128) * (int)((N + bn - 1) / bn);
   const int grid = tiles < st->sm_count ? tiles : st->sm_count;
@@ -583,6 +599,90 @@ torq_status torq_rotated_linear_nvfp4(const void* X, const void* R_inter, const 
     return TORQ_ERR_LAUNCH;
   if (dbg_scales && cudaMemcpyAsync(dbg_scales, scales, torq_nvfp4_scales_bytes(M, d),
                                     cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return TORQ_ERR_LAUNCH;
+  return TORQ_OK;
+}
+
+// ---- MXINT4 (format study of Section 6): integer codes, E8M0 scales, E4M3 operand bytes ----------
+
+size_t torq_mxint4_workspace_bytes(int64_t M, int64_t d, int64_t N) {
+  (void)N;
+  if (M <= 0 || d <= 0) return 0;
+  return ((size_t)M * (size_t)d + 255) / 256 * 256 + torq_scales_bytes(M, d);
+}
+
+torq_status torq_quantize_mxint4(const void* Z, torq_dtype z_dtype, int64_t M, int64_t d, int packed, void* out_codes,
+                                 void* out_scales, void* stream) {
+  if (!Z || !out_codes || !out_scales) return TORQ_ERR_NULL;
+  if (M < 1 || d < 32 || d % 32 != 0 || M > (1 << 30) || d > (1 << 30)) return TORQ_ERR_SHAPE;
+  if (z_dtype != TORQ_F32 && z_dtype != TORQ_BF16) return TORQ_ERR_SHAPE;
+  if (!aligned16(Z) || !aligned16(out_codes) || !aligned16(out_scales)) return TORQ_ERR_ALIGN;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t kb4 = (d / 32 + 3) / 4;
+  const int64_t items = ((M + 127) / 128 * 128) * ((kb4 * 128 + 255) / 256);   // warps
+  const int grid = ew_grid(items, 8, st->sm_count);
+  uint8_t* c = static_cast<uint8_t*>(out_codes);
+  uint8_t* sc = static_cast<uint8_t*>(out_scales);
+  if (z_dtype == TORQ_F32) {
+    const float* z = static_cast<const float*>(Z);
+    if (packed) mxint4_quantize_kernel<float, true><<<grid, 256, 0, s>>>(z, M, d, c, sc);
+    else mxint4_quantize_kernel<float, false><<<grid, 256, 0, s>>>(z, M, d, c, sc);
+  } else {
+    const __nv_bfloat16* z = static_cast<const __nv_bfloat16*>(Z);
+    if (packed) mxint4_quantize_kernel<__nv_bfloat16, true><<<grid, 256, 0, s>>>(z, M, d, c, sc);
+    else mxint4_quantize_kernel<__nv_bfloat16, false><<<grid, 256, 0, s>>>(z, M, d, c, sc);
+  }
+  return launch_status();
+}
+
+torq_status torq_mxint4_expand(const void* packed, int64_t rows, int64_t k, void* out_bytes, void* stream) {
+  if (!packed || !out_bytes) return TORQ_ERR_NULL;
+  if (rows < 1 || k < 32 || k % 32 != 0 || rows > (1 << 30) || k > (1 << 30)) return TORQ_ERR_SHAPE;
+  if (!aligned16(packed) || !aligned16(out_bytes)) return TORQ_ERR_ALIGN;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  const int64_t words = rows * (k / 8);
+  mxint4_expand_kernel<<<ew_grid(words, 256, st->sm_count), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint32_t*>(packed), words, static_cast<uint2*>(out_bytes));
+  return launch_status();
+}
+
+torq_status torq_rotate_quantize_mxint4(const void* X, const void* R_inter, const void* R_intra, int64_t M,
+                                        int64_t d, void* out_bytes, void* out_scales, void* stream) {
+  return rotate_quantize_impl(X, R_inter, R_intra, M, d, out_bytes, out_scales, nullptr, 0, stream, FMT_MXINT4,
+                              0.0f);
+}
+
+torq_status torq_mxint4_gemm(const void* A8, const void* As, const void* W8, const void* Ws, int64_t M, int64_t N,
+                             int64_t K, void* Y, torq_dtype y_dtype, void* stream) {
+  return gemm_impl<FMT_MXINT4>(A8, As, W8, Ws, M, N, K, Y, y_dtype, 1.0f, stream);
+}
+
+torq_status torq_rotated_linear_mxint4(const void* X, const void* R_inter, const void* R_intra, const void* W8,
+                                       const void* Ws, int64_t M, int64_t d, int64_t N, void* Y, torq_dtype y_dtype,
+                                       void* workspace, size_t workspace_bytes, void* dbg_bytes, void* dbg_scales,
+                                       void* stream) {
+  if (!X || !R_inter || !W8 || !Ws || !Y) return TORQ_ERR_NULL;
+  if (M < 1 || d < 128 || d % 128 != 0 || N < 8 || N % 8 != 0 || M > (1 << 30) || d > (1 << 24))
+    return TORQ_ERR_SHAPE;
+  if (!workspace || workspace_bytes < torq_mxint4_workspace_bytes(M, d, N)) return TORQ_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return TORQ_ERR_ALIGN;
+  uint8_t* bytes = static_cast<uint8_t*>(workspace);
+  const size_t n_bytes = (size_t)M * (size_t)d;
+  uint8_t* scales = bytes + (n_bytes + 255) / 256 * 256;
+  torq_status rc = rotate_quantize_impl(X, R_inter, R_intra, M, d, bytes, scales, nullptr, 0, stream, FMT_MXINT4, 0.0f);
+  if (rc != TORQ_OK) return rc;
+  rc = torq_mxint4_gemm(bytes, scales, W8, Ws, M, N, d, Y, y_dtype, stream);
+  if (rc != TORQ_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dbg_bytes && cudaMemcpyAsync(dbg_bytes, bytes, n_bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return TORQ_ERR_LAUNCH;
+  if (dbg_scales &&
+      cudaMemcpyAsync(dbg_scales, scales, torq_scales_bytes(M, d), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
     return TORQ_ERR_LAUNCH;
   return TORQ_OK;
 }

@@ -75,6 +75,18 @@ def lib() -> ctypes.CDLL:
     L.torq_nvfp4_gemm.restype = ci
     L.torq_rotated_linear_nvfp4.argtypes = [vp, vp, vp, f32, vp, vp, f32, i64, i64, i64, vp, ci, vp, sz, vp, vp, vp]
     L.torq_rotated_linear_nvfp4.restype = ci
+    L.torq_mxint4_workspace_bytes.argtypes = [i64, i64, i64]
+    L.torq_mxint4_workspace_bytes.restype = sz
+    L.torq_quantize_mxint4.argtypes = [vp, ci, i64, i64, ci, vp, vp, vp]
+    L.torq_quantize_mxint4.restype = ci
+    L.torq_mxint4_expand.argtypes = [vp, i64, i64, vp, vp]
+    L.torq_mxint4_expand.restype = ci
+    L.torq_rotate_quantize_mxint4.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp]
+    L.torq_rotate_quantize_mxint4.restype = ci
+    L.torq_mxint4_gemm.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, ci, vp]
+    L.torq_mxint4_gemm.restype = ci
+    L.torq_rotated_linear_mxint4.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, vp, sz, vp, vp, vp]
+    L.torq_rotated_linear_mxint4.restype = ci
     L.torq_block_covariance.argtypes = [vp, i64, i64, vp, vp]
     L.torq_block_covariance.restype = ci
     L.torq_givens_equalize.argtypes = [vp, i64, ctypes.c_double, vp, vp, vp, vp]
@@ -396,6 +408,102 @@ def prepare_weights_nvfp4(R_inter, R_intra32, W):
     ts = float(Wp.abs().max().item()) / (6.0 * 448.0)
     Wq, Ws = torq_quantize_nvfp4(Wp, ts)
     return Wq, Ws, ts
+
+
+# ---- MXINT4 variant (format study of Section 6) ---------------------------------------------------------
+def torq_mxint4_workspace_bytes(M: int, d: int, N: int) -> int:
+    return int(lib().torq_mxint4_workspace_bytes(M, d, N))
+
+
+def torq_quantize_mxint4(Z, packed: bool = False, out_codes=None, out_scales=None, stream=None):
+    """Z [M,d] float32 or bfloat16 -> (codes, tiled E8M0 scale bytes).  packed: [M,d/2] two's-complement
+    nibbles (stored form); otherwise [M,d] E4M3 bytes whose values are the integer codes (operand form)."""
+    M, d = Z.shape
+    dt = TORQ_F32 if Z.dtype == torch.float32 else TORQ_BF16
+    _check(Z, torch.float32 if dt == TORQ_F32 else torch.bfloat16, "Z")
+    if out_codes is None:
+        out_codes = torch.empty((M, d // 2 if packed else d), dtype=torch.uint8, device=Z.device)
+    if out_scales is None:
+        out_scales = torch.empty(torq_scales_bytes(M, d), dtype=torch.uint8, device=Z.device)
+    _check(out_codes, torch.uint8, "out_codes")
+    _check(out_scales, torch.uint8, "out_scales")
+    _raise(lib().torq_quantize_mxint4(_ptr(Z), dt, M, d, 1 if packed else 0, _ptr(out_codes), _ptr(out_scales),
+                                      _stream(stream)), "torq_quantize_mxint4")
+    return out_codes, out_scales
+
+
+def torq_mxint4_expand(packed, out=None, stream=None):
+    """Stored form [rows,k/2] -> operand form [rows,k]."""
+    _check(packed, torch.uint8, "packed")
+    rows, k2 = packed.shape
+    if out is None:
+        out = torch.empty((rows, 2 * k2), dtype=torch.uint8, device=packed.device)
+    _check(out, torch.uint8, "out")
+    _raise(lib().torq_mxint4_expand(_ptr(packed), rows, 2 * k2, _ptr(out), _stream(stream)), "torq_mxint4_expand")
+    return out
+
+
+def torq_rotate_quantize_mxint4(X, R_inter, R_intra, out_bytes=None, out_scales=None, stream=None):
+    """X [M,d] bf16, R_inter [d,d] bf16, R_intra [d/32,32,32] bf16 or None -> (operand bytes [M,d], scales)."""
+    M, d = X.shape
+    for t, n in ((X, "X"), (R_inter, "R_inter"), (R_intra, "R_intra")):
+        _check(t, torch.bfloat16, n)
+    if out_bytes is None:
+        out_bytes = torch.empty((M, d), dtype=torch.uint8, device=X.device)
+    if out_scales is None:
+        out_scales = torch.empty(torq_scales_bytes(M, d), dtype=torch.uint8, device=X.device)
+    _raise(lib().torq_rotate_quantize_mxint4(_ptr(X), _ptr(R_inter), _ptr(R_intra), M, d, _ptr(out_bytes),
+                                             _ptr(out_scales), _stream(stream)), "torq_rotate_quantize_mxint4")
+    return out_bytes, out_scales
+
+
+def torq_mxint4_gemm(A8, As, W8, Ws, out_dtype=torch.bfloat16, Y=None, stream=None):
+    """A8 [M,K], W8 [N,K] operand bytes; As, Ws tiled E8M0 scale bytes -> Y [M,N]."""
+    M, K = A8.shape
+    N = W8.shape[0]
+    for t, n in ((A8, "A8"), (As, "As"), (W8, "W8"), (Ws, "Ws")):
+        _check(t, torch.uint8, n)
+    if Y is None:
+        Y = torch.empty((M, N), dtype=out_dtype, device=A8.device)
+    _check(Y, Y.dtype, "Y")
+    dt = TORQ_F32 if Y.dtype == torch.float32 else TORQ_BF16
+    _raise(lib().torq_mxint4_gemm(_ptr(A8), _ptr(As), _ptr(W8), _ptr(Ws), M, N, K, _ptr(Y), dt, _stream(stream)),
+           "torq_mxint4_gemm")
+    return Y
+
+
+def torq_rotated_linear_mxint4(X, R_inter, R_intra, W8, Ws, out_dtype=torch.bfloat16, Y=None, workspace=None,
+                               dbg_bytes=None, dbg_scales=None, stream=None):
+    """Rotate, quantize to MXINT4 and multiply in one call.  Returns Y [M,N]."""
+    M, d = X.shape
+    N = W8.shape[0]
+    for t, n in ((X, "X"), (R_inter, "R_inter"), (R_intra, "R_intra")):
+        _check(t, torch.bfloat16, n)
+    for t, n in ((W8, "W8"), (Ws, "Ws"), (dbg_bytes, "dbg_bytes"), (dbg_scales, "dbg_scales")):
+        _check(t, torch.uint8, n)
+    if Y is None:
+        Y = torch.empty((M, N), dtype=out_dtype, device=X.device)
+    if workspace is None:
+        workspace = torch.empty(torq_mxint4_workspace_bytes(M, d, N), dtype=torch.uint8, device=X.device)
+    dt = TORQ_F32 if Y.dtype == torch.float32 else TORQ_BF16
+    _raise(lib().torq_rotated_linear_mxint4(_ptr(X), _ptr(R_inter), _ptr(R_intra), _ptr(W8), _ptr(Ws), M, d, N,
+                                            _ptr(Y), dt, _ptr(workspace), workspace.numel(), _ptr(dbg_bytes),
+                                            _ptr(dbg_scales), _stream(stream)), "torq_rotated_linear_mxint4")
+    return Y
+
+
+def prepare_weights_mxint4(R_inter, R_intra, W):
+    """Offline weight side in MXINT4: W' = R~^T W (as prepare_weights), quantized along K.
+    Returns (stored form [N,d/2], operand form [N,d], tiled scales)."""
+    Rm = torq_merge_rotations(R_inter, R_intra)
+    prev = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = False
+    try:
+        Wp = torch.matmul(W.t().contiguous().to(torch.float32), Rm).contiguous()
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = prev
+    Wn, Ws = torq_quantize_mxint4(Wp, packed=True)
+    return Wn, torq_mxint4_expand(Wn), Ws
 
 
 # ---- calibration of the inter-block rotation (Section 5.1, Algorithm 1; offline) -----------------------

@@ -98,3 +98,25 @@ def test_nvfp4_and_calibration_argument_errors_and_sizes():
     assert L.torq_givens_equalize(one, 0, 1e-9, one, None, None, None) == 2
     assert L.torq_givens_equalize(one, 8, -1.0, one, None, None, None) == 2
     assert L.torq_givens_equalize(None, 8, 1e-9, one, None, None, None) == 1
+
+
+def test_mxint4_argument_errors_and_sizes():
+    L = torq.lib()
+    one = ctypes.c_void_p(16)
+    odd = ctypes.c_void_p(24)
+    # operand form: one byte per element, plus the 32-block scale tiles
+    assert torq.torq_mxint4_workspace_bytes(2048, 4096, 6144) == 2048 * 4096 + torq.torq_scales_bytes(2048, 4096)
+    assert torq.torq_mxint4_workspace_bytes(0, 4096, 8) == 0
+    assert L.torq_quantize_mxint4(one, 0, 4, 64, 0, None, one, None) == 1
+    assert L.torq_quantize_mxint4(one, 0, 4, 48, 1, one, one, None) == 2              # d % 32 != 0
+    assert L.torq_quantize_mxint4(odd, 0, 4, 64, 1, one, one, None) == 3
+    assert L.torq_mxint4_expand(None, 4, 64, one, None) == 1
+    assert L.torq_mxint4_expand(one, 4, 40, one, None) == 2
+    assert L.torq_rotate_quantize_mxint4(one, None, None, 4, 64, one, one, None) == 1         # R_inter is required
+    assert L.torq_rotate_quantize_mxint4(one, one, None, 4, 48, one, one, None) == 2
+    assert L.torq_mxint4_gemm(one, one, one, one, 4, 8, 96, one, 0, None) == 2               # K % 128 != 0
+    assert L.torq_mxint4_gemm(one, None, one, one, 4, 8, 128, one, 0, None) == 1
+    assert L.torq_mxint4_gemm(one, one, odd, one, 4, 8, 128, one, 0, None) == 3
+    assert L.torq_rotated_linear_mxint4(one, one, one, one, one, 4, 128, 8, one, 0, one, 16, None, None, None) == 7
+    assert L.torq_rotated_linear_mxint4(one, None, one, one, one, 4, 128, 8, one, 0, one, 1 << 20, None, None,
+                                        None) == 1
