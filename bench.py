@@ -212,6 +212,9 @@ def main():
     # exceeds its token's 2-norm, so the largest norm over the top of the E4M3 range never saturates
     x_ts_nv = float(X0.float().norm(dim=1).max().item()) / (6.0 * 448.0)
     ws_nv = [torch.empty(torq.torq_nvfp4_workspace_bytes(M, d, N), dtype=torch.uint8, device="cuda") for _ in range(2)]
+    # the MXINT4 variant (integer codes as E4M3 operand bytes, same rotations as the MXFP4 layer)
+    _, W8_i4, Ws_i4 = torq.prepare_weights_mxint4(R0, Ri0, torch.from_numpy(w).cuda())
+    ws_i4 = [torch.empty(torq.torq_mxint4_workspace_bytes(M, d, N), dtype=torch.uint8, device="cuda") for _ in range(2)]
     del w
     set_bytes = X0.numel() * 2 + R0.numel() * 2 + Wq0.numel() + M * N * 2
     n_sets = max(2, min(N_BUFFER_SETS, int(8e9 // set_bytes)))     # bounded device memory
@@ -332,6 +335,26 @@ def main():
                                        workspace=ws_nv[nv_i[0]])
 
     t_nv_rot, t_nv_gemm, t_nv_layer = timed_loop(nv_rot), timed_loop(nv_gemm), timed_loop(nv_layer)
+
+    # the MXINT4 variant, likewise
+    def i4_bytes_scales(k):
+        return ws_i4[k][: M * d].view(M, d), ws_i4[k][(M * d + 255) // 256 * 256:][: torq.torq_scales_bytes(M, d)]
+
+    def i4_rot(b):
+        nv_i[0] ^= 1
+        c, sc = i4_bytes_scales(nv_i[0])
+        torq.torq_rotate_quantize_mxint4(b["X"], b["R"], b["Ri"], out_bytes=c, out_scales=sc)
+
+    def i4_gemm(b):
+        nv_i[0] ^= 1
+        c, sc = i4_bytes_scales(nv_i[0])
+        torq.torq_mxint4_gemm(c, sc, W8_i4, Ws_i4, Y=b["Y"])
+
+    def i4_layer(b):
+        nv_i[0] ^= 1
+        torq.torq_rotated_linear_mxint4(b["X"], b["R"], b["Ri"], W8_i4, Ws_i4, Y=b["Y"], workspace=ws_i4[nv_i[0]])
+
+    t_i4_rot, t_i4_gemm, t_i4_layer = timed_loop(i4_rot), timed_loop(i4_gemm), timed_loop(i4_layer)
     barrier()
     clocks = sampler.stop()
     assert torq.torq_last_device_error() == 0
@@ -450,6 +473,14 @@ def main():
                 "gemm_ms": t_nv_gemm * 1e3, "gemm_TFLOPs": gemm_flop / t_nv_gemm / 1e12,
                 "gemm_frac": gemm_flop / t_nv_gemm / 1e12 / fp4_peak,
                 "whole_layer_ms_per_step": t_nv_layer * 1e3, "whole_layer_tokens_per_s": world * M / t_nv_layer},
+            "mxint4_variant": {
+                "what": "the same layer in MXINT4 (32-element blocks, E8M0 scales, integers in [-7,7] fed to the tensor "
+                        "cores as E4M3 bytes; kind::mxf8f6f4 GEMM at the 8-bit rate), single-pass rotation kernels",
+                "rotate_quant_ms": t_i4_rot * 1e3, "rotate_quant_TFLOPs": rot_flop / t_i4_rot / 1e12,
+                "rotate_quant_frac": rot_flop / t_i4_rot / 1e12 / bf16_peak,
+                "gemm_ms": t_i4_gemm * 1e3, "gemm_TFLOPs": gemm_flop / t_i4_gemm / 1e12,
+                "gemm_frac_of_half_fp4_peak": gemm_flop / t_i4_gemm / 1e12 / (fp4_peak / 2),
+                "whole_layer_ms_per_step": t_i4_layer * 1e3, "whole_layer_tokens_per_s": world * M / t_i4_layer},
             "e2e": {"value": world * M / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": Xh.numel() * 2,
                     "d2h_bytes_per_step": Yh.numel() * 2},
             "gpu_launches": int(launches), "clocks": clocks,
