@@ -265,13 +265,21 @@ torq_status torq_mxint4_expand(const void* packed, int64_t rows, int64_t k, void
 torq_status torq_rotate_quantize_mxint4(const void* X, const void* R_inter, const void* R_intra, int64_t M,
                                         int64_t d, void* out_bytes, void* out_scales, void* stream);
 
+/* torq_rotate_quantize_structured with the MXINT4 quantizer at its end (R_B [d/32, d/32] bf16, one
+ * shared R_intra [32, 32] bf16 or NULL; d % 256 == 0).  out_bytes [M, d] operand form. */
+torq_status torq_rotate_quantize_structured_mxint4(const void* X, const void* R_B, const void* R_intra,
+                                                   int64_t M, int64_t d, void* out_bytes, void* out_scales,
+                                                   void* stream);
+
 /* Algorithm 3 step 5 on MXINT4 operands: Y[m,n] = sum_k a^[m,k] w^[n,k].  A8 [M, K], W8 [N, K]
  * operand form; As, Ws tiled E8M0 scales; K % 128 == 0, N % 8 == 0; Y [M, N] fp32 or bf16. */
 torq_status torq_mxint4_gemm(const void* A8, const void* As, const void* W8, const void* Ws, int64_t M,
                              int64_t N, int64_t K, void* Y, torq_dtype y_dtype, void* stream);
 
 /* Steps 1-5 in MXINT4: torq_rotate_quantize_mxint4 into `workspace` (at least
- * torq_mxint4_workspace_bytes(M, d, N) bytes, 256-byte aligned), then torq_mxint4_gemm.  dbg_bytes
+ * torq_mxint4_workspace_bytes(M, d, N) bytes, 256-byte aligned), then torq_mxint4_gemm.  As in
+ * torq_rotated_linear, few tokens take the rotation split along its contraction, its fp32 partial
+ * sums in the same workspace.  dbg_bytes
  * [M, d] / dbg_scales, when not NULL, receive copies of the quantized activations.
  * d % 128 == 0, N % 8 == 0. */
 torq_status torq_rotated_linear_mxint4(const void* X, const void* R_inter, const void* R_intra, const void* W8,

@@ -12,6 +12,7 @@
 #pragma once
 #include <cuda_bf16.h>
 #include "nvfp4_quantize.cuh"
+#include "mxint4_quantize.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -196,6 +197,7 @@ rotate_splitk_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 // Rows M .. (group end) and K-blocks d/32 .. (padded to 4) only get their padding scale byte (0).
 // FMT_NVFP4: the 32 columns are two 16-element blocks (two threads each), E4M3 scales at twice the
 // block index, `tensor_scale` the tensor's float32 scale; the grid covers the padded 16-blocks in pairs.
+// FMT_MXINT4: integer codes as one E4M3 operand byte per element (`codes` is [M, d] bytes).
 template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(256)
 splitk_reduce_quantize_kernel(const float* __restrict__ P, const __nv_bfloat16* __restrict__ R_intra,
@@ -286,9 +288,19 @@ splitk_reduce_quantize_kernel(const float* __restrict__ P, const __nv_bfloat16* 
       const int r = 16 * warp + r8 + 8 * rh;
       const int row = row0 + r;
       uint32_t word, sb;
-      if constexpr (FMT == FMT_NVFP4) nv_quantize_row_fragment(v, p, nv_scale(tensor_scale), word, sb);
-      else quantize_row_fragment(v, p, word, sb);
-      if (r < rows) *reinterpret_cast<uint32_t*>(codes + (size_t)row * (d / 2) + b * 16 + 4 * p) = word;
+      if constexpr (FMT == FMT_MXINT4) {
+        uint32_t pr[4];
+        mxint4_quantize_row_fragment(v, pr, sb);
+        if (r < rows) {
+          uint8_t* dst = codes + (size_t)row * d + b * 32 + 2 * p;
+#pragma unroll
+          for (int nt = 0; nt < 4; ++nt) *reinterpret_cast<uint16_t*>(dst + 8 * nt) = (uint16_t)pr[nt];
+        }
+      } else {
+        if constexpr (FMT == FMT_NVFP4) nv_quantize_row_fragment(v, p, nv_scale(tensor_scale), word, sb);
+        else quantize_row_fragment(v, p, word, sb);
+        if (r < rows) *reinterpret_cast<uint32_t*>(codes + (size_t)row * (d / 2) + b * 16 + 4 * p) = word;
+      }
       if (p == 0) {
         if constexpr (FMT == FMT_NVFP4) {
           scales[scale_offset(row, 2 * b, kb4)] = r < rows ? (uint8_t)(sb & 0xFF) : (uint8_t)0;
@@ -328,9 +340,15 @@ splitk_reduce_quantize_kernel(const float* __restrict__ P, const __nv_bfloat16* 
   float inv;
   block_scale(amax, sbyte, inv);
   if (r < rows) {
-    const uint32_t w = pack8_e2m1(z[0] * inv, z[1] * inv, z[2] * inv, z[3] * inv, z[4] * inv, z[5] * inv,
-                                  z[6] * inv, z[7] * inv);
-    *reinterpret_cast<uint32_t*>(codes + (size_t)row * (d / 2) + b * 16 + 4 * p) = w;
+    if constexpr (FMT == FMT_MXINT4) {
+      *reinterpret_cast<uint2*>(codes + (size_t)row * d + b * 32 + 8 * p) = make_uint2(
+          pack4_e4m3(int4_round(z[0] * inv), int4_round(z[1] * inv), int4_round(z[2] * inv), int4_round(z[3] * inv)),
+          pack4_e4m3(int4_round(z[4] * inv), int4_round(z[5] * inv), int4_round(z[6] * inv), int4_round(z[7] * inv)));
+    } else {
+      const uint32_t w = pack8_e2m1(z[0] * inv, z[1] * inv, z[2] * inv, z[3] * inv, z[4] * inv, z[5] * inv,
+                                    z[6] * inv, z[7] * inv);
+      *reinterpret_cast<uint32_t*>(codes + (size_t)row * (d / 2) + b * 16 + 4 * p) = w;
+    }
   }
   if (p == 0) scales[scale_offset(row, b, kb4)] = r < rows ? (uint8_t)sbyte : (uint8_t)0;
 }

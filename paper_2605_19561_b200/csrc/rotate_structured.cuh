@@ -26,6 +26,7 @@
 #pragma once
 #include <cuda_bf16.h>
 #include "nvfp4_quantize.cuh"
+#include "mxint4_quantize.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -53,7 +54,8 @@ struct RotStructCfg {
 // 64-byte swizzle.
 // FMT_NVFP4: the NVFP4 quantizer at the end (two 16-element blocks per row of 32, E4M3 scales,
 // `tensor_scale` the tensor's float32 scale; unused for MXFP4); R_intra stays a 32 x 32 matrix (two
-// 16 x 16 blocks on its diagonal for a 16-wide intra rotation).
+// 16 x 16 blocks on its diagonal for a 16-wide intra rotation).  FMT_MXINT4: integer codes as one E4M3
+// operand byte per element (`codes` is [M, d] bytes), scale bytes as for MXFP4.
 template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(608, 1)
 rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_constant__ CUtensorMap tmX3,
@@ -275,12 +277,19 @@ rotate_structured_kernel(const __grid_constant__ CUtensorMap tmRB, const __grid_
         float z[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(y[i]);
-        uint4 cw;
+        uint4 cw, cw2;
         uint32_t sbyte;
-        if constexpr (FMT == FMT_NVFP4) nv_quantize_2x16(z, nv_scale(tensor_scale), cw, sbyte);
+        if constexpr (FMT == FMT_MXINT4) mxint4_quantize_block32(z, cw, cw2, sbyte);
+        else if constexpr (FMT == FMT_NVFP4) nv_quantize_2x16(z, nv_scale(tensor_scale), cw, sbyte);
         else quantize_block32(z, cw, sbyte);
         if (token < M && blk < nblocks) {
-          *reinterpret_cast<uint4*>(codes + token * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+          if constexpr (FMT == FMT_MXINT4) {             // one operand byte per element
+            uint4* dst = reinterpret_cast<uint4*>(codes + token * (int64_t)d + (int64_t)blk * 32);
+            dst[0] = cw;
+            dst[1] = cw2;
+          } else {
+            *reinterpret_cast<uint4*>(codes + token * (int64_t)(d / 2) + (int64_t)blk * 16) = cw;
+          }
           if constexpr (FMT == FMT_NVFP4) {              // two scale bytes, adjacent in the tiled layout
             *reinterpret_cast<uint16_t*>(scales + scale_offset(token, 2 * blk, (2 * nblocks + 3) / 4)) = (uint16_t)sbyte;
           } else {

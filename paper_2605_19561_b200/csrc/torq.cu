@@ -113,7 +113,8 @@ static DeviceState* device_state() {
               opt_in_smem(mxfp4_gemm_kernel<128, 2, FMT_MXINT4>, GemmCfg<128, 2, FMT_MXINT4>::SMEM_BYTES) &&
               opt_in_smem(mxfp4_gemm_pair_kernel<FMT_MXINT4>, GemmPairCfgT<FMT_MXINT4>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_kernel<256, FMT_MXINT4>, RotCfg<256>::SMEM_BYTES) &&
-              opt_in_smem(rotate_quantize_pair_kernel<FMT_MXINT4>, RotPairCfg::SMEM_BYTES);
+              opt_in_smem(rotate_quantize_pair_kernel<FMT_MXINT4>, RotPairCfg::SMEM_BYTES) &&
+              opt_in_smem(rotate_structured_kernel<FMT_MXINT4>, RotStructCfg::SMEM_BYTES);
     if (!ok) return nullptr;
     st.rot_pairs = max_active_pairs(rotate_quantize_pair_kernel<FMT_MXFP4>, RotPairCfg::THREADS,
                                     RotPairCfg::SMEM_BYTES, st.sm_count);
@@ -318,7 +319,7 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
   if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d, 128, 64) ||
       !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
     return TORQ_ERR_LAUNCH;
-  const int splits = fmt == FMT_MXINT4 ? 1 : rotation_splits(M, d, st->sm_count);   // MXINT4: single pass only
+  const int splits = rotation_splits(M, d, st->sm_count);
   if (splits >= 2 && scratch && scratch_bytes >= splitk_scratch_bytes(M, d, splits) &&
       (reinterpret_cast<uintptr_t>(scratch) & 15u) == 0) {
     // Few tokens: split K over the SMs, partial tiles to scratch, then reduce + intra + quantize.
@@ -331,7 +332,11 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
     launch_tc(rotate_splitk_kernel, 1, m_tiles * n_tiles * splits, RotSplitCfg::THREADS, RotSplitCfg::SMEM_BYTES, s, tmX, tmR,
               tmP, (int)M, (int)d, splits, st->err_word);
     if (launch_status() != TORQ_OK) return TORQ_ERR_LAUNCH;
-    if (fmt == FMT_NVFP4)
+    if (fmt == FMT_MXINT4)
+      launch_tc(splitk_reduce_quantize_kernel<FMT_MXINT4>, 1, (int)(((d / 32 + 3) / 4) * 4) * m_tiles * 4, 256, 0, s,
+                static_cast<const float*>(scratch), static_cast<const __nv_bfloat16*>(R_intra), (int)M, (int)d, splits,
+                0.0f, codes, scales);
+    else if (fmt == FMT_NVFP4)
       launch_tc(splitk_reduce_quantize_kernel<FMT_NVFP4>, 1, (int)(((d / 16 + 3) / 4) * 2) * m_tiles * 4, 256, 0, s,
                 static_cast<const float*>(scratch), static_cast<const __nv_bfloat16*>(R_intra), (int)M, (int)d, splits,
                 tensor_scale, codes, scales);
@@ -401,7 +406,11 @@ static torq_status rotate_structured_impl(const void* X, const void* R_B, const 
     return TORQ_ERR_LAUNCH;
   const int64_t tiles = ((nb + 127) / 128) * ((M + RotStructCfg::TOK - 1) / RotStructCfg::TOK);
   const int grid = (int)(tiles < st->sm_count ? tiles : st->sm_count);
-  if (fmt == FMT_NVFP4)
+  if (fmt == FMT_MXINT4)
+    launch_tc(rotate_structured_kernel<FMT_MXINT4>, 1, grid, RotStructCfg::THREADS, RotStructCfg::SMEM_BYTES, s, tmRB,
+              tmX3, static_cast<const __nv_bfloat16*>(R_intra), static_cast<uint8_t*>(out_codes),
+              static_cast<uint8_t*>(out_scales), (int)M, (int)d, 0.0f, st->err_word);
+  else if (fmt == FMT_NVFP4)
     launch_tc(rotate_structured_kernel<FMT_NVFP4>, 1, grid, RotStructCfg::THREADS, RotStructCfg::SMEM_BYTES, s, tmRB,
               tmX3, static_cast<const __nv_bfloat16*>(R_intra), static_cast<uint8_t*>(out_codes),
               static_cast<uint8_t*>(out_scales), (int)M, (int)d, tensor_scale, st->err_word);
@@ -605,10 +614,14 @@ torq_status torq_rotated_linear_nvfp4(const void* X, const void* R_inter, const 
 
 // ---- MXINT4 (format study of Section 6): integer codes, E8M0 scales, E4M3 operand bytes ----------
 
+static size_t mxint4_quantized_bytes(int64_t M, int64_t d) {
+  return ((size_t)M * (size_t)d + 255) / 256 * 256 + torq_scales_bytes(M, d);
+}
+
 size_t torq_mxint4_workspace_bytes(int64_t M, int64_t d, int64_t N) {
   (void)N;
   if (M <= 0 || d <= 0) return 0;
-  return ((size_t)M * (size_t)d + 255) / 256 * 256 + torq_scales_bytes(M, d);
+  return mxint4_quantized_bytes(M, d) + splitk_scratch_bytes(M, d, rotation_splits(M, d, 0));
 }
 
 torq_status torq_quantize_mxint4(const void* Z, torq_dtype z_dtype, int64_t M, int64_t d, int packed, void* out_codes,
@@ -657,6 +670,11 @@ torq_status torq_rotate_quantize_mxint4(const void* X, const void* R_inter, cons
                               0.0f);
 }
 
+torq_status torq_rotate_quantize_structured_mxint4(const void* X, const void* R_B, const void* R_intra, int64_t M,
+                                                   int64_t d, void* out_bytes, void* out_scales, void* stream) {
+  return rotate_structured_impl(X, R_B, R_intra, M, d, out_bytes, out_scales, stream, FMT_MXINT4, 0.0f);
+}
+
 torq_status torq_mxint4_gemm(const void* A8, const void* As, const void* W8, const void* Ws, int64_t M, int64_t N,
                              int64_t K, void* Y, torq_dtype y_dtype, void* stream) {
   return gemm_impl<FMT_MXINT4>(A8, As, W8, Ws, M, N, K, Y, y_dtype, 1.0f, stream);
@@ -674,7 +692,9 @@ torq_status torq_rotated_linear_mxint4(const void* X, const void* R_inter, const
   uint8_t* bytes = static_cast<uint8_t*>(workspace);
   const size_t n_bytes = (size_t)M * (size_t)d;
   uint8_t* scales = bytes + (n_bytes + 255) / 256 * 256;
-  torq_status rc = rotate_quantize_impl(X, R_inter, R_intra, M, d, bytes, scales, nullptr, 0, stream, FMT_MXINT4, 0.0f);
+  const size_t used = mxint4_quantized_bytes(M, d);
+  torq_status rc = rotate_quantize_impl(X, R_inter, R_intra, M, d, bytes, scales, bytes + used, workspace_bytes - used,
+                                        stream, FMT_MXINT4, 0.0f);
   if (rc != TORQ_OK) return rc;
   rc = torq_mxint4_gemm(bytes, scales, W8, Ws, M, N, d, Y, y_dtype, stream);
   if (rc != TORQ_OK) return rc;

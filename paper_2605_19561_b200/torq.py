@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
     L.torq_mxint4_expand.restype = ci
     L.torq_rotate_quantize_mxint4.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp]
     L.torq_rotate_quantize_mxint4.restype = ci
+    L.torq_rotate_quantize_structured_mxint4.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp]
+    L.torq_rotate_quantize_structured_mxint4.restype = ci
     L.torq_mxint4_gemm.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, ci, vp]
     L.torq_mxint4_gemm.restype = ci
     L.torq_rotated_linear_mxint4.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, vp, sz, vp, vp, vp]
@@ -454,6 +456,21 @@ def torq_rotate_quantize_mxint4(X, R_inter, R_intra, out_bytes=None, out_scales=
         out_scales = torch.empty(torq_scales_bytes(M, d), dtype=torch.uint8, device=X.device)
     _raise(lib().torq_rotate_quantize_mxint4(_ptr(X), _ptr(R_inter), _ptr(R_intra), M, d, _ptr(out_bytes),
                                              _ptr(out_scales), _stream(stream)), "torq_rotate_quantize_mxint4")
+    return out_bytes, out_scales
+
+
+def torq_rotate_quantize_structured_mxint4(X, R_B, R_intra, out_bytes=None, out_scales=None, stream=None):
+    """The structured rotation (R_B [d/32,d/32], shared R_intra [32,32] or None) followed by the MXINT4 quantizer."""
+    M, d = X.shape
+    for t, n in ((X, "X"), (R_B, "R_B"), (R_intra, "R_intra")):
+        _check(t, torch.bfloat16, n)
+    if out_bytes is None:
+        out_bytes = torch.empty((M, d), dtype=torch.uint8, device=X.device)
+    if out_scales is None:
+        out_scales = torch.empty(torq_scales_bytes(M, d), dtype=torch.uint8, device=X.device)
+    _raise(lib().torq_rotate_quantize_structured_mxint4(_ptr(X), _ptr(R_B), _ptr(R_intra), M, d, _ptr(out_bytes),
+                                                        _ptr(out_scales), _stream(stream)),
+           "torq_rotate_quantize_structured_mxint4")
     return out_bytes, out_scales
 
 

@@ -115,6 +115,8 @@ def test_mxint4_argument_errors_and_sizes():
     assert L.torq_rotate_quantize_mxint4(one, None, None, 4, 64, one, one, None) == 1         # R_inter is required
     assert L.torq_rotate_quantize_mxint4(one, one, None, 4, 48, one, one, None) == 2
     assert L.torq_mxint4_gemm(one, one, one, one, 4, 8, 96, one, 0, None) == 2               # K % 128 != 0
+    assert L.torq_rotate_quantize_structured_mxint4(one, None, None, 4, 256, one, one, None) == 1
+    assert L.torq_rotate_quantize_structured_mxint4(one, one, None, 4, 96, one, one, None) == 2   # d % 256 != 0
     assert L.torq_mxint4_gemm(one, None, one, one, 4, 8, 128, one, 0, None) == 1
     assert L.torq_mxint4_gemm(one, one, odd, one, 4, 8, 128, one, 0, None) == 3
     assert L.torq_rotated_linear_mxint4(one, one, one, one, one, 4, 128, 8, one, 0, one, 16, None, None, None) == 7

@@ -250,7 +250,7 @@ def test_rotated_linear_end_to_end(M):
                                         dbg_bytes=dbg_b, dbg_scales=dbg_s)
     torch.cuda.synchronize()
     assert torq.torq_last_device_error() == 0
-    assert torq.torq_launch_count() - n0 == 2
+    assert torq.torq_launch_count() - n0 == 3      # so few tiles that the rotation is split along its contraction
     g_q, g_sb = _operand_to_int(dbg_b), O.unswizzle_scales(dbg_s.cpu().numpy(), M, d)
     o_out, o_q, o_sb = O.rotated_linear_mxint4(xb, rb, rib, w_q, w_sb)
     rep = _mismatch(g_q, g_sb, o_q, o_sb)
@@ -261,6 +261,43 @@ def test_rotated_linear_end_to_end(M):
     assert np.linalg.norm(got - o_out) / np.linalg.norm(o_out) <= 2e-2
     exact = O.decode_bf16(xb) @ w                         # the layer approximates x W (two 4-bit operands)
     assert np.linalg.norm(got - exact) / np.linalg.norm(exact) < 0.25
+
+
+@pytest.mark.parametrize("M,intra", [(1, True), (33, True), (128, True), (40, False)])
+def test_rotated_linear_few_tokens_takes_the_split_rotation(M, intra):
+    """Few tokens with a workspace: the rotation is split along its contraction over the SMs and a second
+    kernel adds the partials, rotates inside the blocks and quantizes (three launches instead of two)."""
+    cfg = I.CONFIGS["tiny"]
+    d, N = 1024, 256
+    xb = I.activations(cfg, M=M, d=d)
+    rb, rib, _, _ = I.rotations(cfg, d=d)
+    if not intra:
+        rib = None
+    g = np.random.default_rng(3)
+    wq = g.integers(-7, 8, (N, d)).astype(np.int8)
+    wsb = g.integers(120, 134, (N, d // 32), dtype=np.uint8)
+    dbg_b = torch.empty((M, d), dtype=torch.uint8, device="cuda")
+    dbg_s = torch.empty(torq.torq_scales_bytes(M, d), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    n0 = torq.torq_launch_count()
+    y = torq.torq_rotated_linear_mxint4(dev_bf16(xb), dev_bf16(rb), None if rib is None else dev_bf16(rib),
+                                        dev_u8(O.int4_to_e4m3(wq)), dev_u8(O.swizzle_scales(wsb, d, fill=0)),
+                                        out_dtype=torch.float32, dbg_bytes=dbg_b, dbg_scales=dbg_s)
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    assert torq.torq_launch_count() - n0 == 3
+    g_q, g_sb = _operand_to_int(dbg_b), O.unswizzle_scales(dbg_s.cpu().numpy(), M, d)
+    o_q, o_sb = O.quantize_mxint4(O.round_to_f32(O.rotate(xb, rb, rib)))
+    rep = _mismatch(g_q, g_sb, o_q, o_sb)
+    assert rep["non_adjacent"] == 0 and rep["scale_off_by_more_than_one"] == 0, rep
+    assert rep["elem"] * M * d <= max(2, 1e-4 * M * d) and rep["blocks"] * M * (d // 32) <= max(1, 1e-4 * M * (d // 32)), rep
+    buf = dbg_s.cpu().numpy().copy()                      # padding of the scale tiles is zero
+    rr, cc = np.meshgrid(np.arange(M), np.arange(d // 32), indexing="ij")
+    buf[O.scale_layout_offset(rr, cc, d)] = 0
+    assert not buf.any()
+    ref = O.gemm_mxint4(g_q, g_sb, wq, wsb)
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
 
 
 def test_device_weight_preparation_matches_the_oracle():
@@ -303,3 +340,29 @@ def test_llama3_qkv_shape_sampled_rows():
     ref = O.gemm_mxint4(g_q, g_sb, wq, wsb)
     got = y.cpu().numpy().astype(np.float64)[rows]
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
+
+
+@pytest.mark.parametrize("M,d", [(64, 256), (130, 512), (7, 1024), (2048, 4096)])
+def test_structured_rotation_with_the_mxint4_quantizer(M, d):
+    """The rotation in the paper's own structure (one matrix across blocks, one shared matrix inside them)
+    followed by the MXINT4 quantizer."""
+    cfg = I.CONFIGS["tiny"]
+    xb = I.activations(cfg, M=M, d=d)
+    g = np.random.Generator(np.random.PCG64(I.BASE_SEED + 78))
+    rbb = I.to_bf16_bits(I.orthogonal(d // 32, g))
+    ri = I.to_bf16_bits(I.orthogonal(32, g))
+    rows = np.arange(M) if M <= 256 else np.array([0, 1, 3, 4, 127, 128, 1000, 2046, 2047])
+    byt_t, s_t = torq.torq_rotate_quantize_structured_mxint4(dev_bf16(xb), dev_bf16(rbb), dev_bf16(ri))
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    g_q = _operand_to_int(byt_t[torch.from_numpy(rows).cuda()])
+    g_sb = O.unswizzle_scales(s_t.cpu().numpy(), M, d)[rows]
+    o_q, o_sb = O.quantize_mxint4(O.round_to_f32(O.rotate_structured(xb[rows], rbb, ri)))
+    rep = _mismatch(g_q, g_sb, o_q, o_sb)
+    assert rep["non_adjacent"] == 0 and rep["scale_off_by_more_than_one"] == 0, rep
+    n = rows.size * d
+    assert rep["elem"] * n <= max(2, 2e-4 * n) and rep["blocks"] * (n // 32) <= max(1, 2e-4 * (n // 32)), rep
+    buf = s_t.cpu().numpy().copy()                                       # padding of the scale tiles is zero
+    rr, cc = np.meshgrid(np.arange(M), np.arange(d // 32), indexing="ij")
+    buf[O.scale_layout_offset(rr, cc, d)] = 0
+    assert not buf.any()
