@@ -157,3 +157,27 @@ def test_fp4_peak_probe_reports_a_plausible_rate():
     rate = torq.torq_probe_fp4_peak(20000)
     assert torq.torq_last_device_error() == 0
     assert 1000.0 < rate < 9500.0, rate
+
+
+@pytest.mark.parametrize("M,N,K,dt", [(2300, 6200, 640, torch.float32), (2048, 6144, 384, torch.bfloat16),
+                                      (1100, 12296, 256, torch.float32)])
+def test_several_waves_of_tiles_with_ragged_edges_and_one_hot_rows(M, N, K, dt):
+    """Shapes with several waves of tiles per CTA pair (every pair walks two to four tiles, the last wave
+    partly empty), ragged M and N, K with and without a half last stage.  One-hot activation rows make every
+    output a single product: exact in fp32 and in bf16 after one rounding, so any mix-up of columns, rows of W,
+    scale tiles or store boxes shows up exactly; random rows in between exercise the accumulation."""
+    wc, wsb = _rand_operand(N, K, 21, 100, 150)
+    g = np.random.default_rng(22)
+    ac, asb = _rand_operand(M, K, 23, 100, 150)
+    hot_rows = np.arange(0, M, 3)
+    ac[hot_rows] = 0
+    ac[hot_rows, g.integers(0, K, size=hot_rows.size)] = g.integers(1, 16, size=hot_rows.size).astype(np.uint8)
+    ref = O.gemm_dequant(ac, asb, wc, wsb)
+    got = _gpu_gemm(ac, asb, wc, wsb, dt)
+    if dt == torch.bfloat16:
+        ref = O.round_to_bf16(ref)
+        assert (got[hot_rows] == ref[hot_rows]).all()
+        assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-3
+    else:
+        assert (got[hot_rows] == ref[hot_rows]).all()
+        assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
