@@ -76,3 +76,46 @@ def test_single_nonzero_element_with_permutation_rotations():
     assert np.array_equal(codes, o_codes) and np.array_equal(sb, o_sb)
     j = perm[100]
     assert codes[77, j] == 7 and sb[77, j // 32] == 126 and codes.sum() == 7 and sb.sum() == 126     # 3 = 6 * 2^-1
+
+
+@pytest.mark.parametrize("M", [1, 64, 300])
+def test_all_zero_activations_in_mxint4(M):
+    """The MXINT4 paths on all-zero activations: zero operand bytes, zero scale bytes, zero output; through
+    the dense rotation (single pass, or split for few tokens) and the structured one."""
+    d, N = 512, 256
+    rb, rib, _, g = _layer_operands(d, N)
+    xb = np.zeros((M, d), np.uint16)
+    wq = g.integers(-7, 8, (N, d)).astype(np.int8)
+    wsb = g.integers(120, 131, (N, d // 32), dtype=np.uint8)
+    dbg_b = torch.full((M, d), 0xAA, dtype=torch.uint8, device="cuda")
+    dbg_s = torch.full((torq.torq_scales_bytes(M, d),), 0xAA, dtype=torch.uint8, device="cuda")
+    y = torq.torq_rotated_linear_mxint4(dev_bf16(xb), dev_bf16(rb), dev_bf16(rib), dev_u8(O.int4_to_e4m3(wq)),
+                                        dev_u8(O.swizzle_scales(wsb, d, fill=0)), out_dtype=torch.float32,
+                                        dbg_bytes=dbg_b, dbg_scales=dbg_s)
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    assert not (dbg_b & 0x7F).any() and not dbg_s.any() and not y.any()      # a zero may carry a sign bit
+    rbb = I.to_bf16_bits(I.orthogonal(d // 32, np.random.default_rng(2)))
+    c, s = torq.torq_rotate_quantize_structured_mxint4(dev_bf16(xb), dev_bf16(rbb), dev_bf16(rib[0]))
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    assert not (c & 0x7F).any() and not s.any()
+
+
+def test_single_nonzero_element_in_mxint4():
+    """x = 3.0 at one position through a permutation: amax 3 gives e = -1 (scale byte 126) and the code 6 at
+    the permuted position (E4M3 byte 0x4C); everything else zero."""
+    M, d = 130, 256
+    g = np.random.default_rng(9)
+    x = np.zeros((M, d), np.float32)
+    x[77, 100] = 3.0
+    perm = g.permutation(d)
+    P = np.zeros((d, d), np.float32); P[np.arange(d), perm] = 1
+    b_t, s_t = torq.torq_rotate_quantize_mxint4(dev_bf16(I.to_bf16_bits(x)), dev_bf16(I.to_bf16_bits(P)), None)
+    torch.cuda.synchronize()
+    b = b_t.cpu().numpy()
+    sb = O.unswizzle_scales(s_t.cpu().numpy(), M, d)
+    j = perm[100]
+    assert b[77, j] == 0x4C and sb[77, j // 32] == 126
+    b[77, j] = 0
+    assert not (b & 0x7F).any() and sb.sum() == 126
