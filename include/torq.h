@@ -318,6 +318,16 @@ torq_status torq_givens_equalize(void* Sigma_f64, int64_t B, double eps, void* Q
  * groups >= 20000 (about a millisecond). */
 torq_status torq_probe_fp4_peak(int groups, double* tflops, void* stream);
 
+/* The same probe with background fills (no counterpart in the paper either): one warp of every CTA
+ * also streams 32 KiB per group from `src` (device memory, 16-byte aligned, src_bytes >= 32 KiB;
+ * pseudo-random 32-KiB chunks of it) into a ring of four shared-memory buffers that nothing reads.
+ * with_mma == 0 leaves the instruction stream out: *fill_gbps_per_sm (host pointer) is then the rate at
+ * which one SM takes data in (GB/s), *tflops 0.  with_mma != 0 runs both; the kernel ends when both are
+ * done, so the two numbers are what instructions and fills sustain side by side when nothing couples
+ * them.  Keep `src` within L2 (tens of MiB) to measure the L2 -> SM path rather than HBM. */
+torq_status torq_probe_fp4_peak_fills(int groups, const void* src, size_t src_bytes, int with_mma,
+                                      double* tflops, double* fill_gbps_per_sm, void* stream);
+
 const char* torq_status_string(torq_status s);
 
 /* Synchronises `stream`, then returns and clears the device error word of the current device:

@@ -889,21 +889,27 @@ torq_status torq_rotated_linear_static(const void* X, const void* R_inter, const
                              (size_t)TORQ_STATIC_WORKSPACE_BYTES, nullptr, nullptr, stream, /*allow_fused=*/false);
 }
 
-torq_status torq_probe_fp4_peak(int groups, double* tflops, void* stream) {
-  if (!tflops) return TORQ_ERR_NULL;
+static torq_status probe_impl(int groups, const void* src, size_t src_bytes, int with_mma, double* seconds, int* pairs_out,
+                              void* stream) {
   if (groups < 1 || groups > (1 << 24)) return TORQ_ERR_SHAPE;
+  if (src && (src_bytes < (size_t)Fp4ProbeCfg::FILL_BYTES || src_bytes / Fp4ProbeCfg::FILL_BYTES > 0x7FFFFFFFu))
+    return TORQ_ERR_SHAPE;
+  if (src && !aligned16(src)) return TORQ_ERR_ALIGN;
+  if (!src && !with_mma) return TORQ_ERR_NULL;
   DeviceState* st = device_state();
   if (!st) return TORQ_ERR_LAUNCH;
   if (!st->arch_ok) return TORQ_ERR_ARCH;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (!opt_in_smem(fp4_peak_probe_kernel, Fp4ProbeCfg::SMEM_BYTES)) return TORQ_ERR_LAUNCH;
+  const int smem = src ? Fp4ProbeCfg::SMEM_BYTES_FILLS : Fp4ProbeCfg::SMEM_BYTES;
+  if (!opt_in_smem(fp4_peak_probe_kernel, Fp4ProbeCfg::SMEM_BYTES_FILLS)) return TORQ_ERR_LAUNCH;
   const int pairs = st->gemm_pairs;
+  const unsigned chunks = src ? (unsigned)(src_bytes / Fp4ProbeCfg::FILL_BYTES) : 0u;
+  const uint8_t* sp = static_cast<const uint8_t*>(src);
   cudaEvent_t e0, e1;
   if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return TORQ_ERR_LAUNCH;
-  launch_tc(fp4_peak_probe_kernel, 2, 2 * pairs, Fp4ProbeCfg::THREADS, Fp4ProbeCfg::SMEM_BYTES, s, 64, st->err_word);
+  launch_tc(fp4_peak_probe_kernel, 2, 2 * pairs, Fp4ProbeCfg::THREADS, smem, s, 64, st->err_word, sp, chunks, with_mma);
   cudaEventRecord(e0, s);
-  launch_tc(fp4_peak_probe_kernel, 2, 2 * pairs, Fp4ProbeCfg::THREADS, Fp4ProbeCfg::SMEM_BYTES, s, groups,
-            st->err_word);
+  launch_tc(fp4_peak_probe_kernel, 2, 2 * pairs, Fp4ProbeCfg::THREADS, smem, s, groups, st->err_word, sp, chunks, with_mma);
   cudaEventRecord(e1, s);
   g_launches.fetch_add(2, std::memory_order_relaxed);
   float ms = 0.f;
@@ -912,7 +918,30 @@ torq_status torq_probe_fp4_peak(int groups, double* tflops, void* stream) {
   cudaEventDestroy(e0);
   cudaEventDestroy(e1);
   if (!ok) return TORQ_ERR_LAUNCH;
-  *tflops = (double)pairs * groups * 4.0 * 2.0 * 256.0 * 256.0 * 64.0 / ((double)ms * 1e-3) / 1e12;
+  *seconds = (double)ms * 1e-3;
+  *pairs_out = pairs;
+  return TORQ_OK;
+}
+
+torq_status torq_probe_fp4_peak(int groups, double* tflops, void* stream) {
+  if (!tflops) return TORQ_ERR_NULL;
+  double sec = 0.0;
+  int pairs = 0;
+  const torq_status rc = probe_impl(groups, nullptr, 0, 1, &sec, &pairs, stream);
+  if (rc != TORQ_OK) return rc;
+  *tflops = (double)pairs * groups * 4.0 * 2.0 * 256.0 * 256.0 * 64.0 / sec / 1e12;
+  return TORQ_OK;
+}
+
+torq_status torq_probe_fp4_peak_fills(int groups, const void* src, size_t src_bytes, int with_mma, double* tflops,
+                                      double* fill_gbps_per_sm, void* stream) {
+  if (!src || !tflops || !fill_gbps_per_sm) return TORQ_ERR_NULL;
+  double sec = 0.0;
+  int pairs = 0;
+  const torq_status rc = probe_impl(groups, src, src_bytes, with_mma ? 1 : 0, &sec, &pairs, stream);
+  if (rc != TORQ_OK) return rc;
+  *tflops = with_mma ? (double)pairs * groups * 4.0 * 2.0 * 256.0 * 256.0 * 64.0 / sec / 1e12 : 0.0;
+  *fill_gbps_per_sm = (double)groups * Fp4ProbeCfg::FILL_BYTES / sec / 1e9;
   return TORQ_OK;
 }
 

@@ -95,6 +95,8 @@ def lib() -> ctypes.CDLL:
     L.torq_givens_equalize.restype = ci
     L.torq_probe_fp4_peak.argtypes = [ci, ctypes.POINTER(ctypes.c_double), vp]
     L.torq_probe_fp4_peak.restype = ci
+    L.torq_probe_fp4_peak_fills.argtypes = [ci, vp, sz, ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), vp]
+    L.torq_probe_fp4_peak_fills.restype = ci
     L.torq_status_string.argtypes = [ci]
     L.torq_status_string.restype = ctypes.c_char_p
     L.torq_last_device_error.argtypes = [vp]
@@ -274,6 +276,15 @@ def torq_probe_fp4_peak(groups: int = 40000, stream=None) -> float:
     out = ctypes.c_double(0.0)
     _raise(lib().torq_probe_fp4_peak(groups, ctypes.byref(out), _stream(stream)), "torq_probe_fp4_peak")
     return out.value
+
+
+def torq_probe_fp4_peak_fills(src, with_mma: bool = True, groups: int = 40000, stream=None):
+    """The FP4 probe with background fills from `src` (uint8 device tensor).  Returns (TFLOP/s, fill GB/s per SM)."""
+    _check(src, torch.uint8, "src")
+    t, g = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _raise(lib().torq_probe_fp4_peak_fills(groups, _ptr(src), src.numel(), 1 if with_mma else 0, ctypes.byref(t),
+                                           ctypes.byref(g), _stream(stream)), "torq_probe_fp4_peak_fills")
+    return t.value, g.value
 
 
 def torq_swizzle_scales(linear, k: int, out=None, stream=None):

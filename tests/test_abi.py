@@ -122,3 +122,14 @@ def test_mxint4_argument_errors_and_sizes():
     assert L.torq_rotated_linear_mxint4(one, one, one, one, one, 4, 128, 8, one, 0, one, 16, None, None, None) == 7
     assert L.torq_rotated_linear_mxint4(one, None, one, one, one, 4, 128, 8, one, 0, one, 1 << 20, None, None,
                                         None) == 1
+
+
+def test_probe_argument_errors():
+    L = torq.lib()
+    one = ctypes.c_void_p(16)
+    d = ctypes.c_double(0.0)
+    assert L.torq_probe_fp4_peak(100, None, None) == 1
+    assert L.torq_probe_fp4_peak_fills(100, None, 1 << 20, 1, ctypes.byref(d), ctypes.byref(d), None) == 1
+    assert L.torq_probe_fp4_peak_fills(100, one, 1000, 1, ctypes.byref(d), ctypes.byref(d), None) == 2      # < 32 KiB
+    assert L.torq_probe_fp4_peak_fills(0, one, 1 << 20, 1, ctypes.byref(d), ctypes.byref(d), None) == 2
+    assert L.torq_probe_fp4_peak_fills(100, ctypes.c_void_p(24), 1 << 20, 1, ctypes.byref(d), ctypes.byref(d), None) == 3
