@@ -91,3 +91,40 @@ def test_token_sweep_at_hidden_5120():
     for M in I.SWEEP_M:
         rows = np.arange(M) if M <= 64 else _edge_rows(M)
         _check_layer(cfg, M, *ops, rows=rows, cols=np.arange(cfg.N))
+
+
+def test_llama3_down_projection_shape_in_mxint4_sampled_rows():
+    """The MXINT4 variant at the down-projection shape (2048 x 14336 -> 4096: 224 K steps in the rotation, 112 in
+    the FP8-rate GEMM): sampled rows of the quantized activations against the oracle, the GEMM on the GPU's own
+    codes for those rows, all columns."""
+    cfg = I.CONFIGS["llama3_8b_down"]
+    rb, rib, _, _ = I.rotations(cfg, device="cuda")
+    Rd, Rid = dev_bf16(rb), dev_bf16(rib)
+    Wn, W8, Ws = torq.prepare_weights_mxint4(Rd, Rid, torch.from_numpy(I.weights(cfg)).cuda())
+    xb = I.activations(cfg)
+    M, d, N = cfg.M, cfg.d, cfg.N
+    dbg_b = torch.empty((M, d), dtype=torch.uint8, device="cuda")
+    dbg_s = torch.empty(torq.torq_scales_bytes(M, d), dtype=torch.uint8, device="cuda")
+    y = torq.torq_rotated_linear_mxint4(dev_bf16(xb), Rd, Rid, W8, Ws, out_dtype=torch.bfloat16, dbg_bytes=dbg_b,
+                                        dbg_scales=dbg_s)
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    rows = np.unique(np.array(_edge_rows(M)))
+    tr = torch.from_numpy(rows).cuda()
+    g_q = O.e4m3_to_int4(dbg_b[tr].cpu().numpy())
+    g_sb = O.unswizzle_scales(dbg_s.cpu().numpy(), M, d)[rows]
+    o_q, o_sb = O.quantize_mxint4(O.round_to_f32(O.rotate(xb[rows], rb, rib)))
+    same = g_sb == o_sb
+    diff = (g_q != o_q) & np.repeat(same, 32, axis=1)
+    assert (np.abs(g_q.astype(np.int64) - o_q)[diff] <= 1).all()
+    assert (np.abs(g_sb.astype(np.int64) - o_sb.astype(np.int64)) <= 1).all()
+    assert diff.sum() <= max(1e-4 * g_q.size, 1.5) and (~same).sum() <= max(1e-4 * same.size, 1.5)
+    w_q = O.unpack_int4(Wn.cpu().numpy())
+    assert np.array_equal(O.e4m3_to_int4(W8.cpu().numpy()), w_q)
+    w_sb = O.unswizzle_scales(Ws.cpu().numpy(), N, d)
+    want = O.round_to_bf16(O.gemm_mxint4(g_q, g_sb, w_q, w_sb))
+    got = y[tr].float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) <= 1e-3
+    ulp = np.ldexp(1.0, np.frexp(np.maximum(np.abs(want), 1e-30))[1] - 8)
+    assert (np.abs(got - want) <= ulp).all()
