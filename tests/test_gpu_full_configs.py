@@ -128,3 +128,48 @@ def test_llama3_down_projection_shape_in_mxint4_sampled_rows():
     assert np.linalg.norm(got - want) / np.linalg.norm(want) <= 1e-3
     ulp = np.ldexp(1.0, np.frexp(np.maximum(np.abs(want), 1e-30))[1] - 8)
     assert (np.abs(got - want) <= ulp).all()
+
+
+def test_llama3_down_projection_shape_in_nvfp4_sampled_rows():
+    """The NVFP4 variant at the down-projection shape (2048 x 14336 -> 4096): sampled rows of the quantized
+    activations against the oracle (at most 1e-4 of the elements one lattice step off, at most 1e-3 of the block
+    scales one E4M3 step off at this depth of accumulation), the GEMM on the GPU's own codes for those rows, all columns."""
+    cfg = I.CONFIGS["llama3_8b_down"]
+    rb, _, _, _ = I.rotations(cfg, device="cuda")
+    ri16 = I.intra_rotations16(cfg)
+    Rd = dev_bf16(rb)
+    Ri32 = torq.torq_expand_intra16(dev_bf16(ri16))
+    torch.cuda.synchronize()
+    Wq, Ws, w_ts = torq.prepare_weights_nvfp4(Rd, Ri32, torch.from_numpy(I.weights(cfg)).cuda())
+    xb = I.activations(cfg)
+    M, d, N = cfg.M, cfg.d, cfg.N
+    rows = np.unique(np.array(_edge_rows(M)))
+    z = O.rotate_blocks(xb[rows], rb, ri16)
+    x_ts = np.float32(np.abs(z).max() / (6 * 448) * 2)          # a calibrated-style scale, not this sample's own
+    dbg_c = torch.empty((M, d // 2), dtype=torch.uint8, device="cuda")
+    dbg_s = torch.empty(torq.torq_nvfp4_scales_bytes(M, d), dtype=torch.uint8, device="cuda")
+    y = torq.torq_rotated_linear_nvfp4(dev_bf16(xb), Rd, Ri32, float(x_ts), Wq, Ws, float(w_ts),
+                                       out_dtype=torch.bfloat16, dbg_codes=dbg_c, dbg_scales=dbg_s)
+    torch.cuda.synchronize()
+    assert torq.torq_last_device_error() == 0
+    tr = torch.from_numpy(rows).cuda()
+    g_codes = O.unpack_codes(dbg_c[tr].cpu().numpy())
+    g_sb = O.nv_unswizzle_scales(dbg_s.cpu().numpy(), M, d)[rows]
+    o_codes, o_sb = O.quantize_nvfp4(z.astype(np.float32), x_ts)
+    same = g_sb == o_sb
+    lat = lambda c: np.where(c & 8, -(c & 7).astype(np.int64), (c & 7).astype(np.int64))
+    diff = (lat(g_codes) != lat(o_codes)) & np.repeat(same, 16, axis=1)
+    assert (np.abs(lat(g_codes) - lat(o_codes))[diff] <= 1).all()
+    assert (np.abs(g_sb.astype(np.int64) - o_sb.astype(np.int64)) <= 1).all()
+    # The E4M3 scale has eight rounding thresholds per octave of the block maximum (the E8M0 one has one), and the
+    # fp32 accumulation runs over 14336 terms here: a block maximum within ~1e-5 relative of a threshold may land on
+    # the other side, so up to 1e-3 of the blocks may carry the neighbouring scale byte (observed 2e-4).
+    assert diff.sum() <= max(1e-4 * g_codes.size, 1.5) and (~same).sum() <= max(1e-3 * same.size, 1.5)
+    w_codes = O.unpack_codes(Wq.cpu().numpy())
+    w_sb = O.nv_unswizzle_scales(Ws.cpu().numpy(), N, d)
+    want = O.round_to_bf16(O.gemm_nvfp4(g_codes, g_sb, x_ts, w_codes, w_sb, np.float32(w_ts)))
+    got = y[tr].float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) <= 1e-3
+    ulp = np.ldexp(1.0, np.frexp(np.maximum(np.abs(want), 1e-30))[1] - 8)
+    assert (np.abs(got - want) <= ulp).all()
