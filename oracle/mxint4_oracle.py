@@ -28,7 +28,7 @@ from __future__ import annotations
 
 import numpy as np
 
-from .torq_oracle import K_BLOCK, decode_bf16, merged_rotation, rotate, round_to_f32, shared_exponent
+from .torq_oracle import K_BLOCK, merged_rotation, rotate, round_to_f32, shared_exponent
 from .nvfp4_oracle import e4m3_value
 
 INT4_MAX = 7
