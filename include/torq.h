@@ -108,9 +108,11 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
 /* Algorithm 3 steps 1-5 in one call: rotate, quantize, multiply.  The quantized activations live
  * in `workspace` (>= torq_workspace_bytes(M, d, N) bytes, 256-byte aligned), laid out as codes
  * [M, d/2] followed (256-byte aligned) by the tiled scales; pass dbg_codes / dbg_scales non-NULL
- * to also receive copies of them.  For M <= 128 the workspace also holds fp32 partial tiles: the
- * rotation is then split along its contraction so that every SM streams a share of R_inter, and
- * a second kernel adds the partials in a fixed order before the intra-block step and Eq. 1.
+ * to also receive copies of them.  When the rotation has few output tiles (128 rows x 256 columns
+ * each) relative to the number of SMs -- few tokens, or a narrow layer -- the workspace also holds
+ * fp32 partial tiles: the rotation is then split along its contraction so that every SM streams a
+ * share of R_inter, and a second kernel adds the partials in a fixed order before the intra-block
+ * step and Eq. 1.
  * For many tokens (three or more waves of rotation tiles, N <= 2 d) both steps run as ONE persistent
  * kernel launched cooperatively, whose GEMM tiles start as soon as the row tile they read is quantized;
  * the workspace then also holds a block of counters that the call zeroes itself.
@@ -179,6 +181,30 @@ torq_status torq_swizzle_scales(const void* linear_scales, int64_t rows, int64_t
 torq_status torq_merge_rotations(const void* R_inter, const void* R_intra, int64_t d,
                                  void* R_merged_f32, void* stream);
 
+/* The same merged matrix rounded once (nearest even) to bfloat16: the operand of the one-GEMM form
+ * of the rotation, torq_rotate_quantize(X, R_merged, NULL), which Section 5 writes as
+ * R = R_inter (x) R_intra.  That form is a different quantized operator from the two-level one (the
+ * rounding of R~ to bfloat16 moves about one code in a thousand). */
+torq_status torq_merge_rotations_bf16(const void* R_inter, const void* R_intra, int64_t d,
+                                      void* R_merged_bf16, void* stream);
+
+/* Algorithm 3 step 5, option B ("weight fusion"), the offline weight side: W' = R~^T W with
+ * R~ = R_inter . blockdiag(R_intra), stored as [N, d] (K = d contiguous), then quantized along K
+ * (Section 6.1: weights and activations are both quantized).
+ *   W        [d, N] float32 row-major (out = x W)
+ *   R_inter  [d, d] bf16 (required), R_intra [d/32, 32, 32] bf16 or NULL = identity
+ *   Wq [N, d/2] u8, Ws torq_scales_bytes(N, d) bytes: the operands torq_mxfp4_gemm takes
+ *   workspace: torq_prepare_weights_workspace_bytes(d, N) bytes (10 N d, rounded up), 256-byte aligned
+ * Row n of W' is (W^T[n, :] R_inter) R_intra per block, i.e. steps 2-3 applied to the rows of W^T:
+ * W^T is split exactly into three bfloat16 terms and the rotation kernels contract all of them against
+ * R_inter in one fp32 accumulation on the tensor cores (every product exact); the intra-block step
+ * is fp32 FMAs; the result is quantized by the kernel behind torq_quantize_mxfp4.  d % 64 == 0.
+ * Three launches (split, rotation, quantizer).  Not on the inference path. */
+size_t torq_prepare_weights_workspace_bytes(int64_t d, int64_t N);
+torq_status torq_prepare_weights(const void* W, const void* R_inter, const void* R_intra, int64_t d,
+                                 int64_t N, void* Wq, void* Ws, void* workspace, size_t workspace_bytes,
+                                 void* stream);
+
 /* ---- NVFP4 variant (the paper's format study, Section 6 "Generalizability to Other Formats") -----
  * The same layer with NVFP4 operands: e2m1 codes as above, blocks of 16 along K, one FP8 E4M3
  * scale byte per (row, block) and one float32 scale per tensor; x^ = codeword * e4m3(byte) *
@@ -200,6 +226,15 @@ size_t torq_nvfp4_workspace_bytes(int64_t M, int64_t d, int64_t N);
 /* R_intra16 [d/16, 16, 16] bf16 -> R_intra32 [d/32, 32, 32] bf16: blocks 2b and 2b+1 on the diagonal of
  * block b, zeros elsewhere.  d % 32 == 0. */
 torq_status torq_expand_intra16(const void* R_intra16, int64_t d, void* R_intra32, void* stream);
+
+/* torq_prepare_weights in NVFP4 (R_intra32 as for torq_rotate_quantize_nvfp4).  The tensor scale is
+ * max |W'| / (6 * 448) (one float32 division), found by a reduction on the device and written to
+ * *tensor_scale (HOST pointer): this call therefore synchronises `stream` once, between the
+ * rotation and the quantization.  An all-zero W' has no scale: TORQ_ERR_SHAPE.
+ * Ws: torq_nvfp4_scales_bytes(N, d) bytes. */
+torq_status torq_prepare_weights_nvfp4(const void* W, const void* R_inter, const void* R_intra32, int64_t d,
+                                       int64_t N, void* Wq, void* Ws, float* tensor_scale, void* workspace,
+                                       size_t workspace_bytes, void* stream);
 
 /* Quantize Z [M, d] (fp32 or bf16) to NVFP4; d % 16 == 0.  Bit-exact by the definition above. */
 torq_status torq_quantize_nvfp4(const void* Z, torq_dtype z_dtype, int64_t M, int64_t d,
@@ -251,6 +286,12 @@ torq_status torq_rotated_linear_nvfp4(const void* X, const void* R_inter, const 
  * The rotation entry points write the operand form directly.  All pointers device, 16-byte
  * aligned; errors as elsewhere in this header.  The paper has no worked example of this format. */
 size_t torq_mxint4_workspace_bytes(int64_t M, int64_t d, int64_t N);
+
+/* torq_prepare_weights in MXINT4: Wn [N, d/2] stored form and / or W8 [N, d] operand form (either
+ * may be NULL, not both), Ws torq_scales_bytes(N, d) bytes. */
+torq_status torq_prepare_weights_mxint4(const void* W, const void* R_inter, const void* R_intra, int64_t d,
+                                        int64_t N, void* Wn, void* W8, void* Ws, void* workspace,
+                                        size_t workspace_bytes, void* stream);
 
 /* Quantize Z [M, d] (fp32 or bf16), d % 32 == 0.  packed != 0: stored form, out_codes [M, d/2];
  * packed == 0: operand form, out_codes [M, d].  out_scales: torq_scales_bytes(M, d) bytes. */
@@ -318,15 +359,17 @@ torq_status torq_givens_equalize(void* Sigma_f64, int64_t B, double eps, void* Q
  * groups >= 20000 (about a millisecond). */
 torq_status torq_probe_fp4_peak(int groups, double* tflops, void* stream);
 
-/* The same probe with background fills (no counterpart in the paper either): one warp of every CTA
- * also streams 32 KiB per group from `src` (device memory, 16-byte aligned, src_bytes >= 32 KiB;
- * pseudo-random 32-KiB chunks of it) into a ring of four shared-memory buffers that nothing reads.
- * with_mma == 0 leaves the instruction stream out: *fill_gbps_per_sm (host pointer) is then the rate at
- * which one SM takes data in (GB/s), *tflops 0.  with_mma != 0 runs both; the kernel ends when both are
- * done, so the two numbers are what instructions and fills sustain side by side when nothing couples
- * them.  Keep `src` within L2 (tens of MiB) to measure the L2 -> SM path rather than HBM. */
-torq_status torq_probe_fp4_peak_fills(int groups, const void* src, size_t src_bytes, int with_mma,
-                                      double* tflops, double* fill_gbps_per_sm, void* stream);
+/* Self-test of the bounded device waits (no counterpart in the paper).  Every wait inside the
+ * tensor-core kernels gives up after 2 s, latches TORQ_ERR_TIMEOUT, lets the kernel's other warps
+ * drain and returns; a healthy run never takes that path.  This call runs it on purpose in a
+ * one-CTA kernel whose two barriers nothing ever arrives on: one warp's wait runs out after
+ * `limit_ns` (1 us .. 100 ms) and latches the error word with wait-site id 7, the other warp's wait
+ * (2 s limit) must leave through the CTA's abort flag.  Nothing faults or hangs: the waits give up
+ * by design, and the context stays usable.
+ *   result_u64x3: three device uint64: [0] = 1 if the first wait gave up by itself, [1] = 1 if the
+ *   second left through the abort flag, [2] = nanoseconds the second one waited.
+ * Afterwards torq_last_device_error() returns TORQ_ERR_TIMEOUT | 7 << 8 (and clears the word). */
+torq_status torq_selftest_wait_timeout(uint64_t limit_ns, void* result_u64x3, void* stream);
 
 const char* torq_status_string(torq_status s);
 

@@ -25,11 +25,20 @@ What the paper leaves open is fixed here, each point a reading:
   * scale bytes live in the same 128-row x 4-column tiled layout as the MXFP4 scales, with
     K/16 columns.
 
+  * the format's plain definition, without any float32 step, is `quantize_nvfp4_exact`:
+        byte = E4M3(amax_block / (6 * tensor_scale)),  code = e2m1(z / (e4m3(byte) * tensor_scale))
+    in float64.  The float32 recipe above is that definition up to its own roundings (three per
+    decision, each 2^-24 relative): a decision can differ only for a value within about 2^-22
+    relative of a rounding threshold, and then by one step.  A test measures it.
+
 Pins (tests/test_oracle_nvfp4.py): the E4M3 table and encoder against ml_dtypes' float8_e4m3fn
 over every bit pattern and around every rounding threshold; hand-worked blocks whose arithmetic
 is exact (tensor scale a power of two); error bound |a - Q(a)| <= 1 code unit; idempotence;
-a tiny GEMM against exact rational arithmetic in pure Python.  The paper prints no worked
-example for this format: "parity unpinned" by the paper, pinned by the format's definition.
+a tiny GEMM against exact rational arithmetic in pure Python; the float32 recipe against the
+exact definition on heavy-tailed blocks with tensor scales that are not powers of two (every
+difference one step, at most a stated fraction), and against exact rational arithmetic on single
+blocks.  The paper prints no worked example for this format: "parity unpinned" by the paper,
+pinned by the format's definition.
 """
 from __future__ import annotations
 
@@ -42,7 +51,7 @@ E4M3_MAX = 448.0
 
 __all__ = [
     "NV_BLOCK", "E4M3_MAX", "e4m3_value", "encode_e4m3", "tensor_scale_from_amax", "rotate_blocks",
-    "quantize_nvfp4", "dequantize_nvfp4", "gemm_nvfp4", "nv_scale_layout_bytes", "nv_scale_layout_offset",
+    "quantize_nvfp4", "quantize_nvfp4_exact", "dequantize_nvfp4", "gemm_nvfp4", "nv_scale_layout_bytes", "nv_scale_layout_offset",
     "nv_swizzle_scales", "nv_unswizzle_scales", "expand_intra16", "prepare_weights_nvfp4",
     "rotated_linear_nvfp4",
 ]
@@ -136,6 +145,35 @@ def quantize_nvfp4(z32: np.ndarray, tensor_scale, rows_per_chunk: int = 256):
             r = np.where(byte == 0, np.float32(0.0), one / dec).astype(np.float32)
         a = (blk * r[..., None]).astype(np.float32)
         mag = _nearest_codeword(np.abs(a.astype(np.float64)))
+        sign = np.signbit(blk).astype(np.uint8)
+        codes[r0:r0 + rows_per_chunk] = ((sign << 3) | mag).reshape(-1, d)
+        sbytes[r0:r0 + rows_per_chunk] = byte
+    return codes, sbytes
+
+
+def quantize_nvfp4_exact(z32: np.ndarray, tensor_scale, rows_per_chunk: int = 256):
+    """The format's definition with no float32 step: per 16-element block
+        byte = E4M3(amax / (6 ts))   nearest, ties to the even byte, saturating at 448
+        code = e2m1(z / (e4m3(byte) ts))   nearest, ties to even, saturating at 6; sign of z
+    (a block whose scale byte is 0 encodes as zeros), every quotient one float64 division of
+    exactly represented operands (the tensor scale is the float32 value given).  Same outputs as
+    quantize_nvfp4."""
+    z32 = np.asarray(z32)
+    assert z32.dtype == np.float32 and z32.ndim == 2 and z32.shape[1] % NV_BLOCK == 0
+    ts = np.float64(np.float32(tensor_scale))
+    assert ts > 0 and np.isfinite(ts)
+    m, d = z32.shape
+    nb = d // NV_BLOCK
+    codes = np.empty((m, d), dtype=np.uint8)
+    sbytes = np.empty((m, nb), dtype=np.uint8)
+    for r0 in range(0, m, rows_per_chunk):
+        blk = z32[r0:r0 + rows_per_chunk].astype(np.float64).reshape(-1, nb, NV_BLOCK)
+        amax = np.abs(blk).max(axis=-1)
+        byte = encode_e4m3(amax / (6.0 * ts))
+        dec = e4m3_value(byte) * ts
+        with np.errstate(divide="ignore", invalid="ignore"):
+            a = np.where((byte == 0)[..., None], 0.0, np.abs(blk) / dec[..., None])
+        mag = _nearest_codeword(a)
         sign = np.signbit(blk).astype(np.uint8)
         codes[r0:r0 + rows_per_chunk] = ((sign << 3) | mag).reshape(-1, d)
         sbytes[r0:r0 + rows_per_chunk] = byte

@@ -5,12 +5,6 @@
 // warp keeps a few groups of four MMAs in flight, paced by tcgen05.commit on a ring of barriers as
 // the real kernel's pipeline is.  The result (flop / time) is the denominator the GEMM's roofline
 // fraction is quoted against when no vendor-measured FP4 peak is available.
-//
-// Two switches turn it into a second measurement: `src` != NULL makes warp 0 of every CTA stream
-// 32 KiB per group from global memory (1-D bulk copies, pseudo-random 32-KiB chunks of `src`) into a
-// ring of four shared-memory buffers that nobody reads, and `with_mma` = 0 leaves the instruction
-// stream out.  Fills alone give the rate at which an SM takes data in; fills beside the instructions
-// show what the two cost each other when nothing couples them.
 #pragma once
 #include "sm100_ptx.cuh"
 
@@ -22,14 +16,11 @@ struct Fp4ProbeCfg {
   static constexpr int SF_BYTES = 1024;
   static constexpr int RING = 6;
   static constexpr int SMEM_BYTES = A_BYTES + B_BYTES + SF_BYTES + 256 + 1024;
-  static constexpr int NF = 4, FILL_BYTES = 32768;     // background fills: ring of four 32-KiB buffers
-  static constexpr int SMEM_BYTES_FILLS = SMEM_BYTES + NF * FILL_BYTES;
   static constexpr int THREADS = 128;
 };
 
 // `groups` groups of four MMAs per CTA pair (each group = K 256 of a 256 x 256 tile).
-__global__ void __launch_bounds__(128, 1) fp4_peak_probe_kernel(int groups, int* err_word, const uint8_t* src,
-                                                                unsigned src_chunks, int with_mma) {
+__global__ void __launch_bounds__(128, 1) fp4_peak_probe_kernel(int groups, int* err_word) {
   using C = Fp4ProbeCfg;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -54,10 +45,7 @@ __global__ void __launch_bounds__(128, 1) fp4_peak_probe_kernel(int groups, int*
     }
     *reinterpret_cast<uint4*>(smem_gen + i) = make_uint4(w[0], w[1], w[2], w[3]);
   }
-  const uint32_t fill_base = bar_base + 256;            // behind the barrier block (only with `src`)
-  auto fill_bar = [&](int s) { return bar_base + 8u * (C::RING + s); };
   if (threadIdx.x == 0) {
-    for (int s = 0; s < C::NF; ++s) mbar_init(fill_bar(s), 1);
     for (int s = 0; s < C::RING; ++s) mbar_init(ring_bar(s), 1);
     *cta_abort = 0;
     fence_mbar_init();
@@ -70,30 +58,7 @@ __global__ void __launch_bounds__(128, 1) fp4_peak_probe_kernel(int groups, int*
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0 && src != nullptr) {
-    bool ok = true;
-    uint32_t h = blockIdx.x * 2654435761u + 12345u;
-    for (int gi = 0; gi < groups && ok; ++gi) {
-      const int s = gi % C::NF;                          // the copy that used this buffer last has landed
-      if (gi >= C::NF &&
-          !mbar_wait_warp(fill_bar(s), ((gi / C::NF - 1) & 1), cta_abort, err_word, SITE_PRODUCER_EMPTY)) {
-        ok = false; break;
-      }
-      h = h * 1664525u + 1013904223u;
-      if (elect_one()) {
-        mbar_arrive_expect_tx(fill_bar(s), C::FILL_BYTES);
-        bulk_load_1d(fill_base + s * C::FILL_BYTES, src + (size_t)((h >> 8) % src_chunks) * C::FILL_BYTES,
-                     C::FILL_BYTES, fill_bar(s));
-      }
-      __syncwarp();
-    }
-    for (int s = 0; s < C::NF && ok; ++s) {              // drain: the last copy into every buffer
-      const int last = ((groups - 1 - s) / C::NF) * C::NF + s;
-      if (last >= 0 && last < groups)
-        ok = mbar_wait_warp(fill_bar(s), (last / C::NF) & 1, cta_abort, err_word, SITE_TEARDOWN);
-    }
-  }
-  if (with_mma && warp == 1 && rank == 0) {
+  if (warp == 1 && rank == 0) {
     constexpr uint32_t idesc0 = idesc_mxf4(256, 256, 0, 0), idesc2 = idesc_mxf4(256, 256, 2, 2);
     const uint32_t sfa_t = tmem_base + 256, sfb_t = tmem_base + 264;
     const uint64_t adesc = make_desc(smem_base, 16, 1024, kSwizzle128);

@@ -270,10 +270,12 @@ __global__ void swizzle_scales_kernel(const uint8_t* __restrict__ lin, int64_t r
   }
 }
 
-// R~[i, 32b+j] = sum_t R_inter[i, 32b+t] * R_intra[b][t][j], fp32 (offline weight-side helper).
+// R~[i, 32b+j] = sum_t R_inter[i, 32b+t] * R_intra[b][t][j], fp32 FMAs in index order; stored as
+// float32, or rounded once (nearest even) to bfloat16.
+template <typename OutT>
 __global__ void merge_rotations_kernel(const __nv_bfloat16* __restrict__ R_inter,
                                        const __nv_bfloat16* __restrict__ R_intra, int64_t d,
-                                       float* __restrict__ out) {
+                                       OutT* __restrict__ out) {
   const int64_t total = d * d;
   for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
        t += (int64_t)gridDim.x * blockDim.x) {
@@ -282,7 +284,8 @@ __global__ void merge_rotations_kernel(const __nv_bfloat16* __restrict__ R_inter
     for (int tt = 0; tt < 32; ++tt)
       acc = fmaf(__bfloat162float(R_inter[i * d + b * 32 + tt]),
                  __bfloat162float(R_intra[b * 1024 + tt * 32 + j]), acc);
-    out[t] = acc;
+    if constexpr (sizeof(OutT) == 2) out[t] = __float2bfloat16_rn(acc);
+    else out[t] = acc;
   }
 }
 

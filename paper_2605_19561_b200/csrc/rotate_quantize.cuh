@@ -41,11 +41,15 @@ struct RotCfg {
 // FMT_NVFP4: NVFP4 quantizer in the epilogue (two 16-element blocks per 32 columns, E4M3 scales,
 // `tensor_scale` the tensor's float32 scale; unused for MXFP4).  FMT_MXINT4: integer codes as one
 // E4M3 operand byte per element (`codes` is [M, d] bytes), scale bytes as for MXFP4.
+// FMT_F32OUT: no quantizer; `codes` is a float32 [M, d] array that receives Z itself.  `x_terms` > 1:
+// X = the sum of that many bfloat16 matrices side by side in tmX = [M, x_terms * d], contracted
+// against the same R_inter in one fp32 accumulation (d % 64 == 0 then).
 template <int BN, int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(192, 1)
 rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
                        const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
-                       uint8_t* __restrict__ scales, int M, int d, float tensor_scale, int* err_word) {
+                       uint8_t* __restrict__ scales, int M, int d, float tensor_scale, int x_terms,
+                       int* err_word) {
   using C = RotCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -64,7 +68,8 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
   const int m_tiles = (M + C::BM - 1) / C::BM;
   const int n_tiles = (d + BN - 1) / BN;
   const int total_tiles = m_tiles * n_tiles;
-  const int k_tiles = (d + C::BK - 1) / C::BK;
+  const int kr_tiles = (d + C::BK - 1) / C::BK;         // K steps over R_inter; X has x_terms times as many
+  const int k_tiles = kr_tiles * x_terms;
   const int nblocks = d / 32;
   const int kb4 = (nblocks + 3) / 4;
 
@@ -90,7 +95,7 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int mt = tile % m_tiles, nt = tile / m_tiles;
-      for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+      for (int kt = 0, kr = 0; kt < k_tiles; ++kt, ++it, kr = (kr + 1 == kr_tiles ? 0 : kr + 1)) {
         const int s = it % C::STAGES;
         if (!mbar_wait_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
                        SITE_PRODUCER_EMPTY)) { ok = false; break; }
@@ -100,7 +105,7 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
           tma_load_2d(st, &tmX, kt * C::BK, mt * C::BM, full_bar(s));
 #pragma unroll
           for (int b = 0; b < BN / 64; ++b)
-            tma_load_2d(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR, nt * BN + b * 64, kt * C::BK,
+            tma_load_2d(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR, nt * BN + b * 64, kr * C::BK,
                         full_bar(s));
         }
         __syncwarp();
@@ -210,9 +215,17 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
 #pragma unroll
           for (int j = 0; j < 32; ++j) z[j] = __uint_as_float(yv[j]);
         }
+        const int blk = b0 + bb;
+        if constexpr (FMT == FMT_F32OUT) {                 // the rotated values themselves
+          if (row < M && blk < nblocks) {
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(codes) + row * (int64_t)d + (int64_t)blk * 32);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) dst[j] = make_float4(z[4 * j], z[4 * j + 1], z[4 * j + 2], z[4 * j + 3]);
+          }
+          continue;
+        }
         uint4 cw;
         uint32_t sbyte;
-        const int blk = b0 + bb;
         if constexpr (FMT == FMT_MXINT4) {                 // one operand byte per element
           uint4 cw2;
           mxint4_quantize_block32(z, cw, cw2, sbyte);

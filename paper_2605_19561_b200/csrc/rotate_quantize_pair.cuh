@@ -43,11 +43,16 @@ struct RotPairCfg {
 // is still [d/32, 32, 32]; 16-wide rotations arrive as its block-diagonal form.
 // FMT_MXINT4: integer codes written as one E4M3 operand byte per element (`codes` is [M, d] bytes),
 // the scale bytes as for MXFP4.
+// FMT_F32OUT: no quantizer; `codes` is a float32 [M, d] array that receives Z itself (`scales` unused).
+// `x_terms` > 1: X is the sum of that many bfloat16 matrices stored side by side, tmX = [M, x_terms * d]
+// (an fp32 matrix split exactly into three bf16 terms); the contraction then runs over all of them
+// against the same R_inter, i.e. Z = (X_0 + X_1 + ...) R_inter in one fp32 accumulation.  d % 64 == 0 then.
 template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(320, 1)
 rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
                             const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
-                            uint8_t* __restrict__ scales, int M, int d, float tensor_scale, int* err_word) {
+                            uint8_t* __restrict__ scales, int M, int d, float tensor_scale, int x_terms,
+                            int* err_word) {
   using C = RotPairCfg;
   constexpr int BN = C::BN;
   extern __shared__ uint8_t smem_raw[];
@@ -70,7 +75,8 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
   const int mp_tiles = (M + 255) / 256;                // 256-row pair tiles
   const int n_tiles = (d + BN - 1) / BN;
   const int total_tiles = mp_tiles * n_tiles;
-  const int k_tiles = (d + C::BK - 1) / C::BK;
+  const int kr_tiles = (d + C::BK - 1) / C::BK;         // K steps over R_inter; X has x_terms times as many
+  const int k_tiles = kr_tiles * x_terms;
   const int nblocks = d / 32;
   const int kb4 = (nblocks + 3) / 4;
 
@@ -106,7 +112,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
 #pragma unroll
         for (int b = 0; b < BN / 2 / 64; ++b)
           tma_load_2d_pair(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR,
-                           nt * BN + (int)rank * (BN / 2) + b * 64, kt * C::BK, leader_full);
+                           nt * BN + (int)rank * (BN / 2) + b * 64, (kt % kr_tiles) * C::BK, leader_full);
       }
     }
     __syncwarp();
@@ -121,7 +127,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
       int mp, nt;
       pair_tile_coords(tile, mp_tiles, n_tiles, mp, nt);
       const int mt = 2 * mp + (int)rank;
-      for (int kt = 0; kt < k_tiles; ++kt, ++it) {
+      for (int kt = 0, kr = 0; kt < k_tiles; ++kt, ++it, kr = (kr + 1 == kr_tiles ? 0 : kr + 1)) {
         const int s = it % C::STAGES;
         if (!mbar_wait_cluster_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
                                SITE_PRODUCER_EMPTY)) { ok = false; break; }
@@ -135,7 +141,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
 #pragma unroll
             for (int b = 0; b < BN / 2 / 64; ++b)
               tma_load_2d_pair(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR,
-                               nt * BN + (int)rank * (BN / 2) + b * 64, kt * C::BK, leader_full);
+                               nt * BN + (int)rank * (BN / 2) + b * 64, kr * C::BK, leader_full);
           }
         }
         __syncwarp();
@@ -198,7 +204,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
       const int mt = 2 * mp + (int)rank;
       const int a = tcount % C::NACC;
       const int b0 = nt * (BN / 32);
-      const bool last = tile + npairs >= total_tiles;
+      const bool last = FMT != FMT_F32OUT && tile + npairs >= total_tiles;
       if (R_intra != nullptr) {
         // Executed by every epilogue thread for every tile, also after a wait has given up.
         named_barrier_sync(1, 256);
@@ -252,9 +258,17 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
 #pragma unroll
             for (int j = 0; j < 32; ++j) z[j] = __uint_as_float(yv[j]);
           }
+          const int blk = b0 + h * 4 + bb;
+          if constexpr (FMT == FMT_F32OUT) {               // the rotated values themselves
+            if (row < M && blk < nblocks) {
+              float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(codes) + row * (int64_t)d + (int64_t)blk * 32);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) dst[j] = make_float4(z[4 * j], z[4 * j + 1], z[4 * j + 2], z[4 * j + 3]);
+            }
+            continue;
+          }
           uint4 cw;
           uint32_t sbyte;
-          const int blk = b0 + h * 4 + bb;
           if constexpr (FMT == FMT_MXINT4) {               // one operand byte per element
             uint4 cw2;
             mxint4_quantize_block32(z, cw, cw2, sbyte);
@@ -277,7 +291,9 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
             sc_word |= sbyte << (8 * bb);
           }
         }
-        if constexpr (FMT == FMT_NVFP4) {
+        if constexpr (FMT == FMT_F32OUT) {
+          continue;
+        } else if constexpr (FMT == FMT_NVFP4) {
           const int kb4n = (2 * nblocks + 3) / 4;        // 4-byte groups of 16-block scales per row
           if (mt < m_tiles) {
             if (2 * chunk < kb4n)

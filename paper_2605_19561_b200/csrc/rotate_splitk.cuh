@@ -231,12 +231,13 @@ splitk_reduce_quantize_kernel(const float* __restrict__ P, const __nv_bfloat16* 
 #pragma unroll 4
   for (int r = warp; r < rows; r += nwarps) {
     const float* p = P + (size_t)(row0 + r) * d + b * 32 + lane;
-    float part[8];
+    constexpr int MS = RotSplitCfg::MAX_SPLITS;          // every split's partial is loaded before the first add
+    float part[MS];
 #pragma unroll
-    for (int s = 0; s < 8; ++s) part[s] = s < splits ? __ldg(p + s * split_stride) : 0.f;
+    for (int s = 0; s < MS; ++s) part[s] = s < splits ? __ldg(p + s * split_stride) : 0.f;
     float y = 0.f;
 #pragma unroll
-    for (int s = 0; s < 8; ++s) if (s < splits) y += part[s];
+    for (int s = 0; s < MS; ++s) if (s < splits) y += part[s];
     y_s[r * 33 + lane] = y;
   }
   for (int r = rows + warp; r < 32; r += nwarps) y_s[r * 33 + lane] = 0.f;     // rows past M: zeros

@@ -12,7 +12,7 @@ namespace torq {
 // Low byte: status (6 = a bounded wait ran out); bits 8..15: id of the wait site.
 enum WaitSite : int {
   SITE_PRODUCER_EMPTY = 1, SITE_MMA_FULL = 2, SITE_MMA_ACC_EMPTY = 3, SITE_EPI_ACC_FULL = 4,
-  SITE_TEARDOWN = 5
+  SITE_TEARDOWN = 5, SITE_SELFTEST = 7
 };
 constexpr int kErrTimeout = 6;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
@@ -55,7 +55,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // when this wait itself exceeds kWaitLimitNs; in the latter case it latches the error word and
 // raises the CTA's abort flag so that every other role leaves its loop too.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* cta_abort,
-                                          int* err_word, int site) {
+                                          int* err_word, int site,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   unsigned long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
@@ -64,7 +65,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*cta_abort) return false;
       unsigned long long now = globaltimer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) {
+      else if (now - t0 > limit_ns) {
         *cta_abort = 1;
         atomicCAS(err_word, 0, kErrTimeout | (site << 8));
         return false;
@@ -308,8 +309,9 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
 // Whole-warp forms of the bounded waits: every lane waits, and all lanes agree on the outcome so
 // that the warp stays converged for the election that follows.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* cta_abort,
-                                               int* err_word, int site) {
-  return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, cta_abort, err_word, site));
+                                               int* err_word, int site,
+                                               unsigned long long limit_ns = kWaitLimitNs) {
+  return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, cta_abort, err_word, site, limit_ns));
 }
 
 // ---- CTA pairs (cluster of two CTAs driving one tcgen05 MMA with cta_group::2) -----------------
@@ -493,7 +495,8 @@ __host__ __device__ constexpr uint32_t idesc_mxf8(int M, int N, uint32_t sf_id) 
   return (sf_id << 4) | ((uint32_t)(N >> 3) << 17) | (1u << 23) | ((uint32_t)(M >> 4) << 24) | (sf_id << 29);
 }
 
-// The 4-bit block formats of the library.
-enum : int { FMT_MXFP4 = 0, FMT_NVFP4 = 1, FMT_MXINT4 = 2 };
+// The 4-bit block formats of the library.  FMT_F32OUT is not a format: the rotation kernels then
+// store the rotated values themselves as float32 (the offline weight side quantizes them afterwards).
+enum : int { FMT_MXFP4 = 0, FMT_NVFP4 = 1, FMT_MXINT4 = 2, FMT_F32OUT = 3 };
 
 }  // namespace torq

@@ -18,6 +18,8 @@
 #include "rotated_linear_fused.cuh"
 #include "fp4_peak_probe.cuh"
 #include "calibrate.cuh"
+#include "wait_selftest.cuh"
+#include "prepare_weights.cuh"
 #include "sm100_ptx.cuh"
 
 namespace torq {
@@ -31,7 +33,8 @@ struct DeviceState {
   int sm_count = 0;
   int rot_pairs = 0;    // CTA pairs of the pair kernels that can be resident at once
   int gemm_pairs = 0;
-  int fused_pairs = 0;  // CTA pairs of the one-kernel layer that can be resident at once; 0 = not usable
+  std::atomic<int> fused_pairs{0};  // CTA pairs of the one-kernel layer that can be resident at once; 0 = not usable
+                                    // (host threads may clear it while others read it)
   int* err_word = nullptr;
 };
 static DeviceState g_dev[kMaxDevices];
@@ -114,7 +117,9 @@ static DeviceState* device_state() {
               opt_in_smem(mxfp4_gemm_pair_kernel<FMT_MXINT4>, GemmPairCfgT<FMT_MXINT4>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_kernel<256, FMT_MXINT4>, RotCfg<256>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_pair_kernel<FMT_MXINT4>, RotPairCfg::SMEM_BYTES) &&
-              opt_in_smem(rotate_structured_kernel<FMT_MXINT4>, RotStructCfg::SMEM_BYTES);
+              opt_in_smem(rotate_structured_kernel<FMT_MXINT4>, RotStructCfg::SMEM_BYTES) &&
+              opt_in_smem(rotate_quantize_kernel<256, FMT_F32OUT>, RotCfg<256>::SMEM_BYTES) &&
+              opt_in_smem(rotate_quantize_pair_kernel<FMT_F32OUT>, RotPairCfg::SMEM_BYTES);
     if (!ok) return nullptr;
     st.rot_pairs = max_active_pairs(rotate_quantize_pair_kernel<FMT_MXFP4>, RotPairCfg::THREADS,
                                     RotPairCfg::SMEM_BYTES, st.sm_count);
@@ -291,14 +296,17 @@ torq_status torq_quantize_mxfp4(const void* Z, torq_dtype z_dtype, int64_t M, in
 
 // Steps 1-4.  `scratch` (may be NULL) is fp32 room for the split-K partials of the few-token path;
 // without enough of it the single-pass kernels run.  `fmt` FMT_NVFP4 (with its tensor scale) needs R_inter.
+// FMT_F32OUT: out_codes is float32 [M, d] and receives the rotated values (out_scales unused, may be
+// NULL); `x_terms` > 1: X is [M, x_terms * d], the sum of its d-wide column groups is what is rotated.
 static torq_status rotate_quantize_impl(const void* X, const void* R_inter, const void* R_intra, int64_t M,
                                         int64_t d, void* out_codes, void* out_scales, void* scratch,
                                         size_t scratch_bytes, void* stream, int fmt = FMT_MXFP4,
-                                        float tensor_scale = 0.0f) {
-  if (!X || !out_codes || !out_scales) return TORQ_ERR_NULL;
+                                        float tensor_scale = 0.0f, int x_terms = 1) {
+  if (!X || !out_codes || (!out_scales && fmt != FMT_F32OUT)) return TORQ_ERR_NULL;
   if (fmt != FMT_MXFP4 && !R_inter) return TORQ_ERR_NULL;
   if (M < 1 || d < 32 || d % 32 != 0 || M > (1 << 30) || d > (1 << 24)) return TORQ_ERR_SHAPE;
-  if (!aligned16(X) || !aligned16(out_codes) || !aligned16(out_scales) ||
+  if (x_terms < 1 || x_terms > 4 || (x_terms > 1 && d % 64 != 0)) return TORQ_ERR_SHAPE;
+  if (!aligned16(X) || !aligned16(out_codes) || (out_scales && !aligned16(out_scales)) ||
       (R_inter && !aligned16(R_inter)) || (R_intra && !aligned16(R_intra)))
     return TORQ_ERR_ALIGN;
   DeviceState* st = device_state();
@@ -316,10 +324,10 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
     return launch_status();
   }
   CUtensorMap tmX, tmR;
-  if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d, 128, 64) ||
+  if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d * x_terms, 128, 64) ||
       !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
     return TORQ_ERR_LAUNCH;
-  const int splits = rotation_splits(M, d, st->sm_count);
+  const int splits = (fmt == FMT_F32OUT || x_terms > 1) ? 1 : rotation_splits(M, d, st->sm_count);
   if (splits >= 2 && scratch && scratch_bytes >= splitk_scratch_bytes(M, d, splits) &&
       (reinterpret_cast<uintptr_t>(scratch) & 15u) == 0) {
     // Few tokens: split K over the SMs, partial tiles to scratch, then reduce + intra + quantize.
@@ -354,15 +362,19 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
     if (fmt == FMT_MXINT4)
       launch_tc(rotate_quantize_pair_kernel<FMT_MXINT4>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
                 s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
-                st->err_word);
+                x_terms, st->err_word);
     else if (fmt == FMT_NVFP4)
       launch_tc(rotate_quantize_pair_kernel<FMT_NVFP4>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
                 s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d,
-                tensor_scale, st->err_word);
+                tensor_scale, x_terms, st->err_word);
+    else if (fmt == FMT_F32OUT)
+      launch_tc(rotate_quantize_pair_kernel<FMT_F32OUT>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
+                s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
+                x_terms, st->err_word);
     else
       launch_tc(rotate_quantize_pair_kernel<FMT_MXFP4>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
                 s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
-                st->err_word);
+                x_terms, st->err_word);
     return launch_status();
   }
   const int m_tiles = (int)((M + 127) / 128);
@@ -371,14 +383,19 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
   if (fmt == FMT_MXINT4)
     launch_tc(rotate_quantize_kernel<256, FMT_MXINT4>, 1, grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s,
               tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
-              st->err_word);
+              x_terms, st->err_word);
   else if (fmt == FMT_NVFP4)
     launch_tc(rotate_quantize_kernel<256, FMT_NVFP4>, 1, grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s,
               tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, tensor_scale,
-              st->err_word);
+              x_terms, st->err_word);
+  else if (fmt == FMT_F32OUT)
+    launch_tc(rotate_quantize_kernel<256, FMT_F32OUT>, 1, grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s,
+              tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
+              x_terms, st->err_word);
   else
     launch_tc(rotate_quantize_kernel<256>, 1, grid, RotCfg<256>::THREADS, RotCfg<256>::SMEM_BYTES, s, tmX, tmR,
-              static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f, st->err_word);
+              static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f, x_terms,
+              st->err_word);
   return launch_status();
 }
 
@@ -717,7 +734,8 @@ static torq_status fused_layer(const void* X, const void* R_inter, const void* R
                                uint8_t* codes, uint8_t* scales, int* counters, void* stream, bool* done) {
   *done = false;
   DeviceState* st = device_state();
-  if (!st || !st->arch_ok || st->fused_pairs < 1) return TORQ_OK;
+  const int fused_pairs = st ? st->fused_pairs.load(std::memory_order_relaxed) : 0;
+  if (!st || !st->arch_ok || fused_pairs < 1) return TORQ_OK;
   const int64_t mp_tiles = (M + 255) / 256;
   if (M <= 128 || !R_inter || mp_tiles > kFusedMaxRowTiles || (size_t)d * (size_t)d * 2 > (size_t)(64u << 20) ||
       rotation_splits(M, d, st->sm_count) >= 2 || M > (1 << 30) || N > (1 << 30) || d > (1 << 24))
@@ -731,7 +749,7 @@ static torq_status fused_layer(const void* X, const void* R_inter, const void* R
   // pair's last runs beside the next mainloop and takes most of it, so a row tile is complete about
   // one tile time after its last mainloop: with two waves (2048 x 4096: measured 77 us against 72.5 us
   // for the two kernels) the pairs that skip the second wave would still find no finished row.
-  if (rot_tiles < 3 * (int64_t)st->fused_pairs) return TORQ_OK;
+  if (rot_tiles < 3 * (int64_t)fused_pairs) return TORQ_OK;
   // ... and while the GEMM is not the bulk of the work: its tiles are dealt out row tile by row tile
   // here, which re-streams W for every row tile (8192 x 5120 -> 25600: 759 us against 689 us).
   if (N > 2 * d) return TORQ_OK;
@@ -752,7 +770,7 @@ static torq_status fused_layer(const void* X, const void* R_inter, const void* R
     return TORQ_OK;
   if (cudaMemsetAsync(counters, 0, (size_t)mp_tiles * sizeof(int), s) != cudaSuccess) return TORQ_OK;
   const int64_t most = rot_tiles > gemm_tiles ? rot_tiles : gemm_tiles;
-  const int pairs = (int)(most < st->fused_pairs ? most : st->fused_pairs);
+  const int pairs = (int)(most < fused_pairs ? most : (int64_t)fused_pairs);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
   cfg.blockDim = dim3((unsigned)FusedCfg::THREADS, 1, 1);
@@ -883,33 +901,29 @@ torq_status torq_rotated_linear_static(const void* X, const void* R_inter, const
   if (M < 1 || d < 128 || d % 128 != 0 || N < 8 || N % 8 != 0 || M > (1 << 30) || d > (1 << 24))
     return TORQ_ERR_SHAPE;
   if (quantized_bytes(M, d) > (size_t)TORQ_STATIC_WORKSPACE_BYTES) return TORQ_ERR_WORKSPACE;
+  DeviceState* st = device_state();                // architecture first: another device has no image of the array
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
   void* scratch = static_workspace_address();
   if (!scratch) return TORQ_ERR_LAUNCH;
   return rotated_linear_impl(X, R_inter, R_intra, Wq, Ws, M, d, N, Y, y_dtype, scratch,
                              (size_t)TORQ_STATIC_WORKSPACE_BYTES, nullptr, nullptr, stream, /*allow_fused=*/false);
 }
 
-static torq_status probe_impl(int groups, const void* src, size_t src_bytes, int with_mma, double* seconds, int* pairs_out,
-                              void* stream) {
+torq_status torq_probe_fp4_peak(int groups, double* tflops, void* stream) {
+  if (!tflops) return TORQ_ERR_NULL;
   if (groups < 1 || groups > (1 << 24)) return TORQ_ERR_SHAPE;
-  if (src && (src_bytes < (size_t)Fp4ProbeCfg::FILL_BYTES || src_bytes / Fp4ProbeCfg::FILL_BYTES > 0x7FFFFFFFu))
-    return TORQ_ERR_SHAPE;
-  if (src && !aligned16(src)) return TORQ_ERR_ALIGN;
-  if (!src && !with_mma) return TORQ_ERR_NULL;
   DeviceState* st = device_state();
   if (!st) return TORQ_ERR_LAUNCH;
   if (!st->arch_ok) return TORQ_ERR_ARCH;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const int smem = src ? Fp4ProbeCfg::SMEM_BYTES_FILLS : Fp4ProbeCfg::SMEM_BYTES;
-  if (!opt_in_smem(fp4_peak_probe_kernel, Fp4ProbeCfg::SMEM_BYTES_FILLS)) return TORQ_ERR_LAUNCH;
+  if (!opt_in_smem(fp4_peak_probe_kernel, Fp4ProbeCfg::SMEM_BYTES)) return TORQ_ERR_LAUNCH;
   const int pairs = st->gemm_pairs;
-  const unsigned chunks = src ? (unsigned)(src_bytes / Fp4ProbeCfg::FILL_BYTES) : 0u;
-  const uint8_t* sp = static_cast<const uint8_t*>(src);
   cudaEvent_t e0, e1;
   if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return TORQ_ERR_LAUNCH;
-  launch_tc(fp4_peak_probe_kernel, 2, 2 * pairs, Fp4ProbeCfg::THREADS, smem, s, 64, st->err_word, sp, chunks, with_mma);
+  launch_tc(fp4_peak_probe_kernel, 2, 2 * pairs, Fp4ProbeCfg::THREADS, Fp4ProbeCfg::SMEM_BYTES, s, 64, st->err_word);
   cudaEventRecord(e0, s);
-  launch_tc(fp4_peak_probe_kernel, 2, 2 * pairs, Fp4ProbeCfg::THREADS, smem, s, groups, st->err_word, sp, chunks, with_mma);
+  launch_tc(fp4_peak_probe_kernel, 2, 2 * pairs, Fp4ProbeCfg::THREADS, Fp4ProbeCfg::SMEM_BYTES, s, groups, st->err_word);
   cudaEventRecord(e1, s);
   g_launches.fetch_add(2, std::memory_order_relaxed);
   float ms = 0.f;
@@ -918,31 +932,20 @@ static torq_status probe_impl(int groups, const void* src, size_t src_bytes, int
   cudaEventDestroy(e0);
   cudaEventDestroy(e1);
   if (!ok) return TORQ_ERR_LAUNCH;
-  *seconds = (double)ms * 1e-3;
-  *pairs_out = pairs;
+  *tflops = (double)pairs * groups * 4.0 * 2.0 * 256.0 * 256.0 * 64.0 / ((double)ms * 1e-3) / 1e12;
   return TORQ_OK;
 }
 
-torq_status torq_probe_fp4_peak(int groups, double* tflops, void* stream) {
-  if (!tflops) return TORQ_ERR_NULL;
-  double sec = 0.0;
-  int pairs = 0;
-  const torq_status rc = probe_impl(groups, nullptr, 0, 1, &sec, &pairs, stream);
-  if (rc != TORQ_OK) return rc;
-  *tflops = (double)pairs * groups * 4.0 * 2.0 * 256.0 * 256.0 * 64.0 / sec / 1e12;
-  return TORQ_OK;
-}
-
-torq_status torq_probe_fp4_peak_fills(int groups, const void* src, size_t src_bytes, int with_mma, double* tflops,
-                                      double* fill_gbps_per_sm, void* stream) {
-  if (!src || !tflops || !fill_gbps_per_sm) return TORQ_ERR_NULL;
-  double sec = 0.0;
-  int pairs = 0;
-  const torq_status rc = probe_impl(groups, src, src_bytes, with_mma ? 1 : 0, &sec, &pairs, stream);
-  if (rc != TORQ_OK) return rc;
-  *tflops = with_mma ? (double)pairs * groups * 4.0 * 2.0 * 256.0 * 256.0 * 64.0 / sec / 1e12 : 0.0;
-  *fill_gbps_per_sm = (double)groups * Fp4ProbeCfg::FILL_BYTES / sec / 1e9;
-  return TORQ_OK;
+torq_status torq_selftest_wait_timeout(uint64_t limit_ns, void* result_u64x3, void* stream) {
+  if (!result_u64x3) return TORQ_ERR_NULL;
+  if (limit_ns < 1000ull || limit_ns > 100000000ull) return TORQ_ERR_SHAPE;        // 1 us .. 100 ms
+  if (!aligned16(result_u64x3)) return TORQ_ERR_ALIGN;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(
+      (unsigned long long)limit_ns, st->err_word, static_cast<unsigned long long*>(result_u64x3));
+  return launch_status();
 }
 
 torq_status torq_block_covariance(const void* X, int64_t T, int64_t d, void* Sigma_f64, void* stream) {
@@ -985,6 +988,95 @@ torq_status torq_swizzle_scales(const void* linear_scales, int64_t rows, int64_t
   return launch_status();
 }
 
+// ---- offline weight side (Algorithm 3 step 5, option B) ------------------------------------------
+// Workspace: the three-term bf16 split of W^T [N, 3 d], then (256-byte aligned) W' as float32 [N, d].
+static size_t prep_split_bytes(int64_t d, int64_t N) { return ((size_t)N * (size_t)d * 6 + 255) / 256 * 256; }
+
+size_t torq_prepare_weights_workspace_bytes(int64_t d, int64_t N) {
+  if (d <= 0 || N <= 0) return 0;
+  return prep_split_bytes(d, N) + (size_t)N * (size_t)d * 4;
+}
+
+// W' (float32 [N, d]) into the workspace; returns its address in *wp.
+static torq_status rotate_weights(const void* W, const void* R_inter, const void* R_intra, int64_t d, int64_t N,
+                                  void* workspace, size_t workspace_bytes, void* stream, float** wp) {
+  if (!W || !R_inter) return TORQ_ERR_NULL;
+  if (d < 64 || d % 64 != 0 || N < 1 || N > (1 << 30) || d > (1 << 24)) return TORQ_ERR_SHAPE;
+  if (!workspace || workspace_bytes < torq_prepare_weights_workspace_bytes(d, N)) return TORQ_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || !aligned16(W)) return TORQ_ERR_ALIGN;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  __nv_bfloat16* T = static_cast<__nv_bfloat16*>(workspace);
+  *wp = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + prep_split_bytes(d, N));
+  const int64_t tiles = ((N + 31) / 32) * ((d + 31) / 32);
+  transpose_split3_kernel<<<ew_grid(tiles, 1, st->sm_count), 256, 0, s>>>(static_cast<const float*>(W), d, N, T);
+  if (launch_status() != TORQ_OK) return TORQ_ERR_LAUNCH;
+  return rotate_quantize_impl(T, R_inter, R_intra, N, d, *wp, nullptr, nullptr, 0, stream, FMT_F32OUT, 0.0f, 3);
+}
+
+torq_status torq_prepare_weights(const void* W, const void* R_inter, const void* R_intra, int64_t d, int64_t N,
+                                 void* Wq, void* Ws, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!Wq || !Ws) return TORQ_ERR_NULL;
+  float* wp = nullptr;
+  const torq_status rc = rotate_weights(W, R_inter, R_intra, d, N, workspace, workspace_bytes, stream, &wp);
+  if (rc != TORQ_OK) return rc;
+  return torq_quantize_mxfp4(wp, TORQ_F32, N, d, Wq, Ws, stream);
+}
+
+torq_status torq_prepare_weights_nvfp4(const void* W, const void* R_inter, const void* R_intra32, int64_t d,
+                                       int64_t N, void* Wq, void* Ws, float* tensor_scale, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+  if (!Wq || !Ws || !tensor_scale) return TORQ_ERR_NULL;
+  float* wp = nullptr;
+  torq_status rc = rotate_weights(W, R_inter, R_intra32, d, N, workspace, workspace_bytes, stream, &wp);
+  if (rc != TORQ_OK) return rc;
+  DeviceState* st = device_state();
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // the split of W^T is no longer needed: its first word holds the running maximum
+  unsigned int* amax_bits = static_cast<unsigned int*>(workspace);
+  if (cudaMemsetAsync(amax_bits, 0, sizeof(unsigned int), s) != cudaSuccess) return TORQ_ERR_LAUNCH;
+  absmax_kernel<<<ew_grid(N * d, 1024, st->sm_count), 256, 0, s>>>(wp, N * d, amax_bits);
+  if (launch_status() != TORQ_OK) return TORQ_ERR_LAUNCH;
+  float amax = 0.f;
+  if (cudaMemcpyAsync(&amax, amax_bits, sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return TORQ_ERR_LAUNCH;
+  const float ts = amax / 2688.0f;                       // amax / (6 * 448), one float32 division
+  if (!scale_ok(ts)) return TORQ_ERR_SHAPE;              // an all-zero (or non-finite) W' has no scale
+  *tensor_scale = ts;
+  return torq_quantize_nvfp4(wp, TORQ_F32, N, d, ts, Wq, Ws, stream);
+}
+
+torq_status torq_prepare_weights_mxint4(const void* W, const void* R_inter, const void* R_intra, int64_t d,
+                                        int64_t N, void* Wn, void* W8, void* Ws, void* workspace,
+                                        size_t workspace_bytes, void* stream) {
+  if ((!Wn && !W8) || !Ws) return TORQ_ERR_NULL;
+  float* wp = nullptr;
+  torq_status rc = rotate_weights(W, R_inter, R_intra, d, N, workspace, workspace_bytes, stream, &wp);
+  if (rc != TORQ_OK) return rc;
+  if (Wn) {
+    rc = torq_quantize_mxint4(wp, TORQ_F32, N, d, 1, Wn, Ws, stream);
+    if (rc != TORQ_OK) return rc;
+  }
+  if (W8) return torq_quantize_mxint4(wp, TORQ_F32, N, d, 0, W8, Ws, stream);
+  return TORQ_OK;
+}
+
+torq_status torq_merge_rotations_bf16(const void* R_inter, const void* R_intra, int64_t d, void* R_merged_bf16,
+                                      void* stream) {
+  if (!R_inter || !R_intra || !R_merged_bf16) return TORQ_ERR_NULL;
+  if (d < 32 || d % 32 != 0 || d > (1 << 24)) return TORQ_ERR_SHAPE;
+  DeviceState* st = device_state();
+  if (!st) return TORQ_ERR_LAUNCH;
+  if (!st->arch_ok) return TORQ_ERR_ARCH;
+  merge_rotations_kernel<__nv_bfloat16><<<ew_grid(d * d, 256, st->sm_count), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(R_inter), static_cast<const __nv_bfloat16*>(R_intra), d,
+      static_cast<__nv_bfloat16*>(R_merged_bf16));
+  return launch_status();
+}
+
 torq_status torq_merge_rotations(const void* R_inter, const void* R_intra, int64_t d, void* R_merged_f32,
                                  void* stream) {
   if (!R_inter || !R_intra || !R_merged_f32) return TORQ_ERR_NULL;
@@ -992,7 +1084,7 @@ torq_status torq_merge_rotations(const void* R_inter, const void* R_intra, int64
   DeviceState* st = device_state();
   if (!st) return TORQ_ERR_LAUNCH;
   if (!st->arch_ok) return TORQ_ERR_ARCH;
-  merge_rotations_kernel<<<ew_grid(d * d, 256, st->sm_count), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+  merge_rotations_kernel<float><<<ew_grid(d * d, 256, st->sm_count), 256, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const __nv_bfloat16*>(R_inter), static_cast<const __nv_bfloat16*>(R_intra), d,
       static_cast<float*>(R_merged_f32));
   return launch_status();

@@ -59,6 +59,16 @@ def lib() -> ctypes.CDLL:
     L.torq_merge_rotations.argtypes = [vp, vp, i64, vp, vp]
     L.torq_merge_rotations.restype = ci
     f32 = ctypes.c_float
+    L.torq_merge_rotations_bf16.argtypes = [vp, vp, i64, vp, vp]
+    L.torq_merge_rotations_bf16.restype = ci
+    L.torq_prepare_weights_workspace_bytes.argtypes = [i64, i64]
+    L.torq_prepare_weights_workspace_bytes.restype = sz
+    L.torq_prepare_weights.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp, sz, vp]
+    L.torq_prepare_weights.restype = ci
+    L.torq_prepare_weights_nvfp4.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.POINTER(ctypes.c_float), vp, sz, vp]
+    L.torq_prepare_weights_nvfp4.restype = ci
+    L.torq_prepare_weights_mxint4.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp, vp, sz, vp]
+    L.torq_prepare_weights_mxint4.restype = ci
     L.torq_nvfp4_scales_bytes.argtypes = [i64, i64]
     L.torq_nvfp4_scales_bytes.restype = sz
     L.torq_nvfp4_workspace_bytes.argtypes = [i64, i64, i64]
@@ -95,8 +105,8 @@ def lib() -> ctypes.CDLL:
     L.torq_givens_equalize.restype = ci
     L.torq_probe_fp4_peak.argtypes = [ci, ctypes.POINTER(ctypes.c_double), vp]
     L.torq_probe_fp4_peak.restype = ci
-    L.torq_probe_fp4_peak_fills.argtypes = [ci, vp, sz, ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), vp]
-    L.torq_probe_fp4_peak_fills.restype = ci
+    L.torq_selftest_wait_timeout.argtypes = [ctypes.c_uint64, vp, vp]
+    L.torq_selftest_wait_timeout.restype = ci
     L.torq_status_string.argtypes = [ci]
     L.torq_status_string.restype = ctypes.c_char_p
     L.torq_last_device_error.argtypes = [vp]
@@ -278,13 +288,12 @@ def torq_probe_fp4_peak(groups: int = 40000, stream=None) -> float:
     return out.value
 
 
-def torq_probe_fp4_peak_fills(src, with_mma: bool = True, groups: int = 40000, stream=None):
-    """The FP4 probe with background fills from `src` (uint8 device tensor).  Returns (TFLOP/s, fill GB/s per SM)."""
-    _check(src, torch.uint8, "src")
-    t, g = ctypes.c_double(0.0), ctypes.c_double(0.0)
-    _raise(lib().torq_probe_fp4_peak_fills(groups, _ptr(src), src.numel(), 1 if with_mma else 0, ctypes.byref(t),
-                                           ctypes.byref(g), _stream(stream)), "torq_probe_fp4_peak_fills")
-    return t.value, g.value
+def torq_selftest_wait_timeout(limit_ns: int = 1_000_000, stream=None):
+    """Runs the give-up path of the bounded device waits once, harmlessly (see torq.h).  Returns a
+    device int64 tensor [gave_up, left_through_abort_flag, waited_ns]."""
+    out = torch.zeros(4, dtype=torch.int64, device="cuda")
+    _raise(lib().torq_selftest_wait_timeout(int(limit_ns), _ptr(out), _stream(stream)), "torq_selftest_wait_timeout")
+    return out[:3]
 
 
 def torq_swizzle_scales(linear, k: int, out=None, stream=None):
@@ -307,18 +316,44 @@ def torq_merge_rotations(R_inter, R_intra, out=None, stream=None):
     return out
 
 
-def prepare_weights(R_inter, R_intra, W):
-    """Offline weight side of the layer (not on the timed path): W' = R~^T W for W [d,N] float32,
-    stored [N,d], MXFP4-quantized along K by torq_quantize_mxfp4.  The matrix product is a library
-    call (torch.matmul, fp32); returns (Wq [N,d/2], Ws tiled)."""
-    Rm = torq_merge_rotations(R_inter, R_intra)
-    prev = torch.backends.cuda.matmul.allow_tf32
-    torch.backends.cuda.matmul.allow_tf32 = False
-    try:
-        Wp = torch.matmul(W.t().contiguous().to(torch.float32), Rm).contiguous()   # [N,d] = (R~^T W)^T
-    finally:
-        torch.backends.cuda.matmul.allow_tf32 = prev
-    return torq_quantize_mxfp4(Wp)
+def torq_merge_rotations_bf16(R_inter, R_intra, out=None, stream=None):
+    """R~ = R_inter blockdiag(R_intra) rounded once to bfloat16: the operand of the one-GEMM form of the rotation."""
+    d = R_inter.shape[0]
+    _check(R_inter, torch.bfloat16, "R_inter")
+    _check(R_intra, torch.bfloat16, "R_intra")
+    if out is None:
+        out = torch.empty((d, d), dtype=torch.bfloat16, device=R_inter.device)
+    _raise(lib().torq_merge_rotations_bf16(_ptr(R_inter), _ptr(R_intra), d, _ptr(out), _stream(stream)),
+           "torq_merge_rotations_bf16")
+    return out
+
+
+def torq_prepare_weights_workspace_bytes(d: int, N: int) -> int:
+    return int(lib().torq_prepare_weights_workspace_bytes(d, N))
+
+
+def _prep_args(R_inter, R_intra, W, workspace):
+    _check(W, torch.float32, "W")
+    _check(R_inter, torch.bfloat16, "R_inter")
+    _check(R_intra, torch.bfloat16, "R_intra")
+    d, N = W.shape
+    if workspace is None:
+        workspace = torch.empty(torq_prepare_weights_workspace_bytes(d, N), dtype=torch.uint8, device=W.device)
+    return d, N, workspace
+
+
+def torq_prepare_weights(R_inter, R_intra, W, workspace=None, stream=None):
+    """Offline weight side of the layer: W [d,N] float32 -> (Wq [N,d/2], Ws tiled), W' = R~^T W quantized
+    to MXFP4 along K, all of it by the library's kernels."""
+    d, N, workspace = _prep_args(R_inter, R_intra, W, workspace)
+    Wq = torch.empty((N, d // 2), dtype=torch.uint8, device=W.device)
+    Ws = torch.empty(torq_scales_bytes(N, d), dtype=torch.uint8, device=W.device)
+    _raise(lib().torq_prepare_weights(_ptr(W), _ptr(R_inter), _ptr(R_intra), d, N, _ptr(Wq), _ptr(Ws),
+                                      _ptr(workspace), workspace.numel(), _stream(stream)), "torq_prepare_weights")
+    return Wq, Ws
+
+
+prepare_weights = torq_prepare_weights
 
 
 # ---- NVFP4 variant (16-element blocks, E4M3 block scales, float32 tensor scale) -----------------------
@@ -408,19 +443,20 @@ def torq_rotated_linear_nvfp4(X, R_inter, R_intra32, x_tensor_scale: float, Wq, 
     return Y
 
 
-def prepare_weights_nvfp4(R_inter, R_intra32, W):
-    """Offline weight side in NVFP4: W' = R~^T W (as prepare_weights), tensor scale amax / (6 * 448),
-    quantized along K by torq_quantize_nvfp4.  Returns (Wq [N,d/2], Ws tiled, tensor_scale)."""
-    Rm = torq_merge_rotations(R_inter, R_intra32)
-    prev = torch.backends.cuda.matmul.allow_tf32
-    torch.backends.cuda.matmul.allow_tf32 = False
-    try:
-        Wp = torch.matmul(W.t().contiguous().to(torch.float32), Rm).contiguous()
-    finally:
-        torch.backends.cuda.matmul.allow_tf32 = prev
-    ts = float(Wp.abs().max().item()) / (6.0 * 448.0)
-    Wq, Ws = torq_quantize_nvfp4(Wp, ts)
-    return Wq, Ws, ts
+def torq_prepare_weights_nvfp4(R_inter, R_intra32, W, workspace=None, stream=None):
+    """Offline weight side in NVFP4: returns (Wq [N,d/2], Ws tiled, tensor_scale = max|W'| / (6 * 448)).
+    Synchronises the stream once (the tensor scale comes back to the host)."""
+    d, N, workspace = _prep_args(R_inter, R_intra32, W, workspace)
+    Wq = torch.empty((N, d // 2), dtype=torch.uint8, device=W.device)
+    Ws = torch.empty(torq_nvfp4_scales_bytes(N, d), dtype=torch.uint8, device=W.device)
+    ts = ctypes.c_float(0.0)
+    _raise(lib().torq_prepare_weights_nvfp4(_ptr(W), _ptr(R_inter), _ptr(R_intra32), d, N, _ptr(Wq), _ptr(Ws),
+                                            ctypes.byref(ts), _ptr(workspace), workspace.numel(), _stream(stream)),
+           "torq_prepare_weights_nvfp4")
+    return Wq, Ws, ts.value
+
+
+prepare_weights_nvfp4 = torq_prepare_weights_nvfp4
 
 
 # ---- MXINT4 variant (format study of Section 6) ---------------------------------------------------------
@@ -520,18 +556,19 @@ def torq_rotated_linear_mxint4(X, R_inter, R_intra, W8, Ws, out_dtype=torch.bflo
     return Y
 
 
-def prepare_weights_mxint4(R_inter, R_intra, W):
-    """Offline weight side in MXINT4: W' = R~^T W (as prepare_weights), quantized along K.
-    Returns (stored form [N,d/2], operand form [N,d], tiled scales)."""
-    Rm = torq_merge_rotations(R_inter, R_intra)
-    prev = torch.backends.cuda.matmul.allow_tf32
-    torch.backends.cuda.matmul.allow_tf32 = False
-    try:
-        Wp = torch.matmul(W.t().contiguous().to(torch.float32), Rm).contiguous()
-    finally:
-        torch.backends.cuda.matmul.allow_tf32 = prev
-    Wn, Ws = torq_quantize_mxint4(Wp, packed=True)
-    return Wn, torq_mxint4_expand(Wn), Ws
+def torq_prepare_weights_mxint4(R_inter, R_intra, W, workspace=None, stream=None):
+    """Offline weight side in MXINT4: returns (stored form [N,d/2], operand form [N,d], tiled scales)."""
+    d, N, workspace = _prep_args(R_inter, R_intra, W, workspace)
+    Wn = torch.empty((N, d // 2), dtype=torch.uint8, device=W.device)
+    W8 = torch.empty((N, d), dtype=torch.uint8, device=W.device)
+    Ws = torch.empty(torq_scales_bytes(N, d), dtype=torch.uint8, device=W.device)
+    _raise(lib().torq_prepare_weights_mxint4(_ptr(W), _ptr(R_inter), _ptr(R_intra), d, N, _ptr(Wn), _ptr(W8), _ptr(Ws),
+                                             _ptr(workspace), workspace.numel(), _stream(stream)),
+           "torq_prepare_weights_mxint4")
+    return Wn, W8, Ws
+
+
+prepare_weights_mxint4 = torq_prepare_weights_mxint4
 
 
 # ---- calibration of the inter-block rotation (Section 5.1, Algorithm 1; offline) -----------------------

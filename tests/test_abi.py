@@ -129,7 +129,4 @@ def test_probe_argument_errors():
     one = ctypes.c_void_p(16)
     d = ctypes.c_double(0.0)
     assert L.torq_probe_fp4_peak(100, None, None) == 1
-    assert L.torq_probe_fp4_peak_fills(100, None, 1 << 20, 1, ctypes.byref(d), ctypes.byref(d), None) == 1
-    assert L.torq_probe_fp4_peak_fills(100, one, 1000, 1, ctypes.byref(d), ctypes.byref(d), None) == 2      # < 32 KiB
-    assert L.torq_probe_fp4_peak_fills(0, one, 1 << 20, 1, ctypes.byref(d), ctypes.byref(d), None) == 2
-    assert L.torq_probe_fp4_peak_fills(100, ctypes.c_void_p(24), 1 << 20, 1, ctypes.byref(d), ctypes.byref(d), None) == 3
+    assert L.torq_probe_fp4_peak(0, ctypes.byref(d), None) == 2

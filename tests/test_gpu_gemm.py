@@ -181,15 +181,3 @@ def test_several_waves_of_tiles_with_ragged_edges_and_one_hot_rows(M, N, K, dt):
     else:
         assert (got[hot_rows] == ref[hot_rows]).all()
         assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
-
-
-def test_fp4_probe_with_background_fills_reports_plausible_rates():
-    """Fills alone: an SM takes in tens of GB/s at least; fills beside the instruction stream: both numbers stay
-    within a factor of two of what each does alone (a measurement tool: only sanity is checked)."""
-    src = torch.zeros(48 << 20, dtype=torch.uint8, device="cuda")
-    t0, g0 = torq.torq_probe_fp4_peak_fills(src, with_mma=False, groups=20000)
-    t1, g1 = torq.torq_probe_fp4_peak_fills(src, with_mma=True, groups=20000)
-    alone = torq.torq_probe_fp4_peak(20000)
-    assert torq.torq_last_device_error() == 0
-    assert t0 == 0.0 and 20.0 < g0 < 1000.0
-    assert 0.5 * alone < t1 <= 1.05 * alone and 20.0 < g1 <= 1.05 * g0

@@ -300,20 +300,6 @@ def test_rotated_linear_few_tokens_takes_the_split_rotation(M, intra):
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-5
 
 
-def test_device_weight_preparation_matches_the_oracle():
-    cfg = I.CONFIGS["tiny"]
-    d, N = 256, 192
-    rb, rib, _, _ = I.rotations(cfg, d=d)
-    w = I.weights(cfg, d=d, N=N)
-    Wn, W8, Ws = torq.prepare_weights_mxint4(dev_bf16(rb), dev_bf16(rib), torch.from_numpy(w).cuda())
-    torch.cuda.synchronize()
-    o_q, o_sb = O.prepare_weights_mxint4(rb, rib, w)
-    g_q = O.unpack_int4(Wn.cpu().numpy())
-    assert np.array_equal(O.e4m3_to_int4(W8.cpu().numpy()), g_q)
-    rep = _mismatch(g_q, O.unswizzle_scales(Ws.cpu().numpy(), N, d), o_q, o_sb)
-    assert rep["non_adjacent"] == 0 and rep["elem"] <= 1e-3 and rep["blocks"] <= 1e-3, rep
-
-
 def test_llama3_qkv_shape_sampled_rows():
     """Benchmark shape (2048 x 4096 -> 6144): rotation and quantizer on sampled rows against the oracle
     (rows are independent), the GEMM on the GPU's own codes for the same rows."""

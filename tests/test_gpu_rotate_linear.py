@@ -96,18 +96,6 @@ def test_tiny_config_end_to_end():
     assert np.linalg.norm(got - o_out) / np.linalg.norm(o_out) <= 2e-2
 
 
-def test_device_weight_preparation_matches_oracle_weights():
-    cfg = I.CONFIGS["tiny"]
-    rb, rib, _, _ = I.rotations(cfg)
-    w = I.weights(cfg)
-    Wq, Ws = torq.prepare_weights(dev_bf16(rb), dev_bf16(rib), torch.from_numpy(w).cuda())
-    torch.cuda.synchronize()
-    g_codes, g_sb = gpu_quantized_to_numpy(Wq, Ws, cfg.N, cfg.d)
-    o_codes, o_sb = O.prepare_weights(rb, rib, w)
-    rep = mismatch_report(g_codes, g_sb, o_codes, o_sb)
-    assert rep["non_adjacent"] == 0 and rep["elem_mismatch_frac"] <= 1e-3, rep
-
-
 def test_llama3_qkv_shape_sampled_rows():
     """Config 2 at full size (2048 x 4096 -> 6144): rotate+quantize checked on sampled rows that
     span several row tiles, the GEMM on the same rows, bf16 output."""

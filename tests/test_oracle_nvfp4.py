@@ -187,3 +187,75 @@ def test_rotated_linear_identity_chain_recovers_the_product_up_to_quantization()
     ref = O.decode_bf16(x) @ w
     assert np.linalg.norm(out - ref) / np.linalg.norm(ref) < 0.2     # two 4-bit operands
     assert np.linalg.norm(O.dequantize_nvfp4(wc, wsb, wts) - w.T) / np.linalg.norm(w) < 0.12
+
+
+def _lattice(codes):
+    mag = (codes & 7).astype(np.int64)
+    return np.where(codes & 8, -mag, mag)
+
+
+def _exact_block_by_fractions(z_block, ts):
+    """One 16-element block by the format's definition in exact rational arithmetic (pure Python)."""
+    vals = [Fraction(float(v)) for v in O.e4m3_value(np.arange(0x7F, dtype=np.uint8))]
+    book = [Fraction(float(c)) for c in O.CODEBOOK]
+
+    def nearest_even(x, grid):
+        best = min(range(len(grid)), key=lambda i: (abs(grid[i] - x), i % 2))
+        return best
+
+    zs = [Fraction(float(v)) for v in z_block]
+    t = Fraction(float(np.float32(ts)))
+    amax = max(abs(v) for v in zs)
+    byte = nearest_even(min(amax / (6 * t), Fraction(448)), vals)
+    if byte == 0:
+        return byte, [(8 if np.signbit(v) else 0) for v in z_block]
+    dec = vals[byte] * t
+    codes = []
+    for v, f in zip(z_block, zs):
+        mag = nearest_even(min(abs(f) / dec, Fraction(6)), book)
+        codes.append((8 if np.signbit(v) else 0) | mag)
+    return byte, codes
+
+
+def test_exact_definition_matches_rational_arithmetic_block_by_block():
+    """quantize_nvfp4_exact (float64 divisions) against the definition in exact fractions, on blocks
+    with tensor scales that are not powers of two, including a block on an E4M3 tie."""
+    g = np.random.default_rng(21)
+    for ts in (1.0, 0.37, 3.1e-4, 1.0 / 3.0, 250.0):
+        z = (g.standard_t(3, size=(24, 16)) * float(ts) * np.exp(g.uniform(-2, 6, size=(24, 1)))).astype(np.float32)
+        z[0] = 0.0
+        z[1, 0] = np.float32(6.0 * 1.0625 * float(np.float32(ts)))       # amax / (6 ts) near the tie 1.0625
+        codes, sb = O.quantize_nvfp4_exact(z, ts)
+        for r in range(z.shape[0]):
+            byte, want = _exact_block_by_fractions(z[r], ts)
+            assert sb[r, 0] == byte, (ts, r)
+            assert codes[r].tolist() == want, (ts, r)
+
+
+def test_float32_recipe_is_the_exact_definition_up_to_its_roundings():
+    """The float32 recipe (reciprocal multiplies, three roundings of 2^-24 per decision) against the
+    exact definition on heavy-tailed blocks with tensor scales that are not powers of two.  A
+    decision can move only for a value within ~2^-22 relative of a threshold: E4M3 has 8 thresholds
+    per octave and e2m1 7 over [0, 6], so the expected rate is of order 1e-6 per block or element.
+    Bound asserted: at most 1e-5 of the block scales differ, each by one E4M3 step; outside those
+    blocks at most 1e-5 of the elements differ; every differing element, inside those blocks too
+    (one E4M3 step moves a scaled value by at most 12.5 %, less than one codebook gap), is one
+    lattice step away."""
+    g = np.random.default_rng(5)
+    n_blocks = n_elems = d_blocks = d_elems = 0
+    for mul in (1.0, 0.37, 3.1e-4, 250.0, 1.0 / 3.0, 0.7071):
+        z = (g.standard_t(3, size=(1024, 1024)) * np.exp(g.uniform(-4, 4, size=(1024, 1)))).astype(np.float32)
+        ts = np.float32(np.abs(z).max() / (6 * 448) * mul * 1.2345)
+        c32, s32 = O.quantize_nvfp4(z, ts)
+        cex, sex = O.quantize_nvfp4_exact(z, ts)
+        step = np.abs(s32.astype(np.int64) - sex.astype(np.int64))
+        assert step.max() <= 1
+        lat = np.abs(_lattice(c32) - _lattice(cex))
+        assert lat.max() <= 1
+        same = np.repeat(step == 0, 16, axis=1)
+        n_blocks += step.size
+        n_elems += lat.size
+        d_blocks += int((step != 0).sum())
+        d_elems += int(((lat != 0) & same).sum())
+        assert np.array_equal(c32 >> 3, cex >> 3)                      # sign bits never differ
+    assert d_blocks <= 1e-5 * n_blocks and d_elems <= 1e-5 * n_elems, (d_blocks, n_blocks, d_elems, n_elems)
