@@ -1,0 +1,249 @@
+// Rotate + quantize for few tokens (M <= 64), where the work is streaming R_inter from HBM once
+// (Algorithm 3 steps 2-4).  One kernel, no scratch in global memory.
+//
+// Swapped operands: the tensor-core instruction's 128 rows are 128 output FEATURES (four 32-blocks)
+// and its N columns are the tokens (16, 32 or 64), so no row of the instruction is padding and the
+// accumulator is small:  D[j, m] = sum_i R_inter[i, j] X[m, i].
+//   A = R_inter tile [64 (i) x 128 (j)], features contiguous = MN-major, two 64 x 64 boxes (128-B swizzle)
+//   B = X tile [tokens x 64 (i)], K-major
+// A layer has only d / 128 feature tiles (40 at d = 5120), too few CTAs to pull R_inter at HBM rate,
+// so the contraction is also split: a CLUSTER of S CTAs shares one feature tile, CTA r of the cluster
+// contracts k range r.  The fp32 partial tiles never leave the SMs: every CTA writes its partial
+// [token][feature] into its own shared memory, a cluster barrier publishes them, and each warp of
+// the cluster then owns some (16 tokens x one 32-block) units: it adds the S partials of its unit in
+// rank order through distributed shared memory (plain ld.shared::cluster; fixed order, so the result
+// does not depend on timing), applies the intra-block rotation on the warp-level tensor cores (y split
+// into three bf16 terms, fp32 accumulation) and quantizes (Eq. 1).
+//
+// Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue / reduction.
+// Shared memory: 4 stages of (16 KiB of R_inter + tokens x 128 B of X); after the mainloop the same
+// memory holds the partial tile and the per-warp staging of the reduction.  Small enough (<= 97 KiB)
+// for the CTAs of the kernel that follows in the stream to become resident beside this one.
+#pragma once
+#include <cuda_bf16.h>
+#include "intra_fragment.cuh"
+#include "sm100_ptx.cuh"
+
+namespace torq {
+
+struct RotFewCfg {
+  static constexpr int BF = 128;                       // features per tile = rows of the instruction
+  static constexpr int BK = 64;
+  static constexpr int A_BYTES = BK * BF * 2;          // 16 KiB: two boxes of 64 (k) x 64 (j)
+  static constexpr int A_BOX_BYTES = 64 * 64 * 2;
+  static constexpr int STAGES = 4;
+  static constexpr int MAX_TOK = 64;
+  static constexpr int WARP_SCRATCH = 16 * 33 * 4 + 32 * 80;      // y tile + R_intra block per epilogue warp
+  static constexpr int BAR_BYTES = 256;
+  static constexpr int THREADS = 192;
+  static constexpr int MAX_CLUSTER = 8;
+  __host__ __device__ static constexpr int stage_bytes(int ntok) { return A_BYTES + ntok * BK * 2; }
+  __host__ __device__ static constexpr int smem_bytes(int ntok) {
+    return STAGES * stage_bytes(ntok) + BAR_BYTES + 1024;
+  }
+  // the reduction's buffers must fit inside the stages they reuse
+  static_assert(MAX_TOK * BF * 4 + 4 * WARP_SCRATCH <= STAGES * (A_BYTES + 16 * BK * 2), "reduction buffers");
+};
+
+__device__ __forceinline__ float ld_shared_cluster_f32(uint32_t cluster_addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
+  return v;
+}
+
+// grid = (d / 128) * S CTAs in clusters of S along x: CTA b works feature tile b / S, k split b % S.
+// tmX: X [M, d] bf16, box [ntok rows x 64]; tmR: R_inter [d, d] bf16, box [64 x 64].  ntok = 16, 32 or 64
+// >= M.  d % 128 == 0.  `codes` / `scales` / `tensor_scale` as in rotate_quantize_kernel for FMT.
+template <int FMT = FMT_MXFP4>
+__global__ void __launch_bounds__(192, 1)
+rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
+                     const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
+                     uint8_t* __restrict__ scales, int M, int d, int ntok, int S, float tensor_scale,
+                     int* err_word) {
+  using C = RotFewCfg;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const int stage_bytes = C::stage_bytes(ntok);
+  const uint32_t bar_off = C::STAGES * stage_bytes;
+  const uint32_t bar_base = smem_base + bar_off;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };
+  const uint32_t accf_bar = bar_base + 8u * (2 * C::STAGES);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + bar_off + 192);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(smem_gen + bar_off + 200);
+  // after the mainloop: partial tile P[token][feature] fp32 at offset 0, then the warps' staging
+  float* P = reinterpret_cast<float*>(smem_gen);
+  uint8_t* scratch = smem_gen + ntok * C::BF * 4;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = blockIdx.x % S, ft = blockIdx.x / S;
+  const int k_tiles = d / C::BK;
+  const int kt0 = (int)((long long)k_tiles * rank / S), kt1 = (int)((long long)k_tiles * (rank + 1) / S);
+  const uint32_t tmem_cols = ntok < 32 ? 32u : (uint32_t)ntok;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(accf_bar, 1);
+    *cta_abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), tmem_cols); tmem_relinquish(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  // R_inter is a constant of the layer, never the output of the kernel that runs just before this
+  // one: its loads for the first stages go out right away; X waits for that kernel.
+  griddep_launch_dependents();
+  const int pre = (kt1 - kt0) < C::STAGES ? (kt1 - kt0) : C::STAGES;
+  if (warp == 0) {
+    if (elect_one()) {
+      tma_prefetch_desc(&tmX);
+      tma_prefetch_desc(&tmR);
+      for (int it = 0; it < pre; ++it) {
+        const uint32_t st = smem_base + it * stage_bytes;
+        mbar_arrive_expect_tx(full_bar(it), (uint32_t)stage_bytes);
+        tma_load_2d(st, &tmR, ft * C::BF, (kt0 + it) * C::BK, full_bar(it));
+        tma_load_2d(st + C::A_BOX_BYTES, &tmR, ft * C::BF + 64, (kt0 + it) * C::BK, full_bar(it));
+      }
+    }
+    __syncwarp();
+  }
+  griddep_wait();
+
+  bool acc_ok = false;                                   // epilogue warps: the accumulator is complete
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    bool ok = true;
+    for (int kt = kt0, it = 0; kt < kt1 && ok; ++kt, ++it) {
+      const int s = it % C::STAGES;
+      if (!mbar_wait_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word, SITE_PRODUCER_EMPTY)) {
+        ok = false; break;
+      }
+      const uint32_t st = smem_base + s * stage_bytes;
+      if (elect_one()) {
+        const bool r_issued = it < pre;                  // R side of this stage went out before the wait above
+        if (!r_issued) {
+          mbar_arrive_expect_tx(full_bar(s), (uint32_t)stage_bytes);
+          tma_load_2d(st, &tmR, ft * C::BF, kt * C::BK, full_bar(s));
+          tma_load_2d(st + C::A_BOX_BYTES, &tmR, ft * C::BF + 64, kt * C::BK, full_bar(s));
+        }
+        tma_load_2d(st + C::A_BYTES, &tmX, kt * C::BK, 0, full_bar(s));
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    const uint32_t idesc = idesc_bf16(128, ntok, /*A MN-major*/ true, /*B MN-major*/ false);
+    bool ok = true;
+    for (int kt = kt0, it = 0; kt < kt1 && ok; ++kt, ++it) {
+      const int s = it % C::STAGES;
+      if (!mbar_wait_warp(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
+        ok = false; break;
+      }
+      tc_fence_after_sync();
+      const uint32_t st = smem_base + s * stage_bytes;
+      // A: MN-major.  64 features (128 B) contiguous, k rows 128 B apart, 8-row groups 1024 B apart
+      // (stride offset), the next 64 features one box (8 KiB) further (leading offset).
+      const uint64_t adesc = make_desc(st, C::A_BOX_BYTES, 1024, kSwizzle128);
+      // B: K-major, token rows of 128 B, 8-row groups 1024 B apart.
+      const uint64_t bdesc = make_desc(st + C::A_BYTES, 16, 1024, kSwizzle128);
+      if (elect_one()) {
+#pragma unroll
+        for (int j = 0; j < C::BK / 16; ++j)             // K = 16 per instruction: 16 k rows of A = 2 KiB, 32 B of B
+          mma_bf16(tmem_base, adesc + 128 * j, bdesc + 2 * j, idesc, (it | j) != 0);
+        tc_commit(empty_bar(s));
+      }
+      __syncwarp();
+    }
+    if (ok && elect_one()) tc_commit(accf_bar);
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ epilogue 1: partial tile -> own shared memory
+    const int q = warp & 3;
+    acc_ok = mbar_wait(accf_bar, 0, cta_abort, err_word, SITE_EPI_ACC_FULL);
+    acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
+    if (acc_ok) {
+      tc_fence_after_sync();
+      // every load into the stages has landed and every instruction that read them has completed
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
+      float* prow = P + q * 32 + lane;                   // feature 32 q + lane of token 0
+      for (int c0 = 0; c0 < ntok; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld_32x32_x16(tacc + c0, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) prow[(c0 + j) * C::BF] = __uint_as_float(v[j]);
+      }
+    }
+  }
+  tc_fence_before_sync();
+  cluster_sync_all();                                    // every CTA's partial tile is visible cluster-wide
+
+  if (warp >= 2) {
+    // ------------------------------------------------------------------ epilogue 2: reduce, intra-rotate, quantize
+    const int ew = warp - 2;                             // 0..3
+    const int groups = ntok / 16;                        // token groups of 16
+    const int units = 4 * groups;                        // (32-block of the tile, token group)
+    const int nblocks = d / 32;
+    float* y_s = reinterpret_cast<float*>(scratch + ew * C::WARP_SCRATCH);
+    uint8_t* r_s = scratch + ew * C::WARP_SCRATCH + 16 * 33 * 4;
+    const uint32_t p_saddr = smem_u32(P);
+    // unit u belongs to CTA u % S, and there to warp (u / S) % 4
+    for (int u = rank + S * ew; u < units; u += 4 * S) {
+      const int qb = u / groups, g = u - qb * groups;
+      const int blk = ft * 4 + qb;
+      if (R_intra != nullptr) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {                    // 128 pieces of 16 B: row (piece / 4), 8 columns each
+          const int piece = lane + 32 * i;
+          *reinterpret_cast<uint4*>(r_s + (piece >> 2) * 80 + (piece & 3) * 16) =
+              __ldg(reinterpret_cast<const uint4*>(R_intra + (size_t)blk * 1024) + piece);
+        }
+      }
+      // 16 tokens x 32 features: the S partials in rank order (rows >= M are zero in every partial)
+      const uint32_t off = (uint32_t)(((16 * g) * C::BF + qb * 32 + lane) * 4);
+#pragma unroll 4
+      for (int t = 0; t < 16; ++t) {
+        float part[C::MAX_CLUSTER];
+#pragma unroll
+        for (int s = 0; s < C::MAX_CLUSTER; ++s)
+          part[s] = s < S ? ld_shared_cluster_f32(map_to_cta(p_saddr, (uint32_t)s) + off + (uint32_t)(t * C::BF * 4)) : 0.f;
+        float y = 0.f;
+#pragma unroll
+        for (int s = 0; s < C::MAX_CLUSTER; ++s) if (s < S) y += part[s];
+        y_s[t * 33 + lane] = y;
+      }
+      __syncwarp();
+      intra_quantize_rows16<FMT>(y_s, smem_u32(r_s), R_intra != nullptr, lane, 16 * g, M, blk, d, nblocks,
+                                 tensor_scale, codes, scales);
+      __syncwarp();
+    }
+    // scale bytes of the rows no unit covers (ntok .. 127 of the single 128-row scale tile): zero
+    if (rank == 0) {
+      const int row = ew * 32 + lane;
+      if (row >= ntok) {
+        if constexpr (FMT == FMT_NVFP4) {
+          *reinterpret_cast<uint32_t*>(scales + (size_t)(2 * ft) * 512 + (row & 31) * 16 + (row >> 5) * 4) = 0u;
+          *reinterpret_cast<uint32_t*>(scales + (size_t)(2 * ft + 1) * 512 + (row & 31) * 16 + (row >> 5) * 4) = 0u;
+        } else {
+          *reinterpret_cast<uint32_t*>(scales + (size_t)ft * 512 + (row & 31) * 16 + (row >> 5) * 4) = 0u;
+        }
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncthreads();
+  if (*cta_abort) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  cluster_sync_all();                                    // no CTA of the cluster reads this one's partial tile any more
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, tmem_cols);
+  }
+}
+
+}  // namespace torq

@@ -14,6 +14,8 @@
 #include "rotate_quantize.cuh"
 #include "rotate_quantize_pair.cuh"
 #include "rotate_splitk.cuh"
+#include "rotate_fewtok.cuh"
+#include "gemm_fewtok.cuh"
 #include "rotate_structured.cuh"
 #include "rotated_linear_fused.cuh"
 #include "fp4_peak_probe.cuh"
@@ -118,6 +120,12 @@ static DeviceState* device_state() {
               opt_in_smem(rotate_quantize_kernel<256, FMT_MXINT4>, RotCfg<256>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_pair_kernel<FMT_MXINT4>, RotPairCfg::SMEM_BYTES) &&
               opt_in_smem(rotate_structured_kernel<FMT_MXINT4>, RotStructCfg::SMEM_BYTES) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_MXFP4>, RotFewCfg::smem_bytes(RotFewCfg::MAX_TOK)) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_NVFP4>, RotFewCfg::smem_bytes(RotFewCfg::MAX_TOK)) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_MXINT4>, RotFewCfg::smem_bytes(RotFewCfg::MAX_TOK)) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_MXFP4>, GemmFewCfg<FMT_MXFP4>::smem_bytes(RotFewCfg::MAX_TOK)) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_NVFP4>, GemmFewCfg<FMT_NVFP4>::smem_bytes(RotFewCfg::MAX_TOK)) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_MXINT4>, GemmFewCfg<FMT_MXINT4>::smem_bytes(RotFewCfg::MAX_TOK)) &&
               opt_in_smem(rotate_quantize_kernel<256, FMT_F32OUT>, RotCfg<256>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_pair_kernel<FMT_F32OUT>, RotPairCfg::SMEM_BYTES);
     if (!ok) return nullptr;
@@ -207,6 +215,15 @@ static int rotation_splits(int64_t M, int64_t d, int sm_count) {
   if (s > RotSplitCfg::MAX_SPLITS) s = RotSplitCfg::MAX_SPLITS;
   if (s > k_tiles / 2) s = k_tiles / 2;
   return s < 2 ? 1 : s;
+}
+// Few-token kernels (M <= 64): tokens per instruction and the cluster size = number of K splits of
+// one 128-feature tile, as many as fill the SMs (at most 8, each split at least `min_k` K steps).
+static inline int fewtok_ntok(int64_t M) { return M <= 16 ? 16 : (M <= 32 ? 32 : 64); }
+static inline int fewtok_cluster(int64_t tiles, int64_t k_steps, int min_k, int sm_count) {
+  int64_t s = sm_count / (tiles > 0 ? tiles : 1);
+  if (s > 8) s = 8;
+  if (s > k_steps / min_k) s = k_steps / min_k;
+  return s < 1 ? 1 : (int)s;
 }
 static size_t quantized_bytes(int64_t M, int64_t d) {    // codes, then 256-byte aligned the scales
   return ((size_t)M * (size_t)(d / 2) + 255) / 256 * 256 + torq_scales_bytes(M, d);
@@ -324,6 +341,28 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
     return launch_status();
   }
   CUtensorMap tmX, tmR;
+  if (M <= RotFewCfg::MAX_TOK && d % 128 == 0 && x_terms == 1 && fmt != FMT_F32OUT) {
+    // Few tokens: 128 features x all tokens per CTA, K split over a cluster, reduced through
+    // distributed shared memory; one launch, no scratch.
+    const int ntok = fewtok_ntok(M);
+    const int tiles = (int)(d / 128);
+    const int S = fewtok_cluster(tiles, d / 64, 2, st->sm_count);
+    if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d, (uint32_t)ntok, 64) ||
+        !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
+      return TORQ_ERR_LAUNCH;
+    const int smem = RotFewCfg::smem_bytes(ntok);
+    if (fmt == FMT_MXINT4)
+      launch_tc(rotate_fewtok_kernel<FMT_MXINT4>, S, tiles * S, RotFewCfg::THREADS, smem, s, tmX, tmR,
+                static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, ntok, S, 0.0f, st->err_word);
+    else if (fmt == FMT_NVFP4)
+      launch_tc(rotate_fewtok_kernel<FMT_NVFP4>, S, tiles * S, RotFewCfg::THREADS, smem, s, tmX, tmR,
+                static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, ntok, S, tensor_scale,
+                st->err_word);
+    else
+      launch_tc(rotate_fewtok_kernel<FMT_MXFP4>, S, tiles * S, RotFewCfg::THREADS, smem, s, tmX, tmR,
+                static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, ntok, S, 0.0f, st->err_word);
+    return launch_status();
+  }
   if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d * x_terms, 128, 64) ||
       !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
     return TORQ_ERR_LAUNCH;
@@ -478,6 +517,21 @@ static torq_status gemm_impl(const void* Aq, const void* As, const void* Wq, con
   constexpr int BN = 256;
   const uint64_t krow = (uint64_t)(FMT == FMT_MXINT4 ? K : K / 2);   // operand bytes per row
   CUtensorMap tmA, tmB;
+  if (M <= RotFewCfg::MAX_TOK) {
+    // Few tokens: 128 output features x all tokens per CTA, K split over a cluster, reduced through
+    // distributed shared memory.
+    using FC = GemmFewCfg<FMT>;
+    const int ntok = fewtok_ntok(M);
+    const int tiles = (int)((N + 127) / 128);
+    const int S = fewtok_cluster(tiles, (K + FC::BK - 1) / FC::BK, 1, st->sm_count);
+    if (!encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, krow, 128, 128) ||
+        !encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, krow, (uint32_t)ntok, 128))
+      return TORQ_ERR_LAUNCH;
+    launch_tc(gemm_fewtok_kernel<FMT>, S, tiles * S, FC::THREADS, FC::smem_bytes(ntok), s, tmB, tmA,
+              static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y, y_dtype == TORQ_BF16 ? 1 : 0, (int)M,
+              (int)N, (int)K, ntok, S, alpha, st->err_word);
+    return launch_status();
+  }
   // CTA pairs from two row tiles on -- except for exactly two row tiles with so few 256-column tiles
   // that the pairs would leave more than half of the SMs idle: 128 x 128 tiles on single CTAs then
   // put four times as many SMs to work on streaming W.

@@ -302,8 +302,9 @@ def test_rotated_linear_end_to_end_tiny_config():
 
 @pytest.mark.parametrize("M", [1, 33, 128])
 def test_rotated_linear_few_tokens_takes_the_split_rotation(M):
-    """Few tokens with a workspace: the rotation is split along its contraction over the SMs and a second
-    kernel adds the partials, rotates inside the blocks and quantizes (three launches instead of two)."""
+    """Few tokens: the rotation is split along its contraction over the SMs.  Up to 64 tokens one kernel
+    reduces the splits through distributed shared memory; above, the partial sums go through the workspace
+    and a second kernel adds them, rotates inside the blocks and quantizes (three launches instead of two)."""
     cfg = I.CONFIGS["tiny"]
     d, N = 1024, 256
     xb = I.activations(cfg, M=M, d=d)
@@ -324,7 +325,7 @@ def test_rotated_linear_few_tokens_takes_the_split_rotation(M):
                                        dbg_codes=dbg_c, dbg_scales=dbg_s)
     torch.cuda.synchronize()
     assert torq.torq_last_device_error() == 0
-    assert torq.torq_launch_count() - n0 == 3
+    assert torq.torq_launch_count() - n0 == (2 if M <= 64 else 3)   # up to 64 tokens: one rotation kernel, K splits reduced on chip
     g_codes, g_sb = _to_numpy(dbg_c, dbg_s, M, d)
     o_codes, o_sb = O.quantize_nvfp4(z.astype(np.float32), x_ts)
     rep = _mismatch(g_codes, g_sb, o_codes, o_sb, x_ts)

@@ -54,7 +54,9 @@ def test_tiny_config_all_three_formats():
     Nq, Ns, ts = torq.torq_prepare_weights_nvfp4(Rd, ri32, Wd)
     torch.cuda.synchronize()
     n_codes, n_sb, n_ts = O.prepare_weights_nvfp4(rb, ri16, w)
-    assert abs(ts - float(n_ts)) <= 2e-7 * float(n_ts)        # the maximum itself is an fp32 sum: one ulp at most
+    # the maximum is itself an fp32 tensor-core sum over 3 d terms: up to one unit in the last place (2^-23) lost
+    # in each of its 3 d / 16 accumulation steps, plus the intra-block step and the division
+    assert abs(ts - float(n_ts)) <= (3 * cfg.d / 16 + 34) * 2.0 ** -23 * float(n_ts)
     gc = O.unpack_codes(Nq.cpu().numpy())
     gs = O.nv_unswizzle_scales(Ns.cpu().numpy(), cfg.N, cfg.d)
     if ts == float(n_ts):
@@ -134,7 +136,7 @@ def test_llama3_qkv_weight_sampled_rows_and_the_nvfp4_tensor_scale():
     for n0 in range(0, N, 1024):
         amax = max(amax, float(np.abs(w[:, n0:n0 + 1024].astype(np.float64).T @ rt).max()))
     o_ts = O.tensor_scale_from_amax(np.float32(amax))
-    assert abs(ts - float(o_ts)) <= 2e-7 * float(o_ts)
+    assert abs(ts - float(o_ts)) <= (3 * d / 16 + 34) * 2.0 ** -23 * float(o_ts)       # see the tiny case
     z16 = _rows_of_w_prime(rb, ri16, w, cols, block=16).astype(np.float32)
     n_codes, n_sb = O.quantize_nvfp4(z16, np.float32(ts))       # the scale the device used, so thresholds coincide
     gc = O.unpack_codes(Nq[torch.from_numpy(cols).cuda()].cpu().numpy())
@@ -143,7 +145,12 @@ def test_llama3_qkv_weight_sampled_rows_and_the_nvfp4_tensor_scale():
     lat = np.abs(lattice(gc) - lattice(n_codes))
     assert step.max() <= 1 and lat.max() <= 1
     same = np.repeat(step == 0, 16, axis=1)
-    assert (step != 0).sum() <= 1e-4 * step.size and ((lat != 0) & same).sum() <= 1e-4 * lat.size
+    # Block scales: E4M3 has eight rounding thresholds per octave of the block maximum (density 8 / ln 2 per unit of
+    # ln amax), and a block maximum is an fp32 tensor-core sum over 3 d terms, 3 d / 16 accumulation steps that may
+    # each lose one unit in the last place: delta = (3 d / 16) 2^-23 = 9.2e-5, so at most (8 / ln 2) delta = 1.06e-3
+    # of the blocks can carry the neighbouring scale byte (observed 3e-4).  Elements of equal-scale blocks: 1e-4.
+    scale_bound = 8.0 / np.log(2.0) * (3 * d / 16) * 2.0 ** -23
+    assert (step != 0).sum() <= scale_bound * step.size and ((lat != 0) & same).sum() <= 1e-4 * lat.size
     assert torq.torq_last_device_error() == 0
 
 
