@@ -11,7 +11,7 @@
 // writes its partial [token][feature] into its own shared memory, a cluster barrier publishes them,
 // and CTA r then adds, for the tokens m = r (mod S), the S partials in rank order through
 // distributed shared memory (plain ld.shared::cluster; fixed order) and stores that token's 128
-// outputs as whole 128- or 256-byte pieces of a row of Y.
+// outputs as one 256- or 512-byte piece of a row of Y.
 //
 // Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (scale chunks shared -> tensor memory, then the
 // instructions), warps 2..5 epilogue / reduction.  Shared memory: 4 stages of (16 KiB of W + tokens x
@@ -48,7 +48,7 @@ struct GemmFewCfg {
 // grid = ceil(N / 128) * S CTAs in clusters of S along x: CTA b works feature tile b / S, k split b % S.
 // tmW: Wq [N, K bytes] box [128 x 128]; tmA: Aq [M, K bytes] box [ntok x 128]; As / Ws: tiled scales.
 template <int FMT = FMT_MXFP4>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(192, 2)
 gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA,
                    const uint8_t* __restrict__ As, const uint8_t* __restrict__ Ws, void* __restrict__ Y,
                    int y_is_bf16, int M, int N, int K, int ntok, int S, float alpha, int* err_word) {
@@ -182,55 +182,86 @@ gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     if (ok && elect_one()) tc_commit(accf_bar);
     __syncwarp();
   } else {
-    // ------------------------------------------------------------------ epilogue 1: partial tile -> own shared memory
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // Two passes over the SAME instructions, as in the few-token rotation: pass 0 is a dry run while the
+    // mainloop streams (reads this CTA's own shared memory, stores nothing) so that the reduction's code is
+    // in the instruction cache when it is needed; pass 1: accumulator -> own shared memory, cluster
+    // barrier, then the tokens of this CTA.
+    // A warp takes one token per pass: lane l adds features 4 l .. 4 l + 3 (16-byte loads, 512 contiguous
+    // bytes per warp and partial) and stores 8 or 16 bytes of the token's row of Y.  Two tokens per
+    // iteration, all their loads issued before the first add: few round trips through the cluster.
     const int q = warp & 3;
-    acc_ok = mbar_wait(accf_bar, 0, cta_abort, err_word, SITE_EPI_ACC_FULL);
-    acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
-    if (acc_ok) {
-      tc_fence_after_sync();
-      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
-      float* prow = P + q * 32 + lane;                   // feature 32 q + lane of token 0
-      for (int c0 = 0; c0 < ntok; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld_32x32_x16(tacc + c0, v);
-        tmem_ld_wait();
+    const int ew = warp - 2;
+    const int64_t n = (int64_t)nt * C::BF + 4 * lane;
+    const uint32_t p_saddr = smem_u32(P);
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {
+      const bool live = pass == 1;
+      if (live) {
+        // ---- epilogue 1: partial tile -> own shared memory
+        acc_ok = mbar_wait(accf_bar, 0, cta_abort, err_word, SITE_EPI_ACC_FULL);
+        acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
+        if (acc_ok) {
+          tc_fence_after_sync();
+          const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
+          float* prow = P + q * 32 + lane;               // feature 32 q + lane of token 0
+          for (int c0 = 0; c0 < ntok; c0 += 16) {
+            uint32_t v[16];
+            tmem_ld_32x32_x16(tacc + c0, v);
+            tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 16; ++j) prow[(c0 + j) * C::BF] = __uint_as_float(v[j]);
+            for (int j = 0; j < 16; ++j) prow[(c0 + j) * C::BF] = __uint_as_float(v[j]);
+          }
+        }
+        tc_fence_before_sync();
+        cluster_sync_all();                              // every CTA's partial tile is visible cluster-wide
+      }
+      // ---- epilogue 2: add the partials, store Y
+      uint32_t p_rank[C::MAX_CLUSTER];
+#pragma unroll
+      for (int s = 0; s < C::MAX_CLUSTER; ++s)
+        p_rank[s] = s < S ? map_to_cta(p_saddr, live ? (uint32_t)s : (uint32_t)rank) : 0u;
+      for (int m0 = rank + S * ew; m0 < M; m0 += 8 * S) {
+        float4 part[2][C::MAX_CLUSTER];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int m = m0 + 4 * S * j;
+          if (m < M) {
+            const uint32_t off = (uint32_t)((m * C::BF + 4 * lane) * 4);
+#pragma unroll
+            for (int s = 0; s < C::MAX_CLUSTER; ++s)
+              if (s < S)
+                asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(part[j][s].x), "=f"(part[j][s].y), "=f"(part[j][s].z), "=f"(part[j][s].w)
+                             : "r"(p_rank[s] + off));
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int m = m0 + 4 * S * j;
+          if (m < M) {
+            float4 y = make_float4(0.f, 0.f, 0.f, 0.f);  // rank order: the result does not depend on timing
+#pragma unroll
+            for (int s = 0; s < C::MAX_CLUSTER; ++s)
+              if (s < S) { y.x += part[j][s].x; y.y += part[j][s].y; y.z += part[j][s].z; y.w += part[j][s].w; }
+            if constexpr (FMT == FMT_NVFP4) { y.x *= alpha; y.y *= alpha; y.z *= alpha; y.w *= alpha; }
+            if (live && n < N) {                         // N % 8 == 0: four features are inside or outside together
+              if (y_is_bf16) {
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(y.x, y.y), h1 = __floats2bfloat162_rn(y.z, y.w);
+                *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(Y) + (int64_t)m * N + n) =
+                    make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
+              } else {
+                *reinterpret_cast<float4*>(reinterpret_cast<float*>(Y) + (int64_t)m * N + n) = y;
+              }
+            }
+          }
+        }
       }
     }
   }
-  tc_fence_before_sync();
-  cluster_sync_all();                                    // every CTA's partial tile is visible cluster-wide
-
-  if (warp >= 2) {
-    // ------------------------------------------------------------------ epilogue 2: add the partials, store Y
-    const int e = threadIdx.x - 64;                      // 0..127
-    const int n_local = (e & 63) * 2;                    // this thread's pair of features
-    const int64_t n = (int64_t)nt * C::BF + n_local;
-    const uint32_t p_saddr = smem_u32(P);
-    for (int m = rank + S * (e >> 6); m < M; m += 2 * S) {
-      const uint32_t off = (uint32_t)((m * C::BF + n_local) * 4);
-      float y0 = 0.f, y1 = 0.f;
-#pragma unroll
-      for (int s = 0; s < C::MAX_CLUSTER; ++s) {
-        if (s < S) {
-          float a, b;
-          asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];"
-                       : "=f"(a), "=f"(b) : "r"(map_to_cta(p_saddr, (uint32_t)s) + off) : "memory");
-          y0 += a;
-          y1 += b;
-        }
-      }
-      if constexpr (FMT == FMT_NVFP4) { y0 *= alpha; y1 *= alpha; }
-      if (n < N) {
-        if (y_is_bf16) {
-          __nv_bfloat162 h = __floats2bfloat162_rn(y0, y1);
-          *reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(Y) + (int64_t)m * N + n) = h;
-        } else {
-          *reinterpret_cast<float2*>(reinterpret_cast<float*>(Y) + (int64_t)m * N + n) = make_float2(y0, y1);
-        }
-      }
-    }
+  if (warp < 2) {                                        // the epilogue warps passed this barrier inside their pass 1
+    tc_fence_before_sync();
+    cluster_sync_all();
   }
 
   // ------------------------------------------------------------------ teardown

@@ -17,11 +17,12 @@ namespace torq {
 // of 80 bytes (32 bf16 + padding: conflict-free ldmatrix); ignored when !has_intra.  Rows row0 ..
 // row0 + 15 of the output; rows >= M get no codes and a zero scale byte.  blk: 32-block index along d.
 // Scale bytes go to the single-byte positions of the tiled layout (16-blocks 2 blk, 2 blk + 1 for NVFP4).
+// store == false: everything is computed and nothing is written (a dry pass over the same instructions).
 template <int FMT>
 __device__ __forceinline__ void intra_quantize_rows16(const float* y_s, uint32_t r_saddr, bool has_intra, int lane,
                                                       int row0, int M, int blk, int d, int nblocks,
                                                       float tensor_scale, uint8_t* __restrict__ codes,
-                                                      uint8_t* __restrict__ scales) {
+                                                      uint8_t* __restrict__ scales, bool store = true) {
   const int p = lane & 3, r8 = lane >> 2;
   const int kb4 = FMT == FMT_NVFP4 ? (2 * nblocks + 3) / 4 : (nblocks + 3) / 4;
   float acc[4][4];
@@ -46,16 +47,25 @@ __device__ __forceinline__ void intra_quantize_rows16(const float* y_s, uint32_t
         const int ai = (n >> 1) * 4 + (n & 1) * 2 + rh;
         split3_bf16x2(__float_as_uint(yp[0]), __float_as_uint(yp[1]), ah[ai], am[ai], al[ai]);
       }
+    // one accumulator per term, so that only two instructions depend on each other (a single chain of
+    // six was a third of this function's time); the terms are added smallest first
+    float accm[4][4], acch[4][4];
 #pragma unroll
-    for (int n = 0; n < 4; ++n) { acc[n][0] = 0.f; acc[n][1] = 0.f; acc[n][2] = 0.f; acc[n][3] = 0.f; }
+    for (int n = 0; n < 4; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { acc[n][e] = 0.f; accm[n][e] = 0.f; acch[n][e] = 0.f; }
 #pragma unroll
     for (int kc = 0; kc < 2; ++kc)
 #pragma unroll
       for (int n = 0; n < 4; ++n) {
         mma_16816_bf16(acc[n], al + 4 * kc, bfrag[kc][n]);
-        mma_16816_bf16(acc[n], am + 4 * kc, bfrag[kc][n]);
-        mma_16816_bf16(acc[n], ah + 4 * kc, bfrag[kc][n]);
+        mma_16816_bf16(accm[n], am + 4 * kc, bfrag[kc][n]);
+        mma_16816_bf16(acch[n], ah + 4 * kc, bfrag[kc][n]);
       }
+#pragma unroll
+    for (int n = 0; n < 4; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[n][e] = (acc[n][e] + accm[n][e]) + acch[n][e];
   } else {
 #pragma unroll
     for (int n = 0; n < 4; ++n)
@@ -71,7 +81,7 @@ __device__ __forceinline__ void intra_quantize_rows16(const float* y_s, uint32_t
     const float v[8] = {acc[0][2 * rh], acc[0][2 * rh + 1], acc[1][2 * rh], acc[1][2 * rh + 1],
                         acc[2][2 * rh], acc[2][2 * rh + 1], acc[3][2 * rh], acc[3][2 * rh + 1]};
     const int row = row0 + r8 + 8 * rh;
-    const bool live = row < M;
+    const bool live = store && row < M;
     uint32_t word, sb;
     if constexpr (FMT == FMT_MXINT4) {
       uint32_t pr[4];
@@ -86,7 +96,7 @@ __device__ __forceinline__ void intra_quantize_rows16(const float* y_s, uint32_t
       else quantize_row_fragment(v, p, word, sb);
       if (live) *reinterpret_cast<uint32_t*>(codes + (size_t)row * (d / 2) + blk * 16 + 4 * p) = word;
     }
-    if (p == 0) {
+    if (p == 0 && store) {
       if constexpr (FMT == FMT_NVFP4) {
         scales[scale_offset(row, 2 * blk, kb4)] = live ? (uint8_t)(sb & 0xFF) : (uint8_t)0;
         scales[scale_offset(row, 2 * blk + 1, kb4)] = live ? (uint8_t)(sb >> 8) : (uint8_t)0;

@@ -15,10 +15,14 @@
 // does not depend on timing), applies the intra-block rotation on the warp-level tensor cores (y split
 // into three bf16 terms, fp32 accumulation) and quantizes (Eq. 1).
 //
+// Units: epilogue warp w of every CTA owns 32-block w of the tile (its R_intra block is fetched into
+// shared memory when the kernel starts, long before it is needed: a first touch of that array from a
+// cold TLB costs microseconds); CTA r of the cluster takes the token groups r, r + S, ...
+//
 // Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue / reduction.
 // Shared memory: 4 stages of (16 KiB of R_inter + tokens x 128 B of X); after the mainloop the same
-// memory holds the partial tile and the per-warp staging of the reduction.  Small enough (<= 97 KiB)
-// for the CTAs of the kernel that follows in the stream to become resident beside this one.
+// memory holds the partial tile and the per-warp staging of the reduction.  Small enough (<= 107 KiB)
+// for two CTAs per SM: the grid may exceed the SM count, which keeps more loads in flight.
 #pragma once
 #include <cuda_bf16.h>
 #include "intra_fragment.cuh"
@@ -33,29 +37,24 @@ struct RotFewCfg {
   static constexpr int A_BOX_BYTES = 64 * 64 * 2;
   static constexpr int STAGES = 4;
   static constexpr int MAX_TOK = 64;
-  static constexpr int WARP_SCRATCH = 16 * 33 * 4 + 32 * 80;      // y tile + R_intra block per epilogue warp
+  static constexpr int Y_BYTES = 16 * 33 * 4;          // per epilogue warp: 16 tokens x 32 features, row stride 33
+  static constexpr int RI_BYTES = 32 * 80;             // per epilogue warp: R_intra[block] as bf16 rows of 80 bytes
   static constexpr int BAR_BYTES = 256;
   static constexpr int THREADS = 192;
   static constexpr int MAX_CLUSTER = 8;
   __host__ __device__ static constexpr int stage_bytes(int ntok) { return A_BYTES + ntok * BK * 2; }
   __host__ __device__ static constexpr int smem_bytes(int ntok) {
-    return STAGES * stage_bytes(ntok) + BAR_BYTES + 1024;
+    return STAGES * stage_bytes(ntok) + BAR_BYTES + 4 * RI_BYTES + 1024;
   }
-  // the reduction's buffers must fit inside the stages they reuse
-  static_assert(MAX_TOK * BF * 4 + 4 * WARP_SCRATCH <= STAGES * (A_BYTES + 16 * BK * 2), "reduction buffers");
+  // the partial tile and the warps' y tiles must fit inside the stages they reuse
+  static_assert(MAX_TOK * BF * 4 + 4 * Y_BYTES <= STAGES * (A_BYTES + 16 * BK * 2), "reduction buffers");
 };
-
-__device__ __forceinline__ float ld_shared_cluster_f32(uint32_t cluster_addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
-  return v;
-}
 
 // grid = (d / 128) * S CTAs in clusters of S along x: CTA b works feature tile b / S, k split b % S.
 // tmX: X [M, d] bf16, box [ntok rows x 64]; tmR: R_inter [d, d] bf16, box [64 x 64].  ntok = 16, 32 or 64
 // >= M.  d % 128 == 0.  `codes` / `scales` / `tensor_scale` as in rotate_quantize_kernel for FMT.
 template <int FMT = FMT_MXFP4>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(192, 2)
 rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
                      const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
                      uint8_t* __restrict__ scales, int M, int d, int ntok, int S, float tensor_scale,
@@ -72,9 +71,10 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   const uint32_t accf_bar = bar_base + 8u * (2 * C::STAGES);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + bar_off + 192);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(smem_gen + bar_off + 200);
-  // after the mainloop: partial tile P[token][feature] fp32 at offset 0, then the warps' staging
+  // after the mainloop: partial tile P[token][feature] fp32 at offset 0, then the warps' y tiles
   float* P = reinterpret_cast<float*>(smem_gen);
-  uint8_t* scratch = smem_gen + ntok * C::BF * 4;
+  uint8_t* y_tiles = smem_gen + ntok * C::BF * 4;
+  uint8_t* ri_tiles = smem_gen + bar_off + C::BAR_BYTES;    // not part of the stages: filled at kernel start
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = blockIdx.x % S, ft = blockIdx.x / S;
@@ -109,6 +109,17 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
       }
     }
     __syncwarp();
+  }
+  const int groups = ntok / 16;                          // token groups of 16; group g belongs to CTA g % S
+  if (warp >= 2 && R_intra != nullptr && rank < groups) {
+    // this warp's R_intra block (a constant of the layer as well), 128 pieces of 16 B: row piece / 4
+    uint8_t* r_s = ri_tiles + (warp - 2) * C::RI_BYTES;
+    const uint4* src = reinterpret_cast<const uint4*>(R_intra + (size_t)(ft * 4 + (warp - 2)) * 1024);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int piece = lane + 32 * i;
+      *reinterpret_cast<uint4*>(r_s + (piece >> 2) * 80 + (piece & 3) * 16) = __ldg(src + piece);
+    }
   }
   griddep_wait();
 
@@ -160,65 +171,83 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     if (ok && elect_one()) tc_commit(accf_bar);
     __syncwarp();
   } else {
-    // ------------------------------------------------------------------ epilogue 1: partial tile -> own shared memory
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // Two passes over the SAME instructions.  Pass 0 is a dry run while the mainloop streams: it reads
+    // this CTA's own shared memory (whatever it holds), computes, and stores nothing.  Its only purpose
+    // is to have the reduction's code in the instruction cache: executed cold, after the mainloop,
+    // that code cost about 2.5 us of instruction fetches -- a fifth of the kernel.  Pass 1 is the
+    // real one: accumulator -> own shared memory, cluster barrier, then the units of this warp.
     const int q = warp & 3;
-    acc_ok = mbar_wait(accf_bar, 0, cta_abort, err_word, SITE_EPI_ACC_FULL);
-    acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
-    if (acc_ok) {
-      tc_fence_after_sync();
-      // every load into the stages has landed and every instruction that read them has completed
-      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
-      float* prow = P + q * 32 + lane;                   // feature 32 q + lane of token 0
-      for (int c0 = 0; c0 < ntok; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld_32x32_x16(tacc + c0, v);
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 16; ++j) prow[(c0 + j) * C::BF] = __uint_as_float(v[j]);
-      }
-    }
-  }
-  tc_fence_before_sync();
-  cluster_sync_all();                                    // every CTA's partial tile is visible cluster-wide
-
-  if (warp >= 2) {
-    // ------------------------------------------------------------------ epilogue 2: reduce, intra-rotate, quantize
-    const int ew = warp - 2;                             // 0..3
-    const int groups = ntok / 16;                        // token groups of 16
-    const int units = 4 * groups;                        // (32-block of the tile, token group)
+    const int ew = warp - 2;                             // 0..3 = 32-block of the tile
     const int nblocks = d / 32;
-    float* y_s = reinterpret_cast<float*>(scratch + ew * C::WARP_SCRATCH);
-    uint8_t* r_s = scratch + ew * C::WARP_SCRATCH + 16 * 33 * 4;
+    const int blk = ft * 4 + ew;
+    float* y_s = reinterpret_cast<float*>(y_tiles + ew * C::Y_BYTES);
+    const uint32_t r_saddr = smem_u32(ri_tiles + ew * C::RI_BYTES);
     const uint32_t p_saddr = smem_u32(P);
-    // unit u belongs to CTA u % S, and there to warp (u / S) % 4
-    for (int u = rank + S * ew; u < units; u += 4 * S) {
-      const int qb = u / groups, g = u - qb * groups;
-      const int blk = ft * 4 + qb;
-      if (R_intra != nullptr) {
+    // lane l adds tokens (l / 8) + 4 j, j = 0..3, features 4 (l % 8) .. + 3 of the block, two tokens at a
+    // time: their 2 S loads of 16 bytes go out before the first add, so a unit costs two round trips
+    // through the cluster
+    const int tr = lane >> 3, fc = (lane & 7) * 4;
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {
+      const bool live = pass == 1;
+      if (live) {
+        // ---- epilogue 1: partial tile -> own shared memory
+        acc_ok = mbar_wait(accf_bar, 0, cta_abort, err_word, SITE_EPI_ACC_FULL);
+        acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
+        if (acc_ok) {
+          tc_fence_after_sync();
+          // every load into the stages has landed and every instruction that read them has completed
+          const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
+          float* prow = P + q * 32 + lane;               // feature 32 q + lane of token 0
+          for (int c0 = 0; c0 < ntok; c0 += 16) {
+            uint32_t v[16];
+            tmem_ld_32x32_x16(tacc + c0, v);
+            tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {                    // 128 pieces of 16 B: row (piece / 4), 8 columns each
-          const int piece = lane + 32 * i;
-          *reinterpret_cast<uint4*>(r_s + (piece >> 2) * 80 + (piece & 3) * 16) =
-              __ldg(reinterpret_cast<const uint4*>(R_intra + (size_t)blk * 1024) + piece);
+            for (int j = 0; j < 16; ++j) prow[(c0 + j) * C::BF] = __uint_as_float(v[j]);
+          }
         }
+        tc_fence_before_sync();
+        cluster_sync_all();                              // every CTA's partial tile is visible cluster-wide
       }
-      // 16 tokens x 32 features: the S partials in rank order (rows >= M are zero in every partial)
-      const uint32_t off = (uint32_t)(((16 * g) * C::BF + qb * 32 + lane) * 4);
-#pragma unroll 4
-      for (int t = 0; t < 16; ++t) {
-        float part[C::MAX_CLUSTER];
+      // ---- epilogue 2: reduce, intra-rotate, quantize
+      uint32_t p_rank[C::MAX_CLUSTER];
 #pragma unroll
-        for (int s = 0; s < C::MAX_CLUSTER; ++s)
-          part[s] = s < S ? ld_shared_cluster_f32(map_to_cta(p_saddr, (uint32_t)s) + off + (uint32_t)(t * C::BF * 4)) : 0.f;
-        float y = 0.f;
+      for (int s = 0; s < C::MAX_CLUSTER; ++s)
+        p_rank[s] = s < S ? map_to_cta(p_saddr, live ? (uint32_t)s : (uint32_t)rank) : 0u;
+      for (int g = rank; g < groups; g += S) {
 #pragma unroll
-        for (int s = 0; s < C::MAX_CLUSTER; ++s) if (s < S) y += part[s];
-        y_s[t * 33 + lane] = y;
+        for (int jh = 0; jh < 2; ++jh) {
+          if (16 * g + 8 * jh >= M) break;               // rows 8 jh .. 8 jh + 7 of the group hold no token
+          float4 part[2][C::MAX_CLUSTER];
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const uint32_t off = (uint32_t)(((16 * g + tr + 4 * (2 * jh + j)) * C::BF + ew * 32 + fc) * 4);
+#pragma unroll
+            for (int s = 0; s < C::MAX_CLUSTER; ++s)
+              if (s < S)
+                asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(part[j][s].x), "=f"(part[j][s].y), "=f"(part[j][s].z), "=f"(part[j][s].w)
+                             : "r"(p_rank[s] + off));
+          }
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            float4 y = make_float4(0.f, 0.f, 0.f, 0.f);  // rank order: the result does not depend on timing
+#pragma unroll
+            for (int s = 0; s < C::MAX_CLUSTER; ++s)
+              if (s < S) { y.x += part[j][s].x; y.y += part[j][s].y; y.z += part[j][s].z; y.w += part[j][s].w; }
+            if (live) {                                  // the y tile lies inside the stages: untouched while they are in use
+              float* dst = y_s + (tr + 4 * (2 * jh + j)) * 33 + fc;
+              dst[0] = y.x; dst[1] = y.y; dst[2] = y.z; dst[3] = y.w;
+            }
+          }
+        }
+        __syncwarp();
+        intra_quantize_rows16<FMT>(y_s, r_saddr, R_intra != nullptr, lane, 16 * g, M, blk, d, nblocks, tensor_scale,
+                                   codes, scales, live);
+        __syncwarp();
       }
-      __syncwarp();
-      intra_quantize_rows16<FMT>(y_s, smem_u32(r_s), R_intra != nullptr, lane, 16 * g, M, blk, d, nblocks,
-                                 tensor_scale, codes, scales);
-      __syncwarp();
     }
     // scale bytes of the rows no unit covers (ntok .. 127 of the single 128-row scale tile): zero
     if (rank == 0) {
@@ -232,6 +261,10 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         }
       }
     }
+  }
+  if (warp < 2) {                                        // the epilogue warps passed this barrier inside their pass 1
+    tc_fence_before_sync();
+    cluster_sync_all();
   }
 
   // ------------------------------------------------------------------ teardown

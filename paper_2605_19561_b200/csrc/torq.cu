@@ -217,12 +217,16 @@ static int rotation_splits(int64_t M, int64_t d, int sm_count) {
   return s < 2 ? 1 : s;
 }
 // Few-token kernels (M <= 64): tokens per instruction and the cluster size = number of K splits of
-// one 128-feature tile, as many as fill the SMs (at most 8, each split at least `min_k` K steps).
+// one 128-feature tile.  Two of these CTAs fit on an SM, and a grid of about 1.4 CTAs per SM measured
+// fastest (more loads in flight; beyond that the clusters no longer all become resident at once):
+// the largest S <= 8 with tiles * S <= 1.4 SMs, each split at least `min_k` K steps.  7 is skipped:
+// clusters of 7 did not all become resident at sizes where 6 and 8 did.
 static inline int fewtok_ntok(int64_t M) { return M <= 16 ? 16 : (M <= 32 ? 32 : 64); }
 static inline int fewtok_cluster(int64_t tiles, int64_t k_steps, int min_k, int sm_count) {
-  int64_t s = sm_count / (tiles > 0 ? tiles : 1);
+  int64_t s = (int64_t)sm_count * 14 / 10 / (tiles > 0 ? tiles : 1);
   if (s > 8) s = 8;
   if (s > k_steps / min_k) s = k_steps / min_k;
+  if (s == 7) s = 6;
   return s < 1 ? 1 : (int)s;
 }
 static size_t quantized_bytes(int64_t M, int64_t d) {    // codes, then 256-byte aligned the scales
