@@ -1,6 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the rotated-MXFP4 linear hot path (rotate -> MXFP4 quantize -> block-scaled FP4
-GEMM) at the LLaMA3-8B QKV-projection shape (M=2048 tokens, d=4096, N=6144, bf16 output).
+GEMM).  The timed K steps run the LLaMA3-8B QKV-projection shape (M=2048 tokens, d=4096, N=6144,
+bf16 output); the same line also carries the second 8B shape (down-projection, 2048 x 14336 ->
+4096) and a token sweep at d = N = 5120 (M = 1, 64, 1024, 16384), each with per-kernel times,
+both roofline fractions and the SM clock sampled inside its own loop.
 
 One step = one pass of the whole path over one batch of seeded synthetic activations.  Prints ONE
 JSON line (rank 0).  `--impl reference` times the CPU checker (oracle/) on the host cores instead.
@@ -24,7 +27,6 @@ import torch
 
 METRIC = "rotate+MXFP4-quant GB/s and MXFP4 GEMM TFLOP/s, % of roofline (8B shapes)"
 WORKLOAD = "llama3_8b_qkv"
-N_BUFFER_SETS = 4          # rotated between steps: 4 x ~92 MB of operands > 126 MB of L2
 
 
 def profiled_traffic(kernel: str, workload: str):
@@ -57,18 +59,20 @@ def peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks / throttle reasons of one GPU while the timed region runs."""
+    """Samples nvidia-smi clocks / throttle reasons of one GPU (every 20 ms, each sample with the
+    host time it was read at) so that every timed loop can be given the clock it ran at."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index: int):
-        self.index, self.proc, self.lines = index, None, []
+        self.index, self.proc, self.samples = index, None, []
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -77,31 +81,40 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm, mx = float(f[0]), float(f[1])
+            except ValueError:
+                continue
+            reasons = [n for n, v in zip(self.NAMES, f[4:8]) if v.lower().startswith("active")]
+            self.samples.append((time.time(), sm, mx, reasons))
+
+    def window(self, t0: float, t1: float):
+        """Median SM MHz and the throttle reasons seen between two host times (None without samples)."""
+        sel = [s for s in list(self.samples) if t0 <= s[0] <= t1]
+        if not sel:
+            return {"sm_mhz": None, "samples": 0, "reasons": []}
+        return {"sm_mhz": float(np.median([s[1] for s in sel])), "samples": len(sel),
+                "reasons": sorted({r for s in sel for r in s[3]})}
 
     def stop(self):
         if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for l in self.lines:
-            f = [x.strip() for x in l.split(",")]
-            if len(f) < 8:
-                continue
-            try:
-                sm.append(float(f[0])); mx.append(float(f[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, f[4:8]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+
+    def summary(self, t0: float, t1: float):
+        w = self.window(t0, t1)
+        mx = [s[2] for s in list(self.samples)]
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        return {"sm_mhz": w["sm_mhz"], "sm_max_mhz": max(mx) if mx else None, "samples": w["samples"],
+                "reasons": w["reasons"]}
 
 
 def time_oracle(cfg, rows: int, steps: int, warmup: int):
@@ -165,214 +178,340 @@ def run_reference(args):
     }))
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None, help="default: 2000 (the CUDA path), 20 (--impl reference)")
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default=WORKLOAD, help="one of inputs.CONFIGS (default: the LLaMA3-8B QKV shape)")
-    ap.add_argument("--M", type=int, default=None, help="override the number of tokens (token sweep)")
-    args = ap.parse_args()
-    if args.steps is None:
-        args.steps = 20 if args.impl == "reference" else 2000
-    if args.impl == "reference":
-        return run_reference(args)
 
-    from paper_2605_19561_b200 import inputs as I
-    from paper_2605_19561_b200 import torq
+MIN_LOOP_MS = 100.0        # every per-kernel measurement lasts at least this long, whatever --steps is
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    warmup = max(args.warmup, 3)
-    cfg = I.CONFIGS[args.workload]
-    M, d, N = (args.M or cfg.M), cfg.d, cfg.N
-    pk = peaks()
 
-    # ---- inputs (seeded, synthetic; every rank holds its own M rows: weak scaling over tokens)
-    xb = I.activations(cfg, M=M)
-    # QR of the seeded Gaussian: LAPACK on the host up to d = 4096, on the device above (few host cores)
-    rb, rib, _, _ = I.rotations(cfg, device="cpu" if d <= 4096 else "cuda")
-    w = I.weights(cfg)
-    X0 = I.bf16_bits_to_tensor(xb, "cuda")
-    R0, Ri0 = I.bf16_bits_to_tensor(rb, "cuda"), I.bf16_bits_to_tensor(rib, "cuda")
-    Wq0, Ws0 = torq.prepare_weights(R0, Ri0, torch.from_numpy(w).cuda())
-    # the NVFP4 variant of the same layer (16-element blocks): its own intra rotations and weights
-    Ri32_nv = torq.torq_expand_intra16(I.bf16_bits_to_tensor(I.intra_rotations16(cfg), "cuda"))
-    torch.cuda.synchronize()
-    Wq_nv, Ws_nv, w_ts_nv = torq.prepare_weights_nvfp4(R0, Ri32_nv, torch.from_numpy(w).cuda())
-    # activation tensor scale, fixed ahead of time as a calibrated one would be: no rotated element
-    # exceeds its token's 2-norm, so the largest norm over the top of the E4M3 range never saturates
-    x_ts_nv = float(X0.float().norm(dim=1).max().item()) / (6.0 * 448.0)
-    ws_nv = [torch.empty(torq.torq_nvfp4_workspace_bytes(M, d, N), dtype=torch.uint8, device="cuda") for _ in range(2)]
-    # the MXINT4 variant (integer codes as E4M3 operand bytes, same rotations as the MXFP4 layer)
-    _, W8_i4, Ws_i4 = torq.prepare_weights_mxint4(R0, Ri0, torch.from_numpy(w).cuda())
-    ws_i4 = [torch.empty(torq.torq_mxint4_workspace_bytes(M, d, N), dtype=torch.uint8, device="cuda") for _ in range(2)]
-    del w
-    set_bytes = X0.numel() * 2 + R0.numel() * 2 + Wq0.numel() + M * N * 2
-    n_sets = max(2, min(N_BUFFER_SETS, int(8e9 // set_bytes)))     # bounded device memory
-    sets = []
-    for i in range(n_sets):
-        sets.append(dict(X=X0.clone(), R=R0.clone(), Ri=Ri0.clone(), Wq=Wq0.clone(), Ws=Ws0.clone(),
-                         Y=torch.empty((M, N), dtype=torch.bfloat16, device="cuda"),
-                         ws=torch.empty(torq.torq_workspace_bytes(M, d, N), dtype=torch.uint8, device="cuda")))
-    stream = torch.cuda.current_stream()
-    fp4_probe = max(torq.torq_probe_fp4_peak(40000) for _ in range(2))     # TFLOP/s, ~1 ms each
+class KernelTimer:
+    """Times one kernel (or one call of the library) as the average over back-to-back launches that
+    together last at least MIN_LOOP_MS, between one pair of CUDA events on the launching stream.
+    The launches are captured once in a CUDA graph (a batch that walks through the operand sets, so
+    consecutive launches read different memory) and the graph is replayed: the host then enqueues
+    nothing inside the timed region, which matters for kernels shorter than the host's cost of a
+    call (about 10 us).  If capture is not possible the batch is launched directly behind a busy
+    stream.  Returns the time per launch and the SM clock sampled while the loop ran."""
 
-    def step(i):
-        b = sets[i % n_sets]
-        torq.torq_rotated_linear(b["X"], b["R"], b["Ri"], b["Wq"], b["Ws"], Y=b["Y"], workspace=b["ws"])
+    def __init__(self, stream, sampler, n_sets):
+        self.stream, self.sampler, self.n_sets = stream, sampler, n_sets
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
+    def __call__(self, fn, batch=None, min_ms=MIN_LOOP_MS):
+        batch = batch or max(self.n_sets, 8) // self.n_sets * self.n_sets
+        s = self.stream
         torch.cuda.synchronize()
-
-    for i in range(warmup):
-        step(i)
-    barrier()
-    assert torq.torq_last_device_error() == 0
-
-    # ---- timed region: exactly K steps of the whole path, inputs resident in HBM
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    time.sleep(0.3)
-    launches0 = torq.torq_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    hold_gpu(stream)
-    e0.record(stream)
-    for i in range(args.steps):
-        step(i)
-    e1.record(stream)
-    barrier()
-    launches = torq.torq_launch_count() - launches0
-    ms_total = e0.elapsed_time(e1)
-
-    # ---- per-kernel durations: K back-to-back launches of one kernel (operand sets rotated), one
-    # event pair around them on the launching stream; average = event time / K.  (With an event
-    # between every launch the launch latency that normally overlaps the previous kernel's tail
-    # would be charged to the kernel.)
-    def codes_scales(b):
-        return b["ws"][: M * d // 2].view(M, d // 2), b["ws"][(M * d // 2 + 255) // 256 * 256:][: torq.torq_scales_bytes(M, d)]
-
-    def timed_loop(fn):
-        for i in range(3):
-            fn(sets[i % n_sets])
+        with torch.cuda.stream(s):
+            for i in range(max(3, self.n_sets)):
+                fn(i)
         torch.cuda.synchronize()
-        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        # at most 400 launches per measurement: a kernel shorter than the host's cost of enqueuing it
-        # (about 15 us through ctypes) is only timed correctly while the launches queued during the
-        # hold last
-        k = min(args.steps, 400)
-        hold_gpu(stream, ms=10.0)
-        a0.record(stream)
-        for i in range(k):
-            fn(sets[i % n_sets])
-        a1.record(stream)
-        torch.cuda.synchronize()
-        return a0.elapsed_time(a1) / k * 1e-3
+        graph = None
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=s):
+                for i in range(batch):
+                    fn(i)
+        except Exception as exc:
+            graph = None
+            torch.cuda.synchronize()
+            sys.stderr.write(f"[bench] graph capture not possible ({type(exc).__name__}: {exc}); direct launches\n")
 
-    def gemm_only(b):
-        c, sc = codes_scales(b)
-        torq.torq_mxfp4_gemm(c, sc, b["Wq"], b["Ws"], Y=b["Y"])
+        def run(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if graph is None:
+                hold_gpu(s, ms=10.0)
+            e0.record(s)
+            for _ in range(reps):
+                if graph is not None:
+                    graph.replay()
+                else:
+                    for i in range(batch):
+                        fn(i)
+            e1.record(s)
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1)
 
-    def rot_only(b):
-        c, sc = codes_scales(b)
-        torq.torq_rotate_quantize(b["X"], b["R"], b["Ri"], out_codes=c, out_scales=sc)
+        with torch.cuda.stream(s):
+            ms = run(2)                                     # estimate, also a warm-up of the graph
+            reps = max(2, int(np.ceil(min_ms / max(ms / 2, 1e-3))))
+            if graph is None:
+                reps = min(reps, max(1, 400 // batch))      # direct launches: only what queues behind the hold
+            t0 = time.time()
+            ms = run(reps)
+            t1 = time.time()
+        clk = self.sampler.window(t0, t1)
+        return {"s": ms * 1e-3 / (reps * batch), "launches": reps * batch, "loop_ms": ms, "sm_mhz": clk["sm_mhz"],
+                "reasons": clk["reasons"], "how": "cuda graph replay" if graph is not None else "direct launches"}
 
-    t_gemm = timed_loop(gemm_only)
-    # few output tiles: the rotation of the fused call is the split-K pair of kernels, which only runs
-    # with the workspace of the fused call; its time is the step minus the GEMM
-    sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
-    split_k = 2 * ((M + 127) // 128) * ((d + 255) // 256) <= sm_count     # the library's own rule
-    t_rot = max(ms_total / args.steps * 1e-3 - t_gemm, 1e-9) if split_k else timed_loop(rot_only)
-    # the same activations through the rotation in the paper's own structure (one B x B matrix
-    # across blocks, one shared intra-block matrix): reported beside the dense-R_inter path
-    t_struct = None
+
+def roof_record(kernel, tm, flop, nbytes, pk, tensor_burst, tensor_sustained, tensor_name, workload):
+    """Roofline record of one kernel: the binding bound is the slower of its HBM floor and its tensor
+    floor (at the burst peak).  `frac` is quoted against the burst peak; the fraction of the
+    sustained peak is printed beside it, never substituted for it."""
+    t = tm["s"]
+    t_hbm, t_tc = nbytes / (pk["hbm_gbs"] * 1e9), flop / (tensor_burst * 1e12)
+    rec = {"kernel": kernel, "ms_per_launch": t * 1e3, "launches_timed": tm["launches"], "loop_ms": tm["loop_ms"],
+           "sm_mhz_in_loop": tm["sm_mhz"], "throttle_reasons_in_loop": tm["reasons"], "timing": tm["how"],
+           "algorithmic_flop": flop, "algorithmic_bytes": nbytes, "traffic": profiled_traffic(kernel, workload)}
+    if t_tc >= t_hbm:
+        ach = flop / t / 1e12
+        rec.update({"bound": "tensor", "achieved": ach, "peak": tensor_burst, "unit": "TFLOP/s", "frac": ach / tensor_burst,
+                    "peak_source": tensor_name, "frac_of_burst": ach / tensor_burst})
+        if tensor_sustained:
+            rec["frac_of_sustained"] = ach / tensor_sustained
+    else:
+        ach = nbytes / t / 1e9
+        rec.update({"bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
+                    "peak_source": f"{pk['source']} HBM copy"})
+    return rec
+
+
+def layer_work(M, d, N):
+    """Algorithmic work of the two halves of the path (per call)."""
+    rot_flop = 2.0 * M * d * d + 64.0 * M * d
+    rot_bytes = 2.0 * M * d + 2.0 * d * d + 2.0 * 32 * d + M * d / 2 + M * d / 32
+    gemm_flop = 2.0 * M * N * d
+    gemm_bytes = M * d / 2 + M * d / 32 + N * d / 2 + N * d / 32 + 2.0 * M * N
+    return rot_flop, rot_bytes, gemm_flop, gemm_bytes
+
+
+def rotation_kernel_name(M, d, sm_count):
+    if M <= 64 and d % 128 == 0:
+        return "rotate_fewtok_kernel"
+    if 2 * ((M + 127) // 128) * ((d + 255) // 256) <= sm_count:
+        return "rotate_splitk_kernel + splitk_reduce_quantize_kernel"
+    return "rotate_quantize_pair_kernel" if M > 128 else "rotate_quantize_kernel"
+
+
+def gemm_kernel_name(M):
+    return "gemm_fewtok_kernel" if M <= 64 else ("mxfp4_gemm_pair_kernel" if M > 128 else "mxfp4_gemm_kernel")
+
+
+class Layer:
+    """Operands of one workload on the device: `n_sets` copies of everything a step reads, walked
+    through between steps so that no step finds its operands in L2 (skipped when one copy alone is
+    larger than L2)."""
+
+    def __init__(self, torq, I, name, M, max_bytes=10e9, shared=None):
+        cfg = I.CONFIGS[name]
+        self.name, self.M, self.d, self.N, self.cfg = name, M, cfg.d, cfg.N, cfg
+        d, N = cfg.d, cfg.N
+        self.X0 = I.bf16_bits_to_tensor(I.activations(cfg, M=M), "cuda")
+        if shared is None:
+            # QR of the seeded Gaussian: LAPACK on the host up to d = 4096, on the device above (few host cores)
+            rb, rib, _, _ = I.rotations(cfg, device="cpu" if d <= 4096 else "cuda")
+            self.R0, self.Ri0 = I.bf16_bits_to_tensor(rb, "cuda"), I.bf16_bits_to_tensor(rib, "cuda")
+            W = torch.from_numpy(I.weights(cfg)).cuda()
+            torch.cuda.synchronize()
+            self.Wq0, self.Ws0 = torq.torq_prepare_weights(self.R0, self.Ri0, W)
+            self.W = W
+        else:
+            self.R0, self.Ri0, self.Wq0, self.Ws0, self.W = shared.R0, shared.Ri0, shared.Wq0, shared.Ws0, shared.W
+        set_bytes = self.X0.numel() * 2 + self.R0.numel() * 2 + self.Wq0.numel() + M * N * 2
+        l2 = 126e6
+        want = 1 if set_bytes > 1.5 * l2 else int(np.ceil(2.2 * l2 / set_bytes)) + 1
+        self.n_sets = max(1, min(want, 6, int(max_bytes // set_bytes)))
+        self.l2_note = (f"{self.n_sets} operand sets walked through between steps ({self.n_sets * set_bytes / 1e6:.0f} MB "
+                        f"in all, L2 holds 126 MB)" if self.n_sets > 1 else
+                        f"one operand set of {set_bytes / 1e6:.0f} MB, larger than the 126 MB L2")
+        ws_bytes = torq.torq_workspace_bytes(M, d, N)
+        self.sets = []
+        for i in range(self.n_sets):
+            first = i == 0
+            self.sets.append(dict(X=self.X0 if first else self.X0.clone(), R=self.R0 if first else self.R0.clone(),
+                                  Ri=self.Ri0 if first else self.Ri0.clone(), Wq=self.Wq0 if first else self.Wq0.clone(),
+                                  Ws=self.Ws0 if first else self.Ws0.clone(),
+                                  Y=torch.empty((M, N), dtype=torch.bfloat16, device="cuda"),
+                                  ws=torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")))
+        self.torq = torq
+
+    def with_tokens(self, I, M):
+        """The same layer (rotations, weights) with another number of tokens."""
+        return Layer(self.torq, I, self.name, M, shared=self)
+
+    def codes_scales(self, b):
+        M, d = self.M, self.d
+        return (b["ws"][: M * d // 2].view(M, d // 2),
+                b["ws"][(M * d // 2 + 255) // 256 * 256:][: self.torq.torq_scales_bytes(M, d)])
+
+    def step(self, i):
+        b = self.sets[i % self.n_sets]
+        self.torq.torq_rotated_linear(b["X"], b["R"], b["Ri"], b["Wq"], b["Ws"], Y=b["Y"], workspace=b["ws"])
+
+    def rot(self, i):
+        b = self.sets[i % self.n_sets]
+        c, sc = self.codes_scales(b)
+        self.torq.torq_rotate_quantize(b["X"], b["R"], b["Ri"], out_codes=c, out_scales=sc)
+
+    def gemm(self, i):
+        b = self.sets[i % self.n_sets]
+        c, sc = self.codes_scales(b)
+        self.torq.torq_mxfp4_gemm(c, sc, b["Wq"], b["Ws"], Y=b["Y"])
+
+
+def measure_layer(layer, timer, pk, fp4_peak, sm_count, world):
+    """Step, rotate+quantize and GEMM of one workload, each in its own loop with its own clock sample."""
+    M, d, N = layer.M, layer.d, layer.N
+    rot_flop, rot_bytes, gemm_flop, gemm_bytes = layer_work(M, d, N)
+    t_step = timer(layer.step)
+    layer.rot(0)                                            # the GEMM-only loop reads these codes
+    t_gemm = timer(layer.gemm)
+    rk = rotation_kernel_name(M, d, sm_count)
+    if rk.startswith("rotate_splitk"):
+        # the split-K pair only runs with the fused call's workspace: its time is the step minus the GEMM
+        t_rot = dict(t_step)
+        t_rot["s"] = max(t_step["s"] - t_gemm["s"], 1e-9)
+        t_rot["how"] = "step minus GEMM (" + t_step["how"] + ")"
+    else:
+        t_rot = timer(layer.rot)
+    r_rot = roof_record(rk, t_rot, rot_flop, rot_bytes, pk, pk["bf16_burst"], pk["bf16_sustained"],
+                        f"{pk['source']} bf16 burst", layer.name)
+    r_rot["frac_of_nominal_2250_tflops"] = rot_flop / t_rot["s"] / 1e12 / 2250.0
+    r_rot["GBps"] = rot_bytes / t_rot["s"] / 1e9
+    r_gemm = roof_record(gemm_kernel_name(M), t_gemm, gemm_flop, gemm_bytes, pk, fp4_peak, None,
+                         "self-measured: torq_probe_fp4_peak (FP4 block-scaled MMA issue loop, no loads)", layer.name)
+    r_gemm["frac_of_nominal_9000_tflops"] = gemm_flop / t_gemm["s"] / 1e12 / 9000.0
+    r_gemm["frac_of_4x_measured_bf16_burst"] = gemm_flop / t_gemm["s"] / 1e12 / (4.0 * pk["bf16_burst"])
+    r_gemm["TFLOPs"] = gemm_flop / t_gemm["s"] / 1e12
+    return {"workload": layer.name, "M": M, "d": d, "N": N, "l2": layer.l2_note,
+            "ms_per_step": t_step["s"] * 1e3, "tokens_per_s": world * M / t_step["s"],
+            "sm_mhz_in_step_loop": t_step["sm_mhz"], "step_timing": t_step["how"],
+            "rotate_quantize": r_rot, "gemm": r_gemm}, t_step, t_rot, t_gemm
+
+
+def measure_variants(torq, I, layer, timer, pk, fp4_peak, t_rot, world):
+    """The widened paths on the main workload's activations: the rotation in the paper's own structure,
+    the NVFP4 and MXINT4 formats, and the one-GEMM (merged) form of the rotation."""
+    M, d, N, cfg = layer.M, layer.d, layer.N, layer.cfg
+    rot_flop, rot_bytes, gemm_flop, gemm_bytes = layer_work(M, d, N)
+    sets, n_sets = layer.sets, layer.n_sets
+    out = {}
+
+    def simple(tm):
+        return {"ms": tm["s"] * 1e3, "sm_mhz_in_loop": tm["sm_mhz"]}
+
+    # ---- the paper's structure: one B x B matrix across blocks, one shared intra-block matrix
     if d % 256 == 0:
         RB = I.bf16_bits_to_tensor(I.to_bf16_bits(I.orthogonal(d // 32, np.random.Generator(
             np.random.PCG64(I.BASE_SEED + 100 * cfg.cfg_id + 5)))), "cuda")
-        Ri1 = Ri0[0].contiguous()
+        Ri1 = layer.Ri0[0].contiguous()
 
-        def struct_only(b):
-            c, sc = codes_scales(b)
+        def struct_only(i):
+            b = sets[i % n_sets]
+            c, sc = layer.codes_scales(b)
             torq.torq_rotate_quantize_structured(b["X"], RB, Ri1, out_codes=c, out_scales=sc)
 
-        t_struct = timed_loop(struct_only)
-
-        def struct_layer(b):
+        def struct_layer(i):
+            b = sets[i % n_sets]
             torq.torq_rotated_linear_structured(b["X"], RB, Ri1, b["Wq"], b["Ws"], Y=b["Y"], workspace=b["ws"])
 
-        t_struct_layer = timed_loop(struct_layer)
-    # the NVFP4 variant: rotation + quantizer, GEMM, and the whole layer
-    def nv_codes_scales(k):
+        ts, tl = timer(struct_only), timer(struct_layer)
+        nbytes = 2.0 * M * d + 2.0 * (d // 32) ** 2 + 2048.0 + M * d / 2 + M * d / 32
+        out["structured_rotation"] = {
+            "kernel": "rotate_structured_kernel", "what": "rotate+quantize with R_inter = R_B (x) I_32 and one shared "
+            "R_intra (the paper's structure, 2d(B+32) flop per token) on the same activations", "bound": "hbm",
+            "ms_per_launch": ts["s"] * 1e3, "sm_mhz_in_loop": ts["sm_mhz"], "achieved": nbytes / ts["s"] / 1e9,
+            "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": nbytes / ts["s"] / 1e9 / pk["hbm_gbs"],
+            "algorithmic_bytes": nbytes, "traffic": profiled_traffic("rotate_structured_kernel", layer.name),
+            "speedup_over_dense_rotation": t_rot["s"] / ts["s"],
+            "whole_layer_ms_per_step": tl["s"] * 1e3, "whole_layer_tokens_per_s": world * M / tl["s"]}
+
+    # ---- the one-GEMM form: R_intra merged offline into R_inter (bf16), no intra step in the epilogue
+    Rm = [torq.torq_merge_rotations_bf16(b["R"], b["Ri"]) for b in sets]
+    torch.cuda.synchronize()
+
+    def merged_only(i):
+        b = sets[i % n_sets]
+        c, sc = layer.codes_scales(b)
+        torq.torq_rotate_quantize(b["X"], Rm[i % n_sets], None, out_codes=c, out_scales=sc)
+
+    tm = timer(merged_only)
+    out["merged_rotation"] = {
+        "what": "torq_rotate_quantize(X, bf16(R_inter blockdiag(R_intra)), NULL): one GEMM, no intra step; a different "
+                "quantized operator (its code mismatch against the two-level path is measured in the tests)",
+        "ms_per_launch": tm["s"] * 1e3, "sm_mhz_in_loop": tm["sm_mhz"], "two_level_ms_per_launch": t_rot["s"] * 1e3,
+        "saves_frac": 1.0 - tm["s"] / t_rot["s"]}
+    del Rm
+
+    # ---- NVFP4 (16-element blocks, E4M3 block scales): its own intra rotations and weights
+    Ri32 = torq.torq_expand_intra16(I.bf16_bits_to_tensor(I.intra_rotations16(cfg), "cuda"))
+    torch.cuda.synchronize()
+    Wq_nv, Ws_nv, w_ts = torq.torq_prepare_weights_nvfp4(layer.R0, Ri32, layer.W)
+    # activation tensor scale, fixed ahead of time as a calibrated one would be: no rotated element exceeds
+    # its token's 2-norm, so the largest norm over the top of the E4M3 range never saturates
+    x_ts = float(layer.X0.float().norm(dim=1).max().item()) / (6.0 * 448.0)
+    ws_nv = [torch.empty(torq.torq_nvfp4_workspace_bytes(M, d, N), dtype=torch.uint8, device="cuda") for _ in range(2)]
+
+    def nv_cs(k):
         return (ws_nv[k][: M * d // 2].view(M, d // 2),
                 ws_nv[k][(M * d // 2 + 255) // 256 * 256:][: torq.torq_nvfp4_scales_bytes(M, d)])
 
-    nv_i = [0]
+    def nv_rot(i):
+        b = sets[i % n_sets]
+        c, sc = nv_cs(i & 1)
+        torq.torq_rotate_quantize_nvfp4(b["X"], b["R"], Ri32, x_ts, out_codes=c, out_scales=sc)
 
-    def nv_rot(b):
-        nv_i[0] ^= 1
-        c, sc = nv_codes_scales(nv_i[0])
-        torq.torq_rotate_quantize_nvfp4(b["X"], b["R"], Ri32_nv, x_ts_nv, out_codes=c, out_scales=sc)
+    def nv_gemm(i):
+        c, sc = nv_cs(i & 1)
+        torq.torq_nvfp4_gemm(c, sc, x_ts, Wq_nv, Ws_nv, w_ts, Y=sets[i % n_sets]["Y"])
 
-    def nv_gemm(b):
-        nv_i[0] ^= 1
-        c, sc = nv_codes_scales(nv_i[0])
-        torq.torq_nvfp4_gemm(c, sc, x_ts_nv, Wq_nv, Ws_nv, w_ts_nv, Y=b["Y"])
+    def nv_layer(i):
+        b = sets[i % n_sets]
+        torq.torq_rotated_linear_nvfp4(b["X"], b["R"], Ri32, x_ts, Wq_nv, Ws_nv, w_ts, Y=b["Y"], workspace=ws_nv[i & 1])
 
-    def nv_layer(b):
-        nv_i[0] ^= 1
-        torq.torq_rotated_linear_nvfp4(b["X"], b["R"], Ri32_nv, x_ts_nv, Wq_nv, Ws_nv, w_ts_nv, Y=b["Y"],
-                                       workspace=ws_nv[nv_i[0]])
+    a, g, l = timer(nv_rot), timer(nv_gemm), timer(nv_layer)
+    out["nvfp4_variant"] = {
+        "what": "the same layer in NVFP4 (16-element blocks, E4M3 block scales, float32 tensor scales; "
+                "kind::mxf4nvf4 GEMM)",
+        "rotate_quant": simple(a), "rotate_quant_frac_of_bf16_burst": rot_flop / a["s"] / 1e12 / pk["bf16_burst"],
+        "gemm": simple(g), "gemm_TFLOPs": gemm_flop / g["s"] / 1e12, "gemm_frac_of_fp4_probe": gemm_flop / g["s"] / 1e12 / fp4_peak,
+        "whole_layer_ms_per_step": l["s"] * 1e3, "whole_layer_tokens_per_s": world * M / l["s"]}
+    del Wq_nv, Ws_nv, ws_nv
 
-    t_nv_rot, t_nv_gemm, t_nv_layer = timed_loop(nv_rot), timed_loop(nv_gemm), timed_loop(nv_layer)
+    # ---- MXINT4 (integer codes as E4M3 operand bytes, same rotations as the MXFP4 layer)
+    _, W8, Ws_i4 = torq.torq_prepare_weights_mxint4(layer.R0, layer.Ri0, layer.W)
+    ws_i4 = [torch.empty(torq.torq_mxint4_workspace_bytes(M, d, N), dtype=torch.uint8, device="cuda") for _ in range(2)]
 
-    # the MXINT4 variant, likewise
-    def i4_bytes_scales(k):
+    def i4_cs(k):
         return ws_i4[k][: M * d].view(M, d), ws_i4[k][(M * d + 255) // 256 * 256:][: torq.torq_scales_bytes(M, d)]
 
-    def i4_rot(b):
-        nv_i[0] ^= 1
-        c, sc = i4_bytes_scales(nv_i[0])
+    def i4_rot(i):
+        b = sets[i % n_sets]
+        c, sc = i4_cs(i & 1)
         torq.torq_rotate_quantize_mxint4(b["X"], b["R"], b["Ri"], out_bytes=c, out_scales=sc)
 
-    def i4_gemm(b):
-        nv_i[0] ^= 1
-        c, sc = i4_bytes_scales(nv_i[0])
-        torq.torq_mxint4_gemm(c, sc, W8_i4, Ws_i4, Y=b["Y"])
+    def i4_gemm(i):
+        c, sc = i4_cs(i & 1)
+        torq.torq_mxint4_gemm(c, sc, W8, Ws_i4, Y=sets[i % n_sets]["Y"])
 
-    def i4_layer(b):
-        nv_i[0] ^= 1
-        torq.torq_rotated_linear_mxint4(b["X"], b["R"], b["Ri"], W8_i4, Ws_i4, Y=b["Y"], workspace=ws_i4[nv_i[0]])
+    def i4_layer(i):
+        b = sets[i % n_sets]
+        torq.torq_rotated_linear_mxint4(b["X"], b["R"], b["Ri"], W8, Ws_i4, Y=b["Y"], workspace=ws_i4[i & 1])
 
-    t_i4_rot, t_i4_gemm, t_i4_layer = timed_loop(i4_rot), timed_loop(i4_gemm), timed_loop(i4_layer)
-    barrier()
-    clocks = sampler.stop()
-    assert torq.torq_last_device_error() == 0
+    a, g, l = timer(i4_rot), timer(i4_gemm), timer(i4_layer)
+    out["mxint4_variant"] = {
+        "what": "the same layer in MXINT4 (32-element blocks, E8M0 scales, integers in [-7,7] fed to the tensor "
+                "cores as E4M3 bytes; kind::mxf8f6f4 GEMM at the 8-bit rate)",
+        "rotate_quant": simple(a), "rotate_quant_frac_of_bf16_burst": rot_flop / a["s"] / 1e12 / pk["bf16_burst"],
+        "gemm": simple(g), "gemm_TFLOPs": gemm_flop / g["s"] / 1e12,
+        "gemm_frac_of_half_fp4_probe": gemm_flop / g["s"] / 1e12 / (fp4_peak / 2),
+        "whole_layer_ms_per_step": l["s"] * 1e3, "whole_layer_tokens_per_s": world * M / l["s"]}
+    return out
 
-    # ---- end to end through the public call with HOST buffers (pinned): every step copies its X
-    # host -> device, runs the layer, and copies its Y device -> host, all inside the timed region.
-    # Three streams with two device buffers each way: the upload of step i+1 and the download of
-    # step i-1 run beside the kernels of step i (PCIe is full duplex), ordered by events.
-    Xh = X0.cpu().pin_memory()
+
+def measure_e2e(torq, layer, stream, steps, barrier):
+    """End to end through the public call with HOST buffers (pinned): every step copies its X host ->
+    device, runs the layer, and copies its Y device -> host, all inside the timed region.  Three
+    streams with two device buffers each way: the upload of step i+1 and the download of step i-1 run
+    beside the kernels of step i (PCIe is full duplex), ordered by events."""
+    M, d, N = layer.M, layer.d, layer.N
+    Xh = layer.X0.cpu().pin_memory()
     Yh = [torch.empty((M, N), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
-    e2e_steps = max(3, min(args.steps, 50))
+    n = max(3, min(steps, 50))
     up, down = torch.cuda.Stream(), torch.cuda.Stream()
-    Xd = [sets[0]["X"], sets[1]["X"]]
-    Yd = [sets[0]["Y"], sets[1]["Y"]]
-    wsd = [sets[0]["ws"], sets[1]["ws"]]
-    p0 = sets[0]
+    p0 = layer.sets[0]
+    Xd = [p0["X"], layer.X0.clone()]
+    Yd = [p0["Y"], torch.empty_like(p0["Y"])]
+    wsd = [p0["ws"], torch.empty_like(p0["ws"])]
 
-    def e2e_loop(n):
+    def loop(n):
         x_ready = [torch.cuda.Event() for _ in range(n)]
         y_ready = [torch.cuda.Event() for _ in range(n)]
         x_free = [torch.cuda.Event() for _ in range(n)]
@@ -397,94 +536,152 @@ def main():
         stream.wait_stream(down)
         stream.wait_stream(up)
 
-    e2e_loop(4)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    loop(4)
     barrier()
     e0.record(stream)
-    e2e_loop(e2e_steps)
+    loop(n)
     e1.record(stream)
     barrier()
-    ms_e2e = e0.elapsed_time(e1) / e2e_steps
-    Yh = Yh[0]
+    return e0.elapsed_time(e1) / n, Xh.numel() * 2, Yh[0].numel() * 2
+
+SWEEP_M = (1, 64, 1024, 16384)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None, help="default: 2000 (the CUDA path), 20 (--impl reference)")
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default=WORKLOAD, help="one of inputs.CONFIGS (default: the LLaMA3-8B QKV shape)")
+    ap.add_argument("--M", type=int, default=None, help="override the number of tokens (token sweep)")
+    ap.add_argument("--only-main", action="store_true", help="skip the variants, the second 8B shape and the sweep")
+    args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 20 if args.impl == "reference" else 2000
+    if args.impl == "reference":
+        return run_reference(args)
+
+    from paper_2605_19561_b200 import inputs as I
+    from paper_2605_19561_b200 import torq
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    warmup = max(args.warmup, 3)
+    cfg = I.CONFIGS[args.workload]
+    M, d, N = (args.M or cfg.M), cfg.d, cfg.N
+    pk = peaks()
+    sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    stream = torch.cuda.current_stream()
+    loop_stream = torch.cuda.Stream()                      # graph capture needs a stream of its own
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- inputs (seeded, synthetic; every rank holds its own M rows: weak scaling over tokens)
+    layer = Layer(torq, I, args.workload, M)
+    timer = KernelTimer(loop_stream, sampler, layer.n_sets)
+    fp4_probe = max(torq.torq_probe_fp4_peak(40000) for _ in range(2))     # TFLOP/s, ~1 ms each
+
+    for i in range(warmup):
+        layer.step(i)
+    barrier()
+    assert torq.torq_last_device_error() == 0
+
+    # ---- timed region: exactly K steps of the whole path, inputs resident in HBM
+    time.sleep(0.2)
+    launches0 = torq.torq_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_host0 = time.time()
+    hold_gpu(stream)
+    e0.record(stream)
+    for i in range(args.steps):
+        layer.step(i)
+    e1.record(stream)
+    barrier()
+    t_host1 = time.time()
+    launches = torq.torq_launch_count() - launches0
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.summary(t_host0, t_host1)
+    if clocks.get("samples", 0) == 0:                      # a region shorter than the sampling period
+        clocks = sampler.summary(t_host0 - 0.05, t_host1 + 0.05)
+
+    # ---- per-kernel loops of the main workload, each >= MIN_LOOP_MS with its own clock sample
+    main_rec, t_step, t_rot, t_gemm = measure_layer(layer, timer, pk, fp4_probe, sm_count, world)
+    extras = {}
+    if not args.only_main:
+        extras = measure_variants(torq, I, layer, timer, pk, fp4_probe, t_rot, world)
+    barrier()
+    assert torq.torq_last_device_error() == 0
+    ms_e2e, h2d, d2h = measure_e2e(torq, layer, stream, args.steps, barrier)
+
+    # ---- the second 8B shape and the token sweep (rank 0 measures them; they are per-GPU numbers)
+    others = {}
+    if not args.only_main and rank == 0 and args.workload == WORKLOAD and args.M is None:
+        del layer.sets[1:]
+        torch.cuda.empty_cache()
+        down = Layer(torq, I, "llama3_8b_down", I.CONFIGS["llama3_8b_down"].M)
+        rec, _, _, _ = measure_layer(down, KernelTimer(loop_stream, sampler, down.n_sets), pk, fp4_probe, sm_count, 1)
+        others["llama3_8b_down"] = rec
+        del down
+        torch.cuda.empty_cache()
+        sweep = []
+        base = None
+        for m in SWEEP_M:
+            lay = Layer(torq, I, "qwen3_32b_sweep", m) if base is None else base.with_tokens(I, m)
+            base = base or lay
+            rec, _, _, _ = measure_layer(lay, KernelTimer(loop_stream, sampler, lay.n_sets), pk, fp4_probe, sm_count, 1)
+            sweep.append({"M": m, "us_per_step": rec["ms_per_step"] * 1e3, "tokens_per_s": rec["tokens_per_s"],
+                          "sm_mhz": rec["sm_mhz_in_step_loop"],
+                          "rotate_quantize": {k: rec["rotate_quantize"][k] for k in
+                                              ("kernel", "ms_per_launch", "bound", "achieved", "unit", "frac", "sm_mhz_in_loop")},
+                          "gemm": {k: rec["gemm"][k] for k in
+                                   ("kernel", "ms_per_launch", "bound", "achieved", "unit", "frac", "sm_mhz_in_loop")}})
+            if lay is not base:
+                del lay
+            torch.cuda.empty_cache()
+        others["sweep"] = {"workload": "qwen3_32b_sweep", "d": 5120, "N": 5120, "points": sweep}
+        assert torq.torq_last_device_error() == 0
+    sampler.stop()
 
     from paper_2605_19561_b200.sharding import max_over_ranks
-    ms_total, ms_e2e, t_rot, t_gemm = max_over_ranks([ms_total, ms_e2e, t_rot, t_gemm], device="cuda")
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], device="cuda")
     ms_step = ms_total / args.steps
 
     if rank == 0:
-        rot_flop = 2.0 * M * d * d + 64.0 * M * d
-        rot_bytes = 2.0 * M * d + 2.0 * d * d + 2.0 * 32 * d + M * d / 2 + M * d / 32
-        gemm_flop = 2.0 * M * N * d
-        gemm_bytes = M * d / 2 + M * d / 32 + N * d / 2 + N * d / 32 + 2.0 * M * N
-        # Peak for a kernel timed in a short burst at full clock: the burst figure; when the sampled
-        # SM clock sat clearly below its maximum (power cap in a long run): the sustained one.
-        at_full_clock = bool(clocks.get("sm_mhz") and clocks.get("sm_max_mhz")
-                             and clocks["sm_mhz"] >= 0.95 * clocks["sm_max_mhz"])
-        bf16_peak = pk["bf16_burst"] if at_full_clock else pk["bf16_sustained"]
-        peak_name = f"{pk['source']} bf16 {'burst' if at_full_clock else 'sustained'}"
-        # MEASURED_PEAKS.json has no FP4 entry: the denominator is this device's own issue-bound rate of
-        # the GEMM's instruction (operands resident in shared memory, no loads), measured just before
-        fp4_peak = fp4_probe
-
-        def roof(kernel, t, flop, nbytes, tensor_peak, tensor_name):
-            """Roofline record of one kernel: the binding bound is the slower of its HBM and tensor floors."""
-            t_hbm, t_tc = nbytes / (pk["hbm_gbs"] * 1e9), flop / (tensor_peak * 1e12)
-            if t_tc >= t_hbm:
-                ach, peak, unit, bound, src = flop / t / 1e12, tensor_peak, "TFLOP/s", "tensor", tensor_name
-            else:
-                ach, peak, unit, bound, src = nbytes / t / 1e9, pk["hbm_gbs"], "GB/s", "hbm", f"{pk['source']} HBM copy"
-            return {"kernel": kernel, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
-                    "traffic": profiled_traffic(kernel, args.workload), "peak_source": src,
-                    "ms_per_launch": t * 1e3, "algorithmic_flop": flop, "algorithmic_bytes": nbytes}
-
-        pairs = M > 128
-        r_rot = roof("rotate_splitk_kernel + splitk_reduce_quantize_kernel" if split_k else
-                     ("rotate_quantize_pair_kernel" if pairs else "rotate_quantize_kernel"), t_rot, rot_flop, rot_bytes,
-                     bf16_peak, peak_name)
-        r_gemm = roof("mxfp4_gemm_pair_kernel" if pairs else "mxfp4_gemm_kernel", t_gemm, gemm_flop, gemm_bytes,
-                      fp4_peak, "self-measured: torq_probe_fp4_peak (FP4 block-scaled MMA issue loop, no loads)")
-        r_gemm["frac_of_nominal_9000_tflops"] = gemm_flop / t_gemm / 1e12 / 9000.0
-        r_gemm["frac_of_4x_measured_bf16"] = gemm_flop / t_gemm / 1e12 / (4.0 * bf16_peak)
-        r_rot["frac_of_nominal_2250_tflops"] = rot_flop / t_rot / 1e12 / 2250.0
-        dominant, other = (r_rot, r_gemm) if t_rot >= t_gemm else (r_gemm, r_rot)
+        r_rot, r_gemm = main_rec["rotate_quantize"], main_rec["gemm"]
+        dominant, other = (r_rot, r_gemm) if r_rot["ms_per_launch"] >= r_gemm["ms_per_launch"] else (r_gemm, r_rot)
         out = {
             "metric": METRIC, "value": world * M / (ms_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16+mxfp4", "data": "synthetic",
             "config": {"workload": args.workload, "M_per_gpu": M, "d": d, "N": N, "out_dtype": "bf16",
-                       "l2": f"{n_sets} operand sets rotated between steps (working set > 126 MB L2)",
-                       "sharding": "rows (tokens) per GPU, no collective"},
-            "rotate_quant_GBps": rot_bytes / t_rot / 1e9, "rotate_quant_TFLOPs": rot_flop / t_rot / 1e12,
-            "gemm_TFLOPs": gemm_flop / t_gemm / 1e12,
+                       "l2": layer.l2_note, "sharding": "rows (tokens) per GPU, no collective"},
+            "rotate_quant_GBps": r_rot["GBps"], "rotate_quant_TFLOPs": r_rot["algorithmic_flop"] / r_rot["ms_per_launch"] / 1e9,
+            "gemm_TFLOPs": r_gemm["TFLOPs"],
             "roofline": dominant, "roofline_other_kernel": other,
-            "structured_rotation": None if t_struct is None else (lambda nbytes: {
-                "kernel": "rotate_structured_kernel", "what": "rotate+quantize with R_inter = R_B (x) I_32 and one shared "
-                "R_intra (the paper's structure, 2d(B+32) flop per token) on the same activations", "bound": "hbm",
-                "ms_per_launch": t_struct * 1e3, "achieved": nbytes / t_struct / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                "frac": nbytes / t_struct / 1e9 / pk["hbm_gbs"], "algorithmic_bytes": nbytes,
-                "traffic": profiled_traffic("rotate_structured_kernel", args.workload),
-                "speedup_over_dense_rotation": t_rot / t_struct,
-                "whole_layer_ms_per_step": t_struct_layer * 1e3, "whole_layer_tokens_per_s": world * M / t_struct_layer})(
-                    2.0 * M * d + 2.0 * (d // 32) ** 2 + 2048.0 + M * d / 2 + M * d / 32),
-            "nvfp4_variant": {
-                "what": "the same layer in NVFP4 (16-element blocks, E4M3 block scales, float32 tensor scales; "
-                        "kind::mxf4nvf4 GEMM), single-pass rotation kernels",
-                "rotate_quant_ms": t_nv_rot * 1e3, "rotate_quant_TFLOPs": rot_flop / t_nv_rot / 1e12,
-                "rotate_quant_frac": rot_flop / t_nv_rot / 1e12 / bf16_peak,
-                "gemm_ms": t_nv_gemm * 1e3, "gemm_TFLOPs": gemm_flop / t_nv_gemm / 1e12,
-                "gemm_frac": gemm_flop / t_nv_gemm / 1e12 / fp4_peak,
-                "whole_layer_ms_per_step": t_nv_layer * 1e3, "whole_layer_tokens_per_s": world * M / t_nv_layer},
-            "mxint4_variant": {
-                "what": "the same layer in MXINT4 (32-element blocks, E8M0 scales, integers in [-7,7] fed to the tensor "
-                        "cores as E4M3 bytes; kind::mxf8f6f4 GEMM at the 8-bit rate), single-pass rotation kernels",
-                "rotate_quant_ms": t_i4_rot * 1e3, "rotate_quant_TFLOPs": rot_flop / t_i4_rot / 1e12,
-                "rotate_quant_frac": rot_flop / t_i4_rot / 1e12 / bf16_peak,
-                "gemm_ms": t_i4_gemm * 1e3, "gemm_TFLOPs": gemm_flop / t_i4_gemm / 1e12,
-                "gemm_frac_of_half_fp4_peak": gemm_flop / t_i4_gemm / 1e12 / (fp4_peak / 2),
-                "whole_layer_ms_per_step": t_i4_layer * 1e3, "whole_layer_tokens_per_s": world * M / t_i4_layer},
-            "e2e": {"value": world * M / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": Xh.numel() * 2,
-                    "d2h_bytes_per_step": Yh.numel() * 2},
+            "step_loop": {"ms_per_step": main_rec["ms_per_step"], "sm_mhz": main_rec["sm_mhz_in_step_loop"],
+                          "what": f"the same step timed over at least {MIN_LOOP_MS:.0f} ms ({main_rec['step_timing']})"},
+            "fp4_probe_tflops": fp4_probe,
+            "e2e": {"value": world * M / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches), "clocks": clocks,
         }
+        out.update(extras)
+        out.update(others)
         if not args.no_cpu_baseline:
             rows = min(512, M)
             t, cores = time_oracle(cfg, rows, 2, 1)
