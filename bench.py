@@ -194,7 +194,10 @@ class KernelTimer:
     def __init__(self, stream, sampler, n_sets):
         self.stream, self.sampler, self.n_sets = stream, sampler, n_sets
 
-    def __call__(self, fn, batch=None, min_ms=MIN_LOOP_MS):
+    min_ms = MIN_LOOP_MS
+
+    def __call__(self, fn, batch=None, min_ms=None):
+        min_ms = self.min_ms if min_ms is None else min_ms
         batch = batch or max(self.n_sets, 8) // self.n_sets * self.n_sets
         s = self.stream
         torch.cuda.synchronize()
@@ -346,7 +349,7 @@ class Layer:
         self.torq.torq_mxfp4_gemm(c, sc, b["Wq"], b["Ws"], Y=b["Y"])
 
 
-def measure_layer(layer, timer, pk, fp4_peak, sm_count, world):
+def measure_layer(layer, timer, pk, fp4_peak, sm_count, world, fp4_sustained=None):
     """Step, rotate+quantize and GEMM of one workload, each in its own loop with its own clock sample."""
     M, d, N = layer.M, layer.d, layer.N
     rot_flop, rot_bytes, gemm_flop, gemm_bytes = layer_work(M, d, N)
@@ -365,7 +368,7 @@ def measure_layer(layer, timer, pk, fp4_peak, sm_count, world):
                         f"{pk['source']} bf16 burst", layer.name)
     r_rot["frac_of_nominal_2250_tflops"] = rot_flop / t_rot["s"] / 1e12 / 2250.0
     r_rot["GBps"] = rot_bytes / t_rot["s"] / 1e9
-    r_gemm = roof_record(gemm_kernel_name(M), t_gemm, gemm_flop, gemm_bytes, pk, fp4_peak, None,
+    r_gemm = roof_record(gemm_kernel_name(M), t_gemm, gemm_flop, gemm_bytes, pk, fp4_peak, fp4_sustained,
                          "self-measured: torq_probe_fp4_peak (FP4 block-scaled MMA issue loop, no loads)", layer.name)
     r_gemm["frac_of_nominal_9000_tflops"] = gemm_flop / t_gemm["s"] / 1e12 / 9000.0
     r_gemm["frac_of_4x_measured_bf16_burst"] = gemm_flop / t_gemm["s"] / 1e12 / (4.0 * pk["bf16_burst"])
@@ -558,6 +561,8 @@ def main():
     ap.add_argument("--workload", default=WORKLOAD, help="one of inputs.CONFIGS (default: the LLaMA3-8B QKV shape)")
     ap.add_argument("--M", type=int, default=None, help="override the number of tokens (token sweep)")
     ap.add_argument("--only-main", action="store_true", help="skip the variants, the second 8B shape and the sweep")
+    ap.add_argument("--min-loop-ms", type=float, default=MIN_LOOP_MS,
+                    help="length of every per-kernel timing loop (shorter only for runs under a profiler)")
     args = ap.parse_args()
     if args.steps is None:
         args.steps = 20 if args.impl == "reference" else 2000
@@ -592,8 +597,12 @@ def main():
 
     # ---- inputs (seeded, synthetic; every rank holds its own M rows: weak scaling over tokens)
     layer = Layer(torq, I, args.workload, M)
+    KernelTimer.min_ms = args.min_loop_ms
     timer = KernelTimer(loop_stream, sampler, layer.n_sets)
-    fp4_probe = max(torq.torq_probe_fp4_peak(40000) for _ in range(2))     # TFLOP/s, ~1 ms each
+    fp4_probe = max(torq.torq_probe_fp4_peak(40000) for _ in range(2))     # TFLOP/s, ~12 ms each: burst
+    t0 = time.time()
+    fp4_sustained = torq.torq_probe_fp4_peak(400000)                       # ~125 ms under the power cap
+    fp4_sustained_clk = sampler.window(t0, time.time())
 
     for i in range(warmup):
         layer.step(i)
@@ -620,7 +629,7 @@ def main():
         clocks = sampler.summary(t_host0 - 0.05, t_host1 + 0.05)
 
     # ---- per-kernel loops of the main workload, each >= MIN_LOOP_MS with its own clock sample
-    main_rec, t_step, t_rot, t_gemm = measure_layer(layer, timer, pk, fp4_probe, sm_count, world)
+    main_rec, t_step, t_rot, t_gemm = measure_layer(layer, timer, pk, fp4_probe, sm_count, world, fp4_sustained)
     extras = {}
     if not args.only_main:
         extras = measure_variants(torq, I, layer, timer, pk, fp4_probe, t_rot, world)
@@ -634,7 +643,7 @@ def main():
         del layer.sets[1:]
         torch.cuda.empty_cache()
         down = Layer(torq, I, "llama3_8b_down", I.CONFIGS["llama3_8b_down"].M)
-        rec, _, _, _ = measure_layer(down, KernelTimer(loop_stream, sampler, down.n_sets), pk, fp4_probe, sm_count, 1)
+        rec, _, _, _ = measure_layer(down, KernelTimer(loop_stream, sampler, down.n_sets), pk, fp4_probe, sm_count, 1, fp4_sustained)
         others["llama3_8b_down"] = rec
         del down
         torch.cuda.empty_cache()
@@ -643,7 +652,7 @@ def main():
         for m in SWEEP_M:
             lay = Layer(torq, I, "qwen3_32b_sweep", m) if base is None else base.with_tokens(I, m)
             base = base or lay
-            rec, _, _, _ = measure_layer(lay, KernelTimer(loop_stream, sampler, lay.n_sets), pk, fp4_probe, sm_count, 1)
+            rec, _, _, _ = measure_layer(lay, KernelTimer(loop_stream, sampler, lay.n_sets), pk, fp4_probe, sm_count, 1, fp4_sustained)
             sweep.append({"M": m, "us_per_step": rec["ms_per_step"] * 1e3, "tokens_per_s": rec["tokens_per_s"],
                           "sm_mhz": rec["sm_mhz_in_step_loop"],
                           "rotate_quantize": {k: rec["rotate_quantize"][k] for k in
@@ -676,6 +685,8 @@ def main():
             "step_loop": {"ms_per_step": main_rec["ms_per_step"], "sm_mhz": main_rec["sm_mhz_in_step_loop"],
                           "what": f"the same step timed over at least {MIN_LOOP_MS:.0f} ms ({main_rec['step_timing']})"},
             "fp4_probe_tflops": fp4_probe,
+            "fp4_probe_sustained": {"tflops": fp4_sustained, "sm_mhz": fp4_sustained_clk["sm_mhz"],
+                                    "what": "the same issue loop run for about 100 ms (power-capped clock)"},
             "e2e": {"value": world * M / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches), "clocks": clocks,
