@@ -113,9 +113,6 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
  * fp32 partial tiles: the rotation is then split along its contraction so that every SM streams a
  * share of R_inter, and a second kernel adds the partials in a fixed order before the intra-block
  * step and Eq. 1.
- * For many tokens (three or more waves of rotation tiles, N <= 2 d) both steps run as ONE persistent
- * kernel launched cooperatively, whose GEMM tiles start as soon as the row tile they read is quantized;
- * the workspace then also holds a block of counters that the call zeroes itself.
  * Requires d % 128 == 0 and N % 8 == 0. */
 torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* R_intra,
                                 const void* Wq, const void* Ws, int64_t M, int64_t d, int64_t N,

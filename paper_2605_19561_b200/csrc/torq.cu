@@ -17,7 +17,6 @@
 #include "rotate_fewtok.cuh"
 #include "gemm_fewtok.cuh"
 #include "rotate_structured.cuh"
-#include "rotated_linear_fused.cuh"
 #include "fp4_peak_probe.cuh"
 #include "calibrate.cuh"
 #include "wait_selftest.cuh"
@@ -35,8 +34,6 @@ struct DeviceState {
   int sm_count = 0;
   int rot_pairs = 0;    // CTA pairs of the pair kernels that can be resident at once
   int gemm_pairs = 0;
-  std::atomic<int> fused_pairs{0};  // CTA pairs of the one-kernel layer that can be resident at once; 0 = not usable
-                                    // (host threads may clear it while others read it)
   int* err_word = nullptr;
 };
 static DeviceState g_dev[kMaxDevices];
@@ -134,9 +131,6 @@ static DeviceState* device_state() {
     st.gemm_pairs = max_active_pairs(mxfp4_gemm_pair_kernel<FMT_NVFP4>, GemmPairCfg::THREADS,
                                      GemmPairCfgT<FMT_NVFP4>::SMEM_BYTES, st.sm_count);
     if (st.rot_pairs < 1 || st.gemm_pairs < 1) return nullptr;
-    if (opt_in_smem(rotated_linear_pair_kernel, FusedCfg::SMEM_BYTES))
-      st.fused_pairs = max_active_pairs(rotated_linear_pair_kernel, FusedCfg::THREADS, FusedCfg::SMEM_BYTES,
-                                        st.sm_count);
     cudaGetLastError();
   }
   st.ready = true;
@@ -232,9 +226,6 @@ static inline int fewtok_cluster(int64_t tiles, int64_t k_steps, int min_k, int 
 static size_t quantized_bytes(int64_t M, int64_t d) {    // codes, then 256-byte aligned the scales
   return ((size_t)M * (size_t)(d / 2) + 255) / 256 * 256 + torq_scales_bytes(M, d);
 }
-// Row-tile counters of the one-kernel layer: behind the quantized activations in the workspace.
-constexpr size_t kCounterBytes = 1024;
-constexpr int64_t kFusedMaxRowTiles = (int64_t)(kCounterBytes / sizeof(int));
 static size_t splitk_scratch_bytes(int64_t M, int64_t d, int splits) {
   return splits < 2 ? 0 : (size_t)splits * (size_t)((M + 127) / 128 * 128) * (size_t)d * sizeof(float);
 }
@@ -272,7 +263,7 @@ size_t torq_scale_offset(int64_t row, int64_t kblock, int64_t k) {
 size_t torq_workspace_bytes(int64_t M, int64_t d, int64_t N) {
   (void)N;
   if (M <= 0 || d <= 0) return 0;
-  return quantized_bytes(M, d) + kCounterBytes + splitk_scratch_bytes(M, d, rotation_splits(M, d, 0));
+  return quantized_bytes(M, d) + splitk_scratch_bytes(M, d, rotation_splits(M, d, 0));
 }
 
 const char* torq_status_string(torq_status s) {
@@ -782,105 +773,21 @@ torq_status torq_rotated_linear_mxint4(const void* X, const void* R_inter, const
   return TORQ_OK;
 }
 
-// The whole layer as one persistent kernel (see rotated_linear_fused.cuh) where that pays and is
-// possible: CTA-pair regime, MXFP4, an R_inter that stays in L2 while the rotation walks row tile by
-// row tile, few enough row tiles for the counter block.  *done = false means "not taken, run the two
-// kernels"; the launch is cooperative (its CTAs wait on one another), and a device that refuses that
-// combination is remembered.
-static torq_status fused_layer(const void* X, const void* R_inter, const void* R_intra, const void* Wq,
-                               const void* Ws, int64_t M, int64_t d, int64_t N, void* Y, torq_dtype y_dtype,
-                               uint8_t* codes, uint8_t* scales, int* counters, void* stream, bool* done) {
-  *done = false;
-  DeviceState* st = device_state();
-  const int fused_pairs = st ? st->fused_pairs.load(std::memory_order_relaxed) : 0;
-  if (!st || !st->arch_ok || fused_pairs < 1) return TORQ_OK;
-  const int64_t mp_tiles = (M + 255) / 256;
-  if (M <= 128 || !R_inter || mp_tiles > kFusedMaxRowTiles || (size_t)d * (size_t)d * 2 > (size_t)(64u << 20) ||
-      rotation_splits(M, d, st->sm_count) >= 2 || M > (1 << 30) || N > (1 << 30) || d > (1 << 24))
-    return TORQ_OK;
-  if (y_dtype != TORQ_F32 && y_dtype != TORQ_BF16) return TORQ_OK;
-  if (!aligned16(X) || !aligned16(R_inter) || (R_intra && !aligned16(R_intra)) || !aligned16(Wq) || !aligned16(Ws) ||
-      !aligned16(Y))
-    return TORQ_OK;                                      // let the two-kernel path report it
-  const int64_t rot_tiles = mp_tiles * ((d + 255) / 256), gemm_tiles = mp_tiles * ((N + 255) / 256);
-  // Worth it only from three rotation waves on.  The epilogue of a rotation tile that is not its
-  // pair's last runs beside the next mainloop and takes most of it, so a row tile is complete about
-  // one tile time after its last mainloop: with two waves (2048 x 4096: measured 77 us against 72.5 us
-  // for the two kernels) the pairs that skip the second wave would still find no finished row.
-  if (rot_tiles < 3 * (int64_t)fused_pairs) return TORQ_OK;
-  // ... and while the GEMM is not the bulk of the work: its tiles are dealt out row tile by row tile
-  // here, which re-streams W for every row tile (8192 x 5120 -> 25600: 759 us against 689 us).
-  if (N > 2 * d) return TORQ_OK;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  CUtensorMap tmX, tmR, tmA, tmB, tmSFA, tmSFB, tmY;
-  const uint64_t kb4 = (uint64_t)(d / 128);
-  const bool ybf = y_dtype == TORQ_BF16;
-  if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d, 128, 64) ||
-      !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64) ||
-      !encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, (uint64_t)M, (uint64_t)(d / 2), 128, 128) ||
-      !encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, (uint64_t)(d / 2), 128, 128) ||
-      !encode_2d(&tmSFA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, scales, (uint64_t)((M + 127) / 128), kb4 * 128, 1, 256,
-                 CU_TENSOR_MAP_SWIZZLE_NONE) ||
-      !encode_2d(&tmSFB, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, Ws, (uint64_t)((N + 127) / 128), kb4 * 128, 1, 256,
-                 CU_TENSOR_MAP_SWIZZLE_NONE) ||
-      !encode_2d(&tmY, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, ybf ? 2 : 4, Y,
-                 (uint64_t)M, (uint64_t)N, 32, ybf ? 64 : 32))
-    return TORQ_OK;
-  if (cudaMemsetAsync(counters, 0, (size_t)mp_tiles * sizeof(int), s) != cudaSuccess) return TORQ_OK;
-  const int64_t most = rot_tiles > gemm_tiles ? rot_tiles : gemm_tiles;
-  const int pairs = (int)(most < fused_pairs ? most : (int64_t)fused_pairs);
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
-  cfg.blockDim = dim3((unsigned)FusedCfg::THREADS, 1, 1);
-  cfg.dynamicSmemBytes = (size_t)FusedCfg::SMEM_BYTES;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  attr[1].id = cudaLaunchAttributeCooperative;
-  attr[1].val.cooperative = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 2;
-  const int early = 4;     // GEMM tiles a pair gets through while the others finish a rotation tile (rate ratio ~4.5)
-  cudaError_t e = cudaLaunchKernelEx(&cfg, rotated_linear_pair_kernel, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra),
-                                     codes, scales, tmA, tmB, tmSFA, tmSFB, tmY, ybf ? 1 : 0, (int)M, (int)d, (int)N,
-                                     counters, early, st->err_word);
-  if (e != cudaSuccess) {                                // e.g. cooperative launch of clusters refused: never again
-    cudaGetLastError();
-    st->fused_pairs = 0;
-    return TORQ_OK;
-  }
-  *done = true;
-  return launch_status();
-}
-
 // Steps 1-5 with `workspace_bytes` >= quantized_bytes(M, d) already checked by the caller: codes,
 // scales, then whatever is left as split-K scratch.
 static torq_status rotated_linear_impl(const void* X, const void* R_inter, const void* R_intra, const void* Wq,
                                        const void* Ws, int64_t M, int64_t d, int64_t N, void* Y,
                                        torq_dtype y_dtype, void* workspace, size_t workspace_bytes,
-                                       void* dbg_codes, void* dbg_scales, void* stream, bool allow_fused) {
+                                       void* dbg_codes, void* dbg_scales, void* stream) {
   uint8_t* codes = static_cast<uint8_t*>(workspace);
   const size_t codes_bytes = (size_t)M * (size_t)(d / 2);
   uint8_t* scales = codes + (codes_bytes + 255) / 256 * 256;
   const size_t used = quantized_bytes(M, d);
-  torq_status rc = TORQ_ERR_LAUNCH;
-  bool done = false;
-  if (allow_fused && workspace_bytes >= used + kCounterBytes) {
-    rc = fused_layer(X, R_inter, R_intra, Wq, Ws, M, d, N, Y, y_dtype, codes, scales,
-                     reinterpret_cast<int*>(codes + used), stream, &done);
-    if (done && rc != TORQ_OK) return rc;
-  }
-  if (!done) {
-    const size_t head = allow_fused ? used + kCounterBytes : used;
-    rc = rotate_quantize_impl(X, R_inter, R_intra, M, d, codes, scales, codes + head,
-                              workspace_bytes > head ? workspace_bytes - head : 0, stream);
-    if (rc != TORQ_OK) return rc;
-    rc = torq_mxfp4_gemm(codes, scales, Wq, Ws, M, N, d, Y, y_dtype, stream);
-    if (rc != TORQ_OK) return rc;
-  }
+  torq_status rc = rotate_quantize_impl(X, R_inter, R_intra, M, d, codes, scales, codes + used,
+                                        workspace_bytes > used ? workspace_bytes - used : 0, stream);
+  if (rc != TORQ_OK) return rc;
+  rc = torq_mxfp4_gemm(codes, scales, Wq, Ws, M, N, d, Y, y_dtype, stream);
+  if (rc != TORQ_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dbg_codes &&
       cudaMemcpyAsync(dbg_codes, codes, codes_bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
@@ -900,7 +807,7 @@ torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* 
   if (!workspace || workspace_bytes < torq_workspace_bytes(M, d, N)) return TORQ_ERR_WORKSPACE;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return TORQ_ERR_ALIGN;
   return rotated_linear_impl(X, R_inter, R_intra, Wq, Ws, M, d, N, Y, y_dtype, workspace, workspace_bytes,
-                             dbg_codes, dbg_scales, stream, /*allow_fused=*/true);
+                             dbg_codes, dbg_scales, stream);
 }
 
 torq_status torq_rotated_linear_structured(const void* X, const void* R_B, const void* R_intra, const void* Wq,
@@ -965,7 +872,7 @@ torq_status torq_rotated_linear_static(const void* X, const void* R_inter, const
   void* scratch = static_workspace_address();
   if (!scratch) return TORQ_ERR_LAUNCH;
   return rotated_linear_impl(X, R_inter, R_intra, Wq, Ws, M, d, N, Y, y_dtype, scratch,
-                             (size_t)TORQ_STATIC_WORKSPACE_BYTES, nullptr, nullptr, stream, /*allow_fused=*/false);
+                             (size_t)TORQ_STATIC_WORKSPACE_BYTES, nullptr, nullptr, stream);
 }
 
 torq_status torq_probe_fp4_peak(int groups, double* tflops, void* stream) {
