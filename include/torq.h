@@ -374,6 +374,19 @@ const char* torq_status_string(torq_status s);
  * 0, or TORQ_ERR_TIMEOUT in the low byte with the id of the wait that gave up in bits 8..15. */
 int torq_last_device_error(void* stream);
 
+/* Host helper (no device work): the list of output tiles that the CTA-pair kernels (more than 128
+ * rows) walk for a [rows x cols] output on `pairs` CTA pairs (74 on a 148-SM part), in the order
+ * in which they are dealt round robin: tile i goes to pair i % pairs.  Tiles are 256 rows high and
+ * 256 columns wide; where that leaves the last wave partly empty and cols is a multiple of 256,
+ * some row tiles are covered by fewer 256-column tiles followed by 192-column ones (three wide
+ * tiles traded for four narrow ones), chosen so that the longest pair finishes earliest.  Both
+ * torq_rotate_quantize (cols = d) and torq_mxfp4_gemm (cols = N), and their format variants, use
+ * this list.
+ *   out: host array of 3 * cap int32, or NULL; receives (row_tile, first_column, width) per tile.
+ * Returns the number of tiles (also when it exceeds cap; only cap triples are written), or -1 for
+ * rows < 1, cols < 1 or pairs < 1. */
+int64_t torq_pair_tile_list(int64_t rows, int64_t cols, int32_t pairs, int32_t* out, int64_t cap);
+
 /* Number of kernels this library has launched since load (all devices, all streams). */
 int64_t torq_launch_count(void);
 

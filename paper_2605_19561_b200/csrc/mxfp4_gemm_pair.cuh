@@ -12,6 +12,11 @@
 // 16 bytes of its own row per instruction made 32 partial-sector writes per warp store and ran at
 // a third of the speed).
 //
+// Tiles are dealt round robin from the list MixedTiles describes: 256 x 256 tiles, and where those
+// would leave the last wave partly empty, 256 x 192 tiles in its place (N = 192 instructions, 96
+// rows of W per CTA; the tile's W scales are still two whole 128-row chunks, read from two columns
+// further on when the tile starts 64 rows into its first chunk).
+//
 // Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (leader CTA only), warps 2..9 epilogue
 // (warp w reads lane quarter w%4, column half (w-2)/4).  Barriers as in the pair rotation kernel;
 // acc_empty takes one arrival per epilogue warp of both CTAs (16).
@@ -59,8 +64,8 @@ template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(320, 1)
 mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                        const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB,
-                       const __grid_constant__ CUtensorMap tmY, int y_is_bf16, int M, int N, int K,
-                       float alpha, int* err_word) {
+                       const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmBn,
+                       const MixedTiles tiles, int y_is_bf16, int M, int N, int K, float alpha, int* err_word) {
   using C = GemmPairCfgT<FMT>;
   constexpr int CH = C::CH;
   constexpr int BN = C::BN;
@@ -80,9 +85,7 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
-  const int mp_tiles = (M + 255) / 256;
-  const int n_tiles = (N + BN - 1) / BN;
-  const int total_tiles = mp_tiles * n_tiles;
+  const int total_tiles = tiles.total;
   const int k_tiles = (K + C::BK - 1) / C::BK;
   const int kb4 = K / (C::BK / CH);                    // scale chunks per row
 
@@ -109,20 +112,22 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     if (elect_one()) {
       tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmB);
       tma_prefetch_desc(&tmSFA); tma_prefetch_desc(&tmSFB);
-      int mp0, nt;
-      pair_tile_coords(pair, mp_tiles, n_tiles, mp0, nt);
+      int mp0 = 0, col0 = 0;
+      bool narrow = false;
+      if (pre > 0) { mixed_tile_coords(pair, tiles, mp0, col0, narrow); tma_prefetch_desc(&tmBn); }
       (void)mp0;
+      const int bn_half = narrow ? kNarrowCols / 2 : BN / 2;
       for (int kt = 0; kt < pre; ++kt) {
         const uint32_t st = smem_base + kt * C::STAGE_BYTES;
         const uint32_t leader_full = map_to_cta(full_bar(kt), 0);
-        if (rank == 0) mbar_arrive_expect_tx(full_bar(kt), 2 * C::STAGE_TX);
-        tma_load_2d_pair(st + C::A_BYTES, &tmB, kt * 128, nt * BN + (int)rank * (BN / 2), leader_full);
+        if (rank == 0) mbar_arrive_expect_tx(full_bar(kt), 2 * (C::STAGE_TX - (BN / 2 - bn_half) * 128));
+        tma_load_2d_pair(st + C::A_BYTES, narrow ? &tmBn : &tmB, kt * 128, col0 + (int)rank * bn_half, leader_full);
 #pragma unroll
         for (int t = 0; t < 2; ++t)                      // one 1 KiB box = two chunks
 #pragma unroll
           for (int b = 0; b < C::SF_BOXES; ++b)
             tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * C::SFA_BYTES + b * 1024, &tmSFB,
-                             kt * CH * 128 + b * 256, 2 * nt + t, leader_full);
+                             kt * CH * 128 + b * 256, (col0 >> 7) + t, leader_full);
       }
     }
     __syncwarp();
@@ -134,9 +139,14 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     uint32_t it = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
-      int mp, nt;
-      pair_tile_coords(tile, mp_tiles, n_tiles, mp, nt);
+      int mp, tcol;
+      bool narrow;
+      mixed_tile_coords(tile, tiles, mp, tcol, narrow);
       const int mt = 2 * mp + (int)rank;
+      // a 192-column tile takes 96 rows of W per CTA; its scale rows start at a multiple of 64, so the two
+      // 128-row scale chunks from (tcol / 128) on still cover it
+      const int bn_half = narrow ? kNarrowCols / 2 : BN / 2;
+      const uint32_t stage_tx = 2 * (C::STAGE_TX - (BN / 2 - bn_half) * 128);
       for (int kt = 0; kt < k_tiles; ++kt, ++it) {
         const int s = it % C::STAGES;
         if (!mbar_wait_cluster_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
@@ -145,10 +155,10 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         const uint32_t leader_full = map_to_cta(full_bar(s), 0);
         if (elect_one()) {
           const bool w_issued = it < (uint32_t)pre;      // W side of this stage went out before the wait above
-          if (rank == 0 && !w_issued) mbar_arrive_expect_tx(full_bar(s), 2 * C::STAGE_TX);
+          if (rank == 0 && !w_issued) mbar_arrive_expect_tx(full_bar(s), stage_tx);
           tma_load_2d_pair(st, &tmA, kt * 128, mt * C::BM, leader_full);
           if (!w_issued)
-            tma_load_2d_pair(st + C::A_BYTES, &tmB, kt * 128, nt * BN + (int)rank * (BN / 2), leader_full);
+            tma_load_2d_pair(st + C::A_BYTES, narrow ? &tmBn : &tmB, kt * 128, tcol + (int)rank * bn_half, leader_full);
           // scale tiles: one row of the [row tile, chunk x 512 B] view per 128 rows, in boxes of
           // 1 KiB (two chunks); anything outside the buffer arrives as zeros (scale 2^-127 or 0,
           // multiplying operand data that is zero there as well).
@@ -162,7 +172,7 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 #pragma unroll
               for (int b = 0; b < C::SF_BOXES; ++b)
                 tma_load_2d_pair(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + t * C::SFA_BYTES + b * 1024, &tmSFB,
-                                 kt * CH * 128 + b * 256, 2 * nt + t, leader_full);
+                                 kt * CH * 128 + b * 256, (tcol >> 7) + t, leader_full);
           }
         }
         __syncwarp();
@@ -173,10 +183,20 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     if (rank == 0) {
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      constexpr uint32_t idesc0 = FMT == FMT_NVFP4 ? idesc_nvf4(256, BN) : idesc_mxf4(256, BN, 0, 0);
-      constexpr uint32_t idesc2 = FMT == FMT_NVFP4 ? idesc_nvf4(256, BN) : idesc_mxf4(256, BN, 2, 2);
+      // instruction descriptors differ between the two tile widths only in the N field ([17,23) = N >> 3)
+      constexpr uint32_t n_less = (uint32_t)((BN - kNarrowCols) >> 3) << 17;
       const uint32_t sfa_t = tmem_base + C::SFA_COL, sfb_t = tmem_base + C::SFB_COL;
       for (int tile = pair; tile < total_tiles && ok; tile += npairs, ++tcount) {
+        int mp, tcol;
+        bool narrow;
+        mixed_tile_coords(tile, tiles, mp, tcol, narrow);
+        (void)mp;
+        const uint32_t nsub = narrow ? n_less : 0u;
+        const uint32_t idesc0 = (FMT == FMT_NVFP4 ? idesc_nvf4(256, BN) : idesc_mxf4(256, BN, 0, 0)) - nsub;
+        const uint32_t idesc2 = (FMT == FMT_NVFP4 ? idesc_nvf4(256, BN) : idesc_mxf4(256, BN, 2, 2)) - nsub;
+        // The W scales of rows 32 j .. 32 j + 31 of a 128-row chunk sit in column j of the chunk's four
+        // columns: a tile that starts 64 rows into its first chunk reads them from two columns further on.
+        const uint32_t sfb_m = sfb_t + ((tcol & 127) ? 2u : 0u);
         if (!mbar_wait_cluster_warp(acce_bar, (tcount & 1) ^ 1, cta_abort, err_word, SITE_MMA_ACC_EMPTY)) {
           ok = false; break;
         }
@@ -205,22 +225,22 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
               }
             }
             if constexpr (FMT == FMT_MXINT4) {             // a quarter chunk (one scale byte) per instruction
-              mma_mxf8_pair(tmem_base, adesc, bdesc, idesc_mxf8(256, BN, 0), sfa_t, sfb_t, kt != 0);
-              mma_mxf8_pair(tmem_base, adesc + 2, bdesc + 2, idesc_mxf8(256, BN, 1), sfa_t, sfb_t, 1);
-              mma_mxf8_pair(tmem_base, adesc + 4, bdesc + 4, idesc_mxf8(256, BN, 2), sfa_t, sfb_t, 1);
-              mma_mxf8_pair(tmem_base, adesc + 6, bdesc + 6, idesc_mxf8(256, BN, 3), sfa_t, sfb_t, 1);
+              mma_mxf8_pair(tmem_base, adesc, bdesc, idesc_mxf8(256, BN, 0) - nsub, sfa_t, sfb_m, kt != 0);
+              mma_mxf8_pair(tmem_base, adesc + 2, bdesc + 2, idesc_mxf8(256, BN, 1) - nsub, sfa_t, sfb_m, 1);
+              mma_mxf8_pair(tmem_base, adesc + 4, bdesc + 4, idesc_mxf8(256, BN, 2) - nsub, sfa_t, sfb_m, 1);
+              mma_mxf8_pair(tmem_base, adesc + 6, bdesc + 6, idesc_mxf8(256, BN, 3) - nsub, sfa_t, sfb_m, 1);
             } else if constexpr (FMT == FMT_NVFP4) {       // one chunk per instruction
 #pragma unroll
               for (int j = 0; j < 4; ++j)
                 if (j < 2 || two)
-                  mma_nvf4_pair(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc0, sfa_t + 4 * j, sfb_t + 8 * j,
+                  mma_nvf4_pair(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc0, sfa_t + 4 * j, sfb_m + 8 * j,
                                 (kt | j) != 0);
             } else {                                       // half a chunk (two scale bytes) per instruction
-              mma_mxf4_pair(tmem_base, adesc, bdesc, idesc0, sfa_t, sfb_t, kt != 0);
-              mma_mxf4_pair(tmem_base, adesc + 2, bdesc + 2, idesc2, sfa_t, sfb_t, 1);
+              mma_mxf4_pair(tmem_base, adesc, bdesc, idesc0, sfa_t, sfb_m, kt != 0);
+              mma_mxf4_pair(tmem_base, adesc + 2, bdesc + 2, idesc2, sfa_t, sfb_m, 1);
               if (two) {
-                mma_mxf4_pair(tmem_base, adesc + 4, bdesc + 4, idesc0, sfa_t + 4, sfb_t + 8, 1);
-                mma_mxf4_pair(tmem_base, adesc + 6, bdesc + 6, idesc2, sfa_t + 4, sfb_t + 8, 1);
+                mma_mxf4_pair(tmem_base, adesc + 4, bdesc + 4, idesc0, sfa_t + 4, sfb_m + 8, 1);
+                mma_mxf4_pair(tmem_base, adesc + 6, bdesc + 6, idesc2, sfa_t + 4, sfb_m + 8, 1);
               }
             }
             tc_commit_pair(empty_bar(s), 3);
@@ -238,9 +258,11 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles && ok; tile += npairs, ++tcount) {
-      int mp, nt;
-      pair_tile_coords(tile, mp_tiles, n_tiles, mp, nt);
+      int mp, tcol;
+      bool narrow;
+      mixed_tile_coords(tile, tiles, mp, tcol, narrow);
       const int mt = 2 * mp + (int)rank;
+      const bool half_only = narrow && h == 1;           // columns 128..191 of a 192-column tile
       ok = mbar_wait_cluster(accf_bar, tcount & 1, cta_abort, err_word, SITE_EPI_ACC_FULL);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
@@ -249,8 +271,10 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       uint32_t v0[32], v1[32], v2[32], v3[32];
       tmem_ld_32x32(tacc, v0);
       tmem_ld_32x32(tacc + 32, v1);
-      tmem_ld_32x32(tacc + 64, v2);
-      tmem_ld_32x32(tacc + 96, v3);
+      if (!half_only) {
+        tmem_ld_32x32(tacc + 64, v2);
+        tmem_ld_32x32(tacc + 96, v3);
+      }
       tmem_ld_wait();
       tc_fence_before_sync();
       __syncwarp();
@@ -268,7 +292,7 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       // with row % 8 as the 128-byte TMA swizzle expects) -> TMA store of a [32 rows x 128 B] box.
       // The store clips rows >= M and columns >= N by itself.
       const int row0 = mt * C::BM + q * 32;
-      const int col0 = nt * BN + h * 128;
+      const int col0 = tcol + h * 128;
       const uint32_t stage_buf = smem_base + out_off + (uint32_t)(warp - 2) * C::OUT_WARP_BYTES;
       const uint32_t my_row = stage_buf + lane * 128;
       const uint32_t sw = (uint32_t)(lane & 7);
@@ -306,7 +330,7 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           flush(col);
         };
         half64(v0, v1, col0);
-        half64(v2, v3, col0 + 64);
+        if (!half_only) half64(v2, v3, col0 + 64);
       } else {
         auto quarter32 = [&](const uint32_t (&v)[32], int col) {
           reuse();
@@ -316,8 +340,10 @@ mxfp4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         };
         quarter32(v0, col0);
         quarter32(v1, col0 + 32);
-        quarter32(v2, col0 + 64);
-        quarter32(v3, col0 + 96);
+        if (!half_only) {
+          quarter32(v2, col0 + 64);
+          quarter32(v3, col0 + 96);
+        }
       }
     }
     if (lane == 0) bulk_wait_group_read<0>();            // shared memory must outlive the stores' reads

@@ -6,6 +6,10 @@
 // feed the tensor pipe.  Every CTA loads only for itself; operand sharing happens inside the MMA, which
 // reads both CTAs' shared memory.
 //
+// Tiles are dealt round robin from the list MixedTiles describes: 256 x 256 tiles, and where those
+// would leave the last wave partly empty, 256 x 192 tiles in its place (N = 192 instructions, 96
+// columns of R_inter per CTA, three 32-blocks per epilogue warp instead of four).
+//
 // Roles per CTA: warp 0 TMA producer (both CTAs), warp 1 MMA issuer (leader CTA only; both
 // allocate tensor memory), warps 2..9 epilogue (each CTA drains its own 128 x 256 accumulator).
 // Barriers: full[s] lives in the leader and counts the bytes of both CTAs' loads; empty[s] and
@@ -50,9 +54,9 @@ struct RotPairCfg {
 template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(320, 1)
 rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
-                            const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
+                            const __grid_constant__ CUtensorMap tmRn, const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
                             uint8_t* __restrict__ scales, int M, int d, float tensor_scale, int x_terms,
-                            int* err_word) {
+                            const MixedTiles tiles, int* err_word) {
   using C = RotPairCfg;
   constexpr int BN = C::BN;
   extern __shared__ uint8_t smem_raw[];
@@ -72,9 +76,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
   const uint32_t rank = cluster_ctarank();             // 0 = leader
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
   const int m_tiles = (M + 127) / 128;                 // 128-row tiles that exist
-  const int mp_tiles = (M + 255) / 256;                // 256-row pair tiles
-  const int n_tiles = (d + BN - 1) / BN;
-  const int total_tiles = mp_tiles * n_tiles;
+  const int total_tiles = tiles.total;                 // 256-row pair tiles, 256 or 192 columns wide
   const int kr_tiles = (d + C::BK - 1) / C::BK;         // K steps over R_inter; X has x_terms times as many
   const int k_tiles = kr_tiles * x_terms;
   const int nblocks = d / 32;
@@ -102,17 +104,19 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
     if (elect_one()) {
       tma_prefetch_desc(&tmX);
       tma_prefetch_desc(&tmR);
-      int mp0, nt;
-      pair_tile_coords(pair, mp_tiles, n_tiles, mp0, nt);
+      int mp0 = 0, col0 = 0;
+      bool narrow = false;
+      if (pre > 0) mixed_tile_coords(pair, tiles, mp0, col0, narrow);
       (void)mp0;
+      const int my_col = col0 + (int)rank * (narrow ? kNarrowCols / 2 : BN / 2);
+      if (narrow) tma_prefetch_desc(&tmRn);
       for (int kt = 0; kt < pre; ++kt) {
         const uint32_t st = smem_base + kt * C::STAGE_BYTES;
         const uint32_t leader_full = map_to_cta(full_bar(kt), 0);
-        if (rank == 0) mbar_arrive_expect_tx(full_bar(kt), 2 * C::STAGE_BYTES);
-#pragma unroll
-        for (int b = 0; b < BN / 2 / 64; ++b)
-          tma_load_2d_pair(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR,
-                           nt * BN + (int)rank * (BN / 2) + b * 64, (kt % kr_tiles) * C::BK, leader_full);
+        if (rank == 0) mbar_arrive_expect_tx(full_bar(kt), 2 * (C::STAGE_BYTES - (narrow ? C::B_BOX_BYTES / 2 : 0)));
+        tma_load_2d_pair(st + C::A_BYTES, &tmR, my_col, (kt % kr_tiles) * C::BK, leader_full);
+        tma_load_2d_pair(st + C::A_BYTES + C::B_BOX_BYTES, narrow ? &tmRn : &tmR, my_col + 64, (kt % kr_tiles) * C::BK,
+                         leader_full);
       }
     }
     __syncwarp();
@@ -124,9 +128,15 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
     uint32_t it = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
-      int mp, nt;
-      pair_tile_coords(tile, mp_tiles, n_tiles, mp, nt);
+      int mp, tcol;
+      bool narrow;
+      mixed_tile_coords(tile, tiles, mp, tcol, narrow);
       const int mt = 2 * mp + (int)rank;
+      // A 192-column tile takes 96 columns of R_inter per CTA: one 64-column box and one 32-column box.
+      // Under the 128-byte swizzle a box whose rows are 64 bytes long still lands on a 128-byte pitch, i.e.
+      // as the first half of the 64-column layout the instruction's descriptor describes.
+      const int my_col = tcol + (int)rank * (narrow ? kNarrowCols / 2 : BN / 2);
+      const uint32_t stage_tx = 2 * (C::STAGE_BYTES - (narrow ? C::B_BOX_BYTES / 2 : 0));
       for (int kt = 0, kr = 0; kt < k_tiles; ++kt, ++it, kr = (kr + 1 == kr_tiles ? 0 : kr + 1)) {
         const int s = it % C::STAGES;
         if (!mbar_wait_cluster_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word,
@@ -135,13 +145,11 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
         const uint32_t leader_full = map_to_cta(full_bar(s), 0);
         if (elect_one()) {
           const bool r_issued = it < (uint32_t)pre;      // R side of this stage went out before the wait above
-          if (rank == 0 && !r_issued) mbar_arrive_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
+          if (rank == 0 && !r_issued) mbar_arrive_expect_tx(full_bar(s), stage_tx);
           tma_load_2d_pair(st, &tmX, kt * C::BK, mt * C::BM, leader_full);
           if (!r_issued) {
-#pragma unroll
-            for (int b = 0; b < BN / 2 / 64; ++b)
-              tma_load_2d_pair(st + C::A_BYTES + b * C::B_BOX_BYTES, &tmR,
-                               nt * BN + (int)rank * (BN / 2) + b * 64, kr * C::BK, leader_full);
+            tma_load_2d_pair(st + C::A_BYTES, &tmR, my_col, kr * C::BK, leader_full);
+            tma_load_2d_pair(st + C::A_BYTES + C::B_BOX_BYTES, narrow ? &tmRn : &tmR, my_col + 64, kr * C::BK, leader_full);
           }
         }
         __syncwarp();
@@ -150,10 +158,16 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader only)
     if (rank == 0) {
-      constexpr uint32_t idesc = idesc_bf16(256, BN, /*A MN-major*/ false, /*B MN-major*/ true);
+      constexpr uint32_t idesc_wide = idesc_bf16(256, BN, /*A MN-major*/ false, /*B MN-major*/ true);
+      constexpr uint32_t idesc_narrow = idesc_bf16(256, kNarrowCols, false, true);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int tile = pair; tile < total_tiles && ok; tile += npairs, ++tcount) {
+        int mp, tcol;
+        bool narrow;
+        mixed_tile_coords(tile, tiles, mp, tcol, narrow);
+        (void)mp; (void)tcol;
+        const uint32_t idesc = narrow ? idesc_narrow : idesc_wide;
         const int a = tcount % C::NACC;
         if (!mbar_wait_cluster_warp(acce_bar(a), ((tcount / C::NACC) & 1) ^ 1, cta_abort, err_word,
                                SITE_MMA_ACC_EMPTY)) { ok = false; break; }
@@ -183,7 +197,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
   } else {
     // ------------------------------------------------------------------ epilogue (8 warps per CTA)
     // warp w reads lane quarter w % 4 (32 rows) and column half (w - 2) / 4 (four 32-blocks = one
-    // 4-byte group of scale bytes).  Two forms of the intra-block rotation:
+    // 4-byte group of scale bytes; three blocks in a 192-column tile).  Two forms of the intra-block rotation:
     //  * fp32 FMAs, one row per thread, R_intra broadcast from shared memory as fp32.  Bound by
     //    that broadcast (8 bytes per lane and cycle): about 3/4 of a mainloop per tile, which does
     //    not matter while the next tile's mainloop runs beside it on the tensor pipe.
@@ -199,11 +213,13 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles; tile += npairs, ++tcount) {
-      int mp, nt;
-      pair_tile_coords(tile, mp_tiles, n_tiles, mp, nt);
+      int mp, tcol;
+      bool narrow;
+      mixed_tile_coords(tile, tiles, mp, tcol, narrow);
       const int mt = 2 * mp + (int)rank;
       const int a = tcount % C::NACC;
-      const int b0 = nt * (BN / 32);
+      const int b0 = tcol >> 5;                          // first 32-block of the tile: even, 2 mod 4 for some narrow tiles
+      const int nbb = narrow ? 3 : 4;                    // this warp's blocks: half of the tile's 8 or 6
       const bool last = FMT != FMT_F32OUT && tile + npairs >= total_tiles;
       if (R_intra != nullptr) {
         // Executed by every epilogue thread for every tile, also after a wait has given up.
@@ -233,8 +249,35 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) continue;
       tc_fence_after_sync();
-      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + h * 128;
-      const int chunk = (b0 + h * 4) >> 2;
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + h * nbb * 32;
+      // Scale bytes: block blk of row r sits in byte blk % 4 of the 4-byte cell of (r, blk / 4).  The four
+      // bytes of a wide tile's half are one cell; the three of a narrow tile's half go out one by one.
+      const int fb = b0 + h * nbb;
+      auto put_scales = [&](uint32_t w, size_t in_tile) {  // byte bb of w = scale of block fb + bb
+        if (nbb == 4) {
+          if ((fb >> 2) < kb4) *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4 + (fb >> 2)) * 512 + in_tile) = w;
+        } else {
+          for (int j = 0; j < nbb; ++j) {
+            const int blk = fb + j;
+            if ((blk >> 2) < kb4) scales[((size_t)mt * kb4 + (blk >> 2)) * 512 + in_tile + (blk & 3)] = (uint8_t)(w >> (8 * j));
+          }
+        }
+      };
+      // NVFP4: two bytes per block, cells of two blocks
+      auto put_scales16 = [&](uint32_t w01, uint32_t w23, size_t in_tile, int kb4n) {
+        if (nbb == 4) {
+          if ((fb >> 1) < kb4n) *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4n + (fb >> 1)) * 512 + in_tile) = w01;
+          if ((fb >> 1) + 1 < kb4n)
+            *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4n + (fb >> 1) + 1) * 512 + in_tile) = w23;
+        } else {
+          for (int j = 0; j < nbb; ++j) {
+            const int blk = fb + j;
+            if ((blk >> 1) < kb4n)
+              *reinterpret_cast<uint16_t*>(scales + ((size_t)mt * kb4n + (blk >> 1)) * 512 + in_tile + 2 * (blk & 1)) =
+                  (uint16_t)((j < 2 ? w01 : w23) >> (16 * (j & 1)));
+          }
+        }
+      };
       if (!last) {
         // ---- one row per thread, fp32 FMAs
         const int64_t row = (int64_t)mt * C::BM + q * 32 + lane;
@@ -242,23 +285,23 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
         NvScale nvs = {};
         if constexpr (FMT == FMT_NVFP4) nvs = nv_scale(tensor_scale);
 #pragma unroll 1
-        for (int bb = 0; bb < 4; ++bb) {
+        for (int bb = 0; bb < nbb; ++bb) {
           uint32_t yv[32];
           tmem_ld_32x32(tacc + bb * 32, yv);
           tmem_ld_wait();
-          if (bb == 3) {                                 // this warp's share is read: tell the leader
+          if (bb == nbb - 1) {                           // this warp's share is read: tell the leader
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar(a), 0));
           }
           float z[32];
           if (R_intra != nullptr) {
-            intra_rotate32(yv, ri_saddr + (uint32_t)(h * 4 + bb) * 4096, z);
+            intra_rotate32(yv, ri_saddr + (uint32_t)(h * nbb + bb) * 4096, z);
           } else {
 #pragma unroll
             for (int j = 0; j < 32; ++j) z[j] = __uint_as_float(yv[j]);
           }
-          const int blk = b0 + h * 4 + bb;
+          const int blk = fb + bb;
           if constexpr (FMT == FMT_F32OUT) {               // the rotated values themselves
             if (row < M && blk < nblocks) {
               float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(codes) + row * (int64_t)d + (int64_t)blk * 32);
@@ -294,16 +337,10 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
         if constexpr (FMT == FMT_F32OUT) {
           continue;
         } else if constexpr (FMT == FMT_NVFP4) {
-          const int kb4n = (2 * nblocks + 3) / 4;        // 4-byte groups of 16-block scales per row
-          if (mt < m_tiles) {
-            if (2 * chunk < kb4n)
-              *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4n + 2 * chunk) * 512 + lane * 16 + q * 4) = sc_word;
-            if (2 * chunk + 1 < kb4n)
-              *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4n + 2 * chunk + 1) * 512 + lane * 16 + q * 4) = sc_word2;
-          }
+          const int kb4n = (2 * nblocks + 3) / 4;        // 4-byte groups of 16-block scales per row: blocks fb, fb + 1
+          if (mt < m_tiles) put_scales16(sc_word, sc_word2, (size_t)lane * 16 + q * 4, kb4n);
         } else {
-          if (chunk < kb4 && mt < m_tiles)               // the pair's second row tile may not exist
-            *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4 + chunk) * 512 + lane * 16 + q * 4) = sc_word;
+          if (mt < m_tiles) put_scales(sc_word, (size_t)lane * 16 + q * 4);   // the pair's second row tile may not exist
         }
         continue;
       }
@@ -315,12 +352,12 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
       NvScale nvs = {};
       if constexpr (FMT == FMT_NVFP4) nvs = nv_scale(tensor_scale);
 #pragma unroll 1
-      for (int bb = 0; bb < 4; ++bb) {
-        const int blk = b0 + h * 4 + bb;
+      for (int bb = 0; bb < nbb; ++bb) {
+        const int blk = fb + bb;
         uint32_t bfrag[2][4][2];                         // [k chunk][n tile][2]
         if (R_intra != nullptr) {
           // lane l: row l % 8 of matrix l / 8; matrices (k 0-7, n), (k 8-15, n), (k 0-7, n+8), (k 8-15, n+8)
-          const uint32_t rb = ri_saddr + (uint32_t)(h * 4 + bb) * C::RI_BLOCK_BYTES +
+          const uint32_t rb = ri_saddr + (uint32_t)(h * nbb + bb) * C::RI_BLOCK_BYTES +
                               (uint32_t)(((lane >> 3) & 1) * 8 + (lane & 7)) * C::RI_ROW_BYTES +
                               (uint32_t)(lane >> 4) * 16;
 #pragma unroll
@@ -335,7 +372,7 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
           uint32_t y[16];
           tmem_ld_16x256b_x4(tacc + ((uint32_t)(16 * mh) << 16) + bb * 32, y);
           tmem_ld_wait();
-          if (bb == 3 && mh == 1) {                      // this warp's share is read: tell the leader
+          if (bb == nbb - 1 && mh == 1) {                // this warp's share is read: tell the leader
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar(a), 0));
@@ -401,18 +438,13 @@ rotate_quantize_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __gri
         if (p == 0 && mt < m_tiles) {
 #pragma unroll
           for (int rs = 0; rs < 4; ++rs) {
-            const size_t in_tile = (size_t)(r8 + 16 * (rs >> 1) + 8 * (rs & 1)) * 16 + q * 4;
-            if (2 * chunk < kb4n)
-              *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4n + 2 * chunk) * 512 + in_tile) = sc_word[rs];
-            if (2 * chunk + 1 < kb4n)
-              *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4n + 2 * chunk + 1) * 512 + in_tile) = sc_hi[rs];
+            put_scales16(sc_word[rs], sc_hi[rs], (size_t)(r8 + 16 * (rs >> 1) + 8 * (rs & 1)) * 16 + q * 4, kb4n);
           }
         }
-      } else if (p == 0 && chunk < kb4 && mt < m_tiles) {  // the pair's second row tile may not exist
+      } else if (p == 0 && mt < m_tiles) {               // the pair's second row tile may not exist
 #pragma unroll
         for (int rs = 0; rs < 4; ++rs)
-          *reinterpret_cast<uint32_t*>(scales + ((size_t)mt * kb4 + chunk) * 512 +
-                                       (r8 + 16 * (rs >> 1) + 8 * (rs & 1)) * 16 + q * 4) = sc_word[rs];
+          put_scales(sc_word[rs], (size_t)(r8 + 16 * (rs >> 1) + 8 * (rs & 1)) * 16 + q * 4);
       }
     }
   }

@@ -471,13 +471,71 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t cta_mask) 
 // 8 row tiles x 9 column tiles, whatever M is, so both operands of a wave stay in L2 (with the row
 // tile as the fast index over ALL of M, a wave at M = 16384 touched 64 row tiles and one or two
 // column tiles, and the row operand was re-read from HBM for every column tile).
-__device__ __forceinline__ void pair_tile_coords(int tile, int mp_tiles, int n_tiles, int& mp, int& nt) {
+__host__ __device__ __forceinline__ void pair_tile_coords(int tile, int mp_tiles, int n_tiles, int& mp, int& nt) {
   constexpr int G = 8;
   const int per_group = G * n_tiles;
   const int g = tile / per_group, r = tile - g * per_group;
-  const int rows_in_group = min(G, mp_tiles - g * G);
+  const int rows_in_group = mp_tiles - g * G < G ? mp_tiles - g * G : G;
   mp = g * G + r % rows_in_group;
   nt = r / rows_in_group;
+}
+
+// Tile list of the pair kernels when the last wave is cut into narrower tiles.  A row tile (256
+// rows) is covered by 256-column tiles followed by 192-column tiles; three wide tiles traded for
+// four narrow ones is one "unit".  The first `rows_a` row tiles trade one unit more than the
+// others, so every split is described by four numbers.  Tiles are numbered wide ones first (the
+// columns every row tile has as wide tiles, then the three more of the rows that trade less),
+// then the narrow ones in the same two groups; each group is walked in the order of
+// pair_tile_coords.  With narrow_b == 0 and rows_a == 0 this is pair_tile_coords itself.
+struct MixedTiles {
+  int rows;        // 256-row tiles
+  int rows_a;      // row tiles [0, rows_a) have wide_b - 3 wide and narrow_b + 4 narrow tiles
+  int wide_b;      // 256-column tiles of the other row tiles
+  int narrow_b;    // 192-column tiles of the other row tiles
+  int total;       // tiles in all
+};
+constexpr int kNarrowCols = 192;
+
+__host__ __device__ __forceinline__ MixedTiles mixed_tiles_make(int rows, int wide_cols, int units) {
+  MixedTiles t;
+  t.rows = rows;
+  t.rows_a = units % rows;
+  t.wide_b = wide_cols - 3 * (units / rows);
+  t.narrow_b = 4 * (units / rows);
+  t.total = rows * wide_cols + units;
+  return t;
+}
+
+__host__ __device__ __forceinline__ void mixed_tile_coords(int tile, const MixedTiles& t, int& mp, int& col0, bool& narrow) {
+  const int wide_common = t.rows_a > 0 ? t.wide_b - 3 : t.wide_b;
+  int nt;
+  const int n1 = t.rows * wide_common;
+  if (tile < n1) {
+    pair_tile_coords(tile, t.rows, wide_common, mp, nt);
+    col0 = nt * 256;
+    narrow = false;
+    return;
+  }
+  tile -= n1;
+  const int rows_b = t.rows - t.rows_a;
+  const int n2 = t.rows_a > 0 ? rows_b * 3 : 0;
+  if (tile < n2) {
+    mp = t.rows_a + tile % rows_b;
+    col0 = (wide_common + tile / rows_b) * 256;
+    narrow = false;
+    return;
+  }
+  tile -= n2;
+  narrow = true;
+  const int n3 = t.rows * t.narrow_b;
+  if (tile < n3) {
+    pair_tile_coords(tile, t.rows, t.narrow_b, mp, nt);
+  } else {
+    tile -= n3;
+    mp = tile % t.rows_a;
+    nt = t.narrow_b + tile / t.rows_a;
+  }
+  col0 = (mp < t.rows_a ? t.wide_b - 3 : t.wide_b) * 256 + nt * kNarrowCols;
 }
 
 // Instruction descriptors (32-bit).  Common fields: [17,23) N>>3, [24,29) M>>4, bit 15 / 16 =

@@ -223,6 +223,52 @@ static inline int fewtok_cluster(int64_t tiles, int64_t k_steps, int min_k, int 
   if (s == 7) s = 6;
   return s < 1 ? 1 : (int)s;
 }
+constexpr double kNarrowTileCost = 0.88;   // a 192-column tile against a 256-column one: 0.75 of the math, 0.875 of the operand bytes
+
+// Tile list of a pair kernel: `rows` 256-row tiles by `cols` columns on `max_pairs` CTA pairs, tiles dealt
+// round robin.  When the 256-column tiles do not fill the last wave, trading three of them for four 192-column
+// tiles (one unit) in some row tiles shortens that wave from one tile time to about three quarters.  The number
+// of units is the one with the smallest longest-pair time, a narrow tile counted as `narrow_cost` wide tiles;
+// zero unless it wins by at least 1 % (and always zero when the columns are not whole 256-column tiles).
+static MixedTiles plan_pair_tiles(int rows, int64_t cols, int max_pairs, double narrow_cost) {
+  const int wide_cols = (int)((cols + 255) / 256);
+  if (cols % 256 != 0 || rows < 1) return mixed_tiles_make(rows < 1 ? 1 : rows, wide_cols, 0);
+  struct Memo { int rows, wide_cols, max_pairs; double cost; int units; };
+  static thread_local Memo memo[8] = {};
+  static thread_local int memo_next = 0;
+  for (const Memo& m : memo)
+    if (m.rows == rows && m.wide_cols == wide_cols && m.max_pairs == max_pairs && m.cost == narrow_cost)
+      return mixed_tiles_make(rows, wide_cols, m.units);
+  auto longest = [&](int units) {
+    const int wide = rows * wide_cols - 3 * units, narrow = 4 * units;
+    const int P = wide + narrow < max_pairs ? wide + narrow : max_pairs;
+    double worst = 0.0;
+    for (int p = 0; p < P; ++p) {
+      const int w = wide / P + (p < wide % P ? 1 : 0);
+      // narrow tiles have the numbers wide .. wide + narrow - 1; pair p takes those congruent to p
+      const int first = wide + ((p - wide) % P + P) % P;
+      const int n = first < wide + narrow ? (wide + narrow - 1 - first) / P + 1 : 0;
+      const double t = w + narrow_cost * n;
+      if (t > worst) worst = t;
+    }
+    return worst;
+  };
+  const int max_units = rows * (wide_cols / 3);
+  const double base = longest(0);
+  double best = base;
+  int best_units = 0;
+  for (int u = 1; u <= max_units && 4 * u <= max_pairs + 8; ++u) {
+    // the row tiles that trade one unit more must have the three wide tiles to give
+    if (u % rows != 0 && 3 * (u / rows + 1) > wide_cols) break;
+    const double t = longest(u);
+    if (t < best - 1e-9) { best = t; best_units = u; }
+  }
+  if (best > 0.99 * base) best_units = 0;
+  memo[memo_next] = Memo{rows, wide_cols, max_pairs, narrow_cost, best_units};
+  memo_next = (memo_next + 1) % 8;
+  return mixed_tiles_make(rows, wide_cols, best_units);
+}
+
 static size_t quantized_bytes(int64_t M, int64_t d) {    // codes, then 256-byte aligned the scales
   return ((size_t)M * (size_t)(d / 2) + 255) / 256 * 256 + torq_scales_bytes(M, d);
 }
@@ -278,6 +324,20 @@ const char* torq_status_string(torq_status s) {
     case TORQ_ERR_WORKSPACE: return "workspace missing or too small";
   }
   return "unknown";
+}
+
+int64_t torq_pair_tile_list(int64_t rows, int64_t cols, int32_t pairs, int32_t* out, int64_t cap) {
+  if (rows < 1 || cols < 1 || pairs < 1 || rows > INT32_MAX / 2 || cols > INT32_MAX / 2) return -1;
+  const torq::MixedTiles t = torq::plan_pair_tiles((int)((rows + 255) / 256), cols, pairs, torq::kNarrowTileCost);
+  for (int i = 0; out && i < t.total && i < cap; ++i) {
+    int mp, col0;
+    bool narrow;
+    torq::mixed_tile_coords(i, t, mp, col0, narrow);
+    out[3 * i] = mp;
+    out[3 * i + 1] = col0;
+    out[3 * i + 2] = narrow ? torq::kNarrowCols : 256;
+  }
+  return t.total;
 }
 
 int64_t torq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
@@ -389,26 +449,29 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
     return launch_status();
   }
   if (M > 128) {
-    // CTA pairs: 256 x 256 tiles, one pair per two SMs.
-    const int ptiles = (int)((M + 255) / 256) * (int)((d + 255) / 256);
+    // CTA pairs: 256 x 256 tiles (the last wave 256 x 192 where that fills it better), one pair per two SMs.
     const int max_pairs = st->rot_pairs;
-    const int pairs = ptiles < max_pairs ? ptiles : max_pairs;
+    CUtensorMap tmRn;                                      // second half of a narrow tile's 96 columns per CTA
+    if (!encode_2d(&tmRn, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 32))
+      return TORQ_ERR_LAUNCH;
+    const MixedTiles tiles = plan_pair_tiles((int)((M + 255) / 256), d, max_pairs, kNarrowTileCost);
+    const int pairs = tiles.total < max_pairs ? tiles.total : max_pairs;
     if (fmt == FMT_MXINT4)
       launch_tc(rotate_quantize_pair_kernel<FMT_MXINT4>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
-                s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
-                x_terms, st->err_word);
+                s, tmX, tmR, tmRn, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
+                x_terms, tiles, st->err_word);
     else if (fmt == FMT_NVFP4)
       launch_tc(rotate_quantize_pair_kernel<FMT_NVFP4>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
-                s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d,
-                tensor_scale, x_terms, st->err_word);
+                s, tmX, tmR, tmRn, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d,
+                tensor_scale, x_terms, tiles, st->err_word);
     else if (fmt == FMT_F32OUT)
       launch_tc(rotate_quantize_pair_kernel<FMT_F32OUT>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
-                s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
-                x_terms, st->err_word);
+                s, tmX, tmR, tmRn, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
+                x_terms, tiles, st->err_word);
     else
       launch_tc(rotate_quantize_pair_kernel<FMT_MXFP4>, 2, 2 * pairs, RotPairCfg::THREADS, RotPairCfg::SMEM_BYTES,
-                s, tmX, tmR, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
-                x_terms, st->err_word);
+                s, tmX, tmR, tmRn, static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, 0.0f,
+                x_terms, tiles, st->err_word);
     return launch_status();
   }
   const int m_tiles = (int)((M + 127) / 128);
@@ -548,11 +611,14 @@ static torq_status gemm_impl(const void* Aq, const void* As, const void* Wq, con
     if (!encode_2d(&tmY, ybf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, ybf ? 2 : 4,
                    Y, (uint64_t)M, (uint64_t)N, 32, ybf ? 64 : 32))
       return TORQ_ERR_LAUNCH;
-    const int ptiles = (int)((M + 255) / 256) * (int)((N + BN - 1) / BN);
+    CUtensorMap tmBn;                                      // half of a 192-column tile: 96 rows of W
+    if (!encode_2d(&tmBn, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, krow, kNarrowCols / 2, 128))
+      return TORQ_ERR_LAUNCH;
     const int max_pairs = st->gemm_pairs;
-    const int pairs = ptiles < max_pairs ? ptiles : max_pairs;
+    const MixedTiles tiles = plan_pair_tiles((int)((M + 255) / 256), N, max_pairs, kNarrowTileCost);
+    const int pairs = tiles.total < max_pairs ? tiles.total : max_pairs;
     launch_tc(mxfp4_gemm_pair_kernel<FMT>, 2, 2 * pairs, GemmPairCfgT<FMT>::THREADS, GemmPairCfgT<FMT>::SMEM_BYTES, s,
-              tmA, tmB, tmSFA, tmSFB, tmY, ybf ? 1 : 0, (int)M, (int)N, (int)K, alpha, st->err_word);
+              tmA, tmB, tmSFA, tmSFB, tmY, tmBn, tiles, ybf ? 1 : 0, (int)M, (int)N, (int)K, alpha, st->err_word);
     return launch_status();
   }
   // One or two row tiles: the work is streaming W once, so prefer the narrower tile while it still leaves

@@ -111,6 +111,8 @@ def lib() -> ctypes.CDLL:
     L.torq_status_string.restype = ctypes.c_char_p
     L.torq_last_device_error.argtypes = [vp]
     L.torq_last_device_error.restype = ci
+    L.torq_pair_tile_list.argtypes = [i64, i64, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), i64]
+    L.torq_pair_tile_list.restype = i64
     L.torq_launch_count.argtypes = []
     L.torq_launch_count.restype = i64
     _lib_handle = L
@@ -148,6 +150,16 @@ def torq_scale_offset(row: int, kblock: int, k: int) -> int:
 
 def torq_workspace_bytes(M: int, d: int, N: int) -> int:
     return lib().torq_workspace_bytes(M, d, N)
+
+
+def torq_pair_tile_list(rows: int, cols: int, pairs: int = 74):
+    """[(row_tile, first_column, width), ...] in dealing order (host helper, no device work)."""
+    n = lib().torq_pair_tile_list(rows, cols, pairs, None, 0)
+    if n < 0:
+        raise ValueError("torq_pair_tile_list: rows, cols and pairs must be positive")
+    buf = (ctypes.c_int32 * (3 * n))()
+    lib().torq_pair_tile_list(rows, cols, pairs, buf, n)
+    return [(buf[3 * i], buf[3 * i + 1], buf[3 * i + 2]) for i in range(n)]
 
 
 def torq_launch_count() -> int:

@@ -130,3 +130,36 @@ def test_probe_argument_errors():
     d = ctypes.c_double(0.0)
     assert L.torq_probe_fp4_peak(100, None, None) == 1
     assert L.torq_probe_fp4_peak(0, ctypes.byref(d), None) == 2
+
+
+def test_pair_tile_list_covers_every_output_exactly_once():
+    """Host logic of the CTA-pair kernels' tile list: whatever the planner trades, the tiles partition the
+    [row tiles x cols] output, narrow tiles start on a multiple of 64 columns (two 32-blocks: the scale bytes
+    of a block pair never straddle two tiles), and the longest pair never gets longer than with 256-column
+    tiles alone."""
+    import numpy as np
+    shapes = [(2048, 4096), (2048, 6144), (2048, 14336), (1024, 5120), (16384, 5120), (8192, 51200), (300, 256),
+              (129, 4096), (4864, 1024), (3840, 1280), (2560, 2048), (2500, 2048), (2048, 4000), (640, 768),
+              (19 * 256, 1024), (75 * 256, 256), (74 * 256 + 1, 512)]
+    for pairs in (74, 66, 8):
+        for rows, cols in shapes:
+            tl = torq.torq_pair_tile_list(rows, cols, pairs)
+            rt = (rows + 255) // 256
+            cover = np.zeros((rt, (cols + 31) // 32), np.int32)
+            for mp, c0, w in tl:
+                assert 0 <= mp < rt and w in (192, 256) and c0 % 64 == 0 and c0 < cols
+                assert w == 256 or (cols % 256 == 0 and c0 + w <= cols)
+                cover[mp, c0 // 32:min(cols, c0 + w + 31) // 32 if c0 + w < cols else cover.shape[1]] += 1
+            assert (cover == 1).all(), (pairs, rows, cols)
+            # wide tiles are dealt before narrow ones
+            widths = [w for _, _, w in tl]
+            assert widths == sorted(widths, reverse=True)
+            load = np.zeros(pairs)
+            for i, w in enumerate(widths):
+                load[i % pairs] += w / 256.0
+            wide_only = -(-(rt * ((cols + 255) // 256)) // pairs)
+            assert load.max() <= wide_only + 1e-9
+    # the LLaMA3-8B QKV rotation on 74 pairs: one wave of 74 wide tiles, then 72 narrow ones
+    tl = torq.torq_pair_tile_list(2048, 4096, 74)
+    assert [w for _, _, w in tl].count(256) == 74 and [w for _, _, w in tl].count(192) == 72
+    assert torq.lib().torq_pair_tile_list(0, 4096, 74, None, 0) == -1
