@@ -2,7 +2,7 @@
 """Benchmark of the rotated-MXFP4 linear hot path (rotate -> MXFP4 quantize -> block-scaled FP4
 GEMM).  The timed K steps run the LLaMA3-8B QKV-projection shape (M=2048 tokens, d=4096, N=6144,
 bf16 output); the same line also carries the second 8B shape (down-projection, 2048 x 14336 ->
-4096) and a token sweep at d = N = 5120 (M = 1, 64, 1024, 16384), each with per-kernel times,
+4096) and a token sweep at d = N = 5120 (M = 1, 64, 256, 1024, 16384), each with per-kernel times,
 both roofline fractions and the SM clock sampled inside its own loop.
 
 One step = one pass of the whole path over one batch of seeded synthetic activations.  Prints ONE
@@ -276,7 +276,7 @@ def layer_work(M, d, N):
 
 
 def rotation_kernel_name(M, d, sm_count):
-    if M <= 64 and d % 128 == 0:
+    if M <= 256 and d % 128 == 0:
         return "rotate_fewtok_kernel"
     if 2 * ((M + 127) // 128) * ((d + 255) // 256) <= sm_count:
         return "rotate_splitk_kernel + splitk_reduce_quantize_kernel"
@@ -284,7 +284,7 @@ def rotation_kernel_name(M, d, sm_count):
 
 
 def gemm_kernel_name(M):
-    return "gemm_fewtok_kernel" if M <= 64 else ("mxfp4_gemm_pair_kernel" if M > 128 else "mxfp4_gemm_kernel")
+    return "gemm_fewtok_kernel" if M <= 128 else ("mxfp4_gemm_pair_kernel" if M > 128 else "mxfp4_gemm_kernel")
 
 
 class Layer:
@@ -548,7 +548,7 @@ def measure_e2e(torq, layer, stream, steps, barrier):
     barrier()
     return e0.elapsed_time(e1) / n, Xh.numel() * 2, Yh[0].numel() * 2
 
-SWEEP_M = (1, 64, 1024, 16384)
+SWEEP_M = (1, 64, 256, 1024, 16384)
 
 
 def main():

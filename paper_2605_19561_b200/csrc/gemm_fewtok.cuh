@@ -1,8 +1,8 @@
-// Block-scaled GEMM for few tokens (M <= 64; Algorithm 3 step 5), where the work is streaming the
+// Block-scaled GEMM for few tokens (M <= 128; Algorithm 3 step 5), where the work is streaming the
 // weights from HBM once.  One kernel, no scratch in global memory.
 //
 // Swapped operands: the tensor-core instruction's 128 rows are 128 output FEATURES (rows of the
-// stored weight W' [N, K]) and its N columns are the tokens (16, 32 or 64):
+// stored weight W' [N, K]) and its N columns are the tokens (16, 32, 64 or 128):
 //   D[n, m] = sum_k w^[n, k] a^[m, k]
 //   A = W tile [128 rows x 128 B of K], scale chunks of W;  B = activation tile [tokens x 128 B],
 //   scale chunks of the activations (their single 128-row scale tile).
@@ -36,12 +36,14 @@ struct GemmFewCfg {
   static constexpr int BAR_BYTES = 256;
   static constexpr int THREADS = 192;
   static constexpr int MAX_CLUSTER = 8;
+  static constexpr int MAX_TOK = 128;                  // one 128-row scale tile of the activations
   __host__ __device__ static constexpr int stage_bytes(int ntok) {
     return (A_BYTES + ntok * 128 + 2 * SF_BYTES + 1023) / 1024 * 1024;
   }
   __host__ __device__ static constexpr int smem_bytes(int ntok) { return STAGES * stage_bytes(ntok) + BAR_BYTES + 1024; }
+  __host__ __device__ static constexpr int ctas_per_sm(int ntok) { return smem_bytes(ntok) <= 113 * 1024 ? 2 : 1; }
   __host__ __device__ static constexpr uint32_t tmem_cols(int ntok) {
-    return ntok + 8 * CH <= 32 ? 32u : (ntok + 8 * CH <= 64 ? 64u : 128u);
+    return ntok + 8 * CH <= 32 ? 32u : (ntok + 8 * CH <= 64 ? 64u : (ntok + 8 * CH <= 128 ? 128u : 256u));
   }
 };
 
@@ -75,37 +77,34 @@ gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   const int kt0 = (int)((long long)k_tiles * rank / S), kt1 = (int)((long long)k_tiles * (rank + 1) / S);
   const uint32_t tmem_cols = C::tmem_cols(ntok);
 
+  // The weights and their scales are constants of the layer, never the output of the kernel that runs
+  // just before this one: the thread that initialises the barriers sends their loads for the first
+  // stages right behind the initialisation (the kernel's time starts with an HBM round trip; tensor-
+  // memory allocation and the block-wide barrier come after it instead of before); the activations wait.
+  const int pre = (kt1 - kt0) < C::STAGES ? (kt1 - kt0) : C::STAGES;
+  auto stage_tx = [&](int kt) { return (uint32_t)(C::A_BYTES + b_bytes) + 2u * 512u * (uint32_t)min(CH, kb4 - CH * kt); };
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(accf_bar, 1);
     *cta_abort = 0;
     fence_mbar_init();
+    fence_proxy_async_smem();                            // the copy engine sees the initialised barriers
+    for (int it = 0; it < pre; ++it) {
+      const int kt = kt0 + it;
+      const uint32_t st = smem_base + it * stage_bytes;
+      mbar_arrive_expect_tx(full_bar(it), stage_tx(kt));
+      tma_load_2d(st, &tmW, kt * 128, nt * C::BF, full_bar(it));
+      bulk_load_1d(st + C::A_BYTES + b_bytes, Ws + ((size_t)nt * kb4 + CH * kt) * 512,
+                   512u * (uint32_t)min(CH, kb4 - CH * kt), full_bar(it));
+    }
+    tma_prefetch_desc(&tmA);
   }
   if (warp == 1) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), tmem_cols); tmem_relinquish(); }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  // The weights and their scales are constants of the layer, never the output of the kernel that runs
-  // just before this one: their loads for the first stages go out right away; the activations wait.
   griddep_launch_dependents();
-  const int pre = (kt1 - kt0) < C::STAGES ? (kt1 - kt0) : C::STAGES;
-  auto stage_tx = [&](int kt) { return (uint32_t)(C::A_BYTES + b_bytes) + 2u * 512u * (uint32_t)min(CH, kb4 - CH * kt); };
-  if (warp == 0) {
-    if (elect_one()) {
-      tma_prefetch_desc(&tmW);
-      tma_prefetch_desc(&tmA);
-      for (int it = 0; it < pre; ++it) {
-        const int kt = kt0 + it;
-        const uint32_t st = smem_base + it * stage_bytes;
-        mbar_arrive_expect_tx(full_bar(it), stage_tx(kt));
-        tma_load_2d(st, &tmW, kt * 128, nt * C::BF, full_bar(it));
-        bulk_load_1d(st + C::A_BYTES + b_bytes, Ws + ((size_t)nt * kb4 + CH * kt) * 512,
-                     512u * (uint32_t)min(CH, kb4 - CH * kt), full_bar(it));
-      }
-    }
-    __syncwarp();
-  }
   griddep_wait();
 
   bool acc_ok = false;

@@ -1,8 +1,8 @@
-// Rotate + quantize for few tokens (M <= 64), where the work is streaming R_inter from HBM once
+// Rotate + quantize for few tokens (M <= 256), where the work is streaming R_inter from HBM once
 // (Algorithm 3 steps 2-4).  One kernel, no scratch in global memory.
 //
 // Swapped operands: the tensor-core instruction's 128 rows are 128 output FEATURES (four 32-blocks)
-// and its N columns are the tokens (16, 32 or 64), so no row of the instruction is padding and the
+// and its N columns are the tokens (16 ... 256), so no row of the instruction is padding and the
 // accumulator is small:  D[j, m] = sum_i R_inter[i, j] X[m, i].
 //   A = R_inter tile [64 (i) x 128 (j)], features contiguous = MN-major, two 64 x 64 boxes (128-B swizzle)
 //   B = X tile [tokens x 64 (i)], K-major
@@ -21,8 +21,9 @@
 //
 // Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue / reduction.
 // Shared memory: 4 stages of (16 KiB of R_inter + tokens x 128 B of X); after the mainloop the same
-// memory holds the partial tile and the per-warp staging of the reduction.  Small enough (<= 107 KiB)
-// for two CTAs per SM: the grid may exceed the SM count, which keeps more loads in flight.
+// memory holds the partial tile and the per-warp staging of the reduction.  Up to 64 tokens that is small
+// enough (<= 107 KiB) for two CTAs per SM: the grid may exceed the SM count, which keeps more loads in
+// flight; with 128 or 256 tokens one CTA fills an SM and the grid stays within the SM count.
 #pragma once
 #include <cuda_bf16.h>
 #include "intra_fragment.cuh"
@@ -36,7 +37,7 @@ struct RotFewCfg {
   static constexpr int A_BYTES = BK * BF * 2;          // 16 KiB: two boxes of 64 (k) x 64 (j)
   static constexpr int A_BOX_BYTES = 64 * 64 * 2;
   static constexpr int STAGES = 4;
-  static constexpr int MAX_TOK = 64;
+  static constexpr int MAX_TOK = 256;                  // N of the instruction; 16, 32, 64, 128 or 256 are used
   static constexpr int Y_BYTES = 16 * 33 * 4;          // per epilogue warp: 16 tokens x 32 features, row stride 33
   static constexpr int RI_BYTES = 32 * 80;             // per epilogue warp: R_intra[block] as bf16 rows of 80 bytes
   static constexpr int BAR_BYTES = 256;
@@ -46,12 +47,14 @@ struct RotFewCfg {
   __host__ __device__ static constexpr int smem_bytes(int ntok) {
     return STAGES * stage_bytes(ntok) + BAR_BYTES + 4 * RI_BYTES + 1024;
   }
-  // the partial tile and the warps' y tiles must fit inside the stages they reuse
-  static_assert(MAX_TOK * BF * 4 + 4 * Y_BYTES <= STAGES * (A_BYTES + 16 * BK * 2), "reduction buffers");
+  // the partial tile (ntok x 512 B) and the warps' y tiles must fit inside the stages they reuse
+  // (4 x (16 KiB + ntok x 128 B)): true for every ntok
+  static_assert(4 * Y_BYTES <= STAGES * A_BYTES && BF * 4 <= STAGES * BK * 2, "reduction buffers");
+  __host__ __device__ static constexpr int ctas_per_sm(int ntok) { return smem_bytes(ntok) <= 113 * 1024 ? 2 : 1; }
 };
 
 // grid = (d / 128) * S CTAs in clusters of S along x: CTA b works feature tile b / S, k split b % S.
-// tmX: X [M, d] bf16, box [ntok rows x 64]; tmR: R_inter [d, d] bf16, box [64 x 64].  ntok = 16, 32 or 64
+// tmX: X [M, d] bf16, box [ntok rows x 64]; tmR: R_inter [d, d] bf16, box [64 x 64].  ntok = 16, 32, 64, 128 or 256
 // >= M.  d % 128 == 0.  `codes` / `scales` / `tensor_scale` as in rotate_quantize_kernel for FMT.
 template <int FMT = FMT_MXFP4>
 __global__ void __launch_bounds__(192, 2)
@@ -82,34 +85,31 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   const int kt0 = (int)((long long)k_tiles * rank / S), kt1 = (int)((long long)k_tiles * (rank + 1) / S);
   const uint32_t tmem_cols = ntok < 32 ? 32u : (uint32_t)ntok;
 
+  // R_inter is a constant of the layer, never the output of the kernel that runs just before this
+  // one: the thread that initialises the barriers sends the loads of the first stages' R_inter tiles
+  // right behind the initialisation (the kernel's time starts with an HBM round trip; tensor-memory
+  // allocation and the block-wide barrier come after it instead of before).  X waits for that kernel.
+  const int pre = (kt1 - kt0) < C::STAGES ? (kt1 - kt0) : C::STAGES;
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(accf_bar, 1);
     *cta_abort = 0;
     fence_mbar_init();
+    fence_proxy_async_smem();                            // the copy engine sees the initialised barriers
+    for (int it = 0; it < pre; ++it) {
+      const uint32_t st = smem_base + it * stage_bytes;
+      mbar_arrive_expect_tx(full_bar(it), (uint32_t)stage_bytes);
+      tma_load_2d(st, &tmR, ft * C::BF, (kt0 + it) * C::BK, full_bar(it));
+      tma_load_2d(st + C::A_BOX_BYTES, &tmR, ft * C::BF + 64, (kt0 + it) * C::BK, full_bar(it));
+    }
+    tma_prefetch_desc(&tmX);
   }
   if (warp == 1) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), tmem_cols); tmem_relinquish(); }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  // R_inter is a constant of the layer, never the output of the kernel that runs just before this
-  // one: its loads for the first stages go out right away; X waits for that kernel.
   griddep_launch_dependents();
-  const int pre = (kt1 - kt0) < C::STAGES ? (kt1 - kt0) : C::STAGES;
-  if (warp == 0) {
-    if (elect_one()) {
-      tma_prefetch_desc(&tmX);
-      tma_prefetch_desc(&tmR);
-      for (int it = 0; it < pre; ++it) {
-        const uint32_t st = smem_base + it * stage_bytes;
-        mbar_arrive_expect_tx(full_bar(it), (uint32_t)stage_bytes);
-        tma_load_2d(st, &tmR, ft * C::BF, (kt0 + it) * C::BK, full_bar(it));
-        tma_load_2d(st + C::A_BOX_BYTES, &tmR, ft * C::BF + 64, (kt0 + it) * C::BK, full_bar(it));
-      }
-    }
-    __syncwarp();
-  }
   const int groups = ntok / 16;                          // token groups of 16; group g belongs to CTA g % S
   if (warp >= 2 && R_intra != nullptr && rank < groups) {
     // this warp's R_intra block (a constant of the layer as well), 128 pieces of 16 B: row piece / 4

@@ -120,9 +120,9 @@ static DeviceState* device_state() {
               opt_in_smem(rotate_fewtok_kernel<FMT_MXFP4>, RotFewCfg::smem_bytes(RotFewCfg::MAX_TOK)) &&
               opt_in_smem(rotate_fewtok_kernel<FMT_NVFP4>, RotFewCfg::smem_bytes(RotFewCfg::MAX_TOK)) &&
               opt_in_smem(rotate_fewtok_kernel<FMT_MXINT4>, RotFewCfg::smem_bytes(RotFewCfg::MAX_TOK)) &&
-              opt_in_smem(gemm_fewtok_kernel<FMT_MXFP4>, GemmFewCfg<FMT_MXFP4>::smem_bytes(RotFewCfg::MAX_TOK)) &&
-              opt_in_smem(gemm_fewtok_kernel<FMT_NVFP4>, GemmFewCfg<FMT_NVFP4>::smem_bytes(RotFewCfg::MAX_TOK)) &&
-              opt_in_smem(gemm_fewtok_kernel<FMT_MXINT4>, GemmFewCfg<FMT_MXINT4>::smem_bytes(RotFewCfg::MAX_TOK)) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_MXFP4>, GemmFewCfg<FMT_MXFP4>::smem_bytes(GemmFewCfg<FMT_MXFP4>::MAX_TOK)) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_NVFP4>, GemmFewCfg<FMT_NVFP4>::smem_bytes(GemmFewCfg<FMT_NVFP4>::MAX_TOK)) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_MXINT4>, GemmFewCfg<FMT_MXINT4>::smem_bytes(GemmFewCfg<FMT_MXINT4>::MAX_TOK)) &&
               opt_in_smem(rotate_quantize_kernel<256, FMT_F32OUT>, RotCfg<256>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_pair_kernel<FMT_F32OUT>, RotPairCfg::SMEM_BYTES);
     if (!ok) return nullptr;
@@ -210,14 +210,18 @@ static int rotation_splits(int64_t M, int64_t d, int sm_count) {
   if (s > k_tiles / 2) s = k_tiles / 2;
   return s < 2 ? 1 : s;
 }
-// Few-token kernels (M <= 64): tokens per instruction and the cluster size = number of K splits of
+constexpr int kRotFewMaxTokens = 256;    // up to here the rotation streams R_inter through the few-token kernel
+constexpr int kGemmFewMaxTokens = 128;   // and the GEMM the weights
+static_assert(kRotFewMaxTokens <= RotFewCfg::MAX_TOK && kGemmFewMaxTokens <= GemmFewCfg<FMT_MXFP4>::MAX_TOK, "few-token limits");
+// Few-token kernels: tokens per instruction and the cluster size = number of K splits of
 // one 128-feature tile.  Two of these CTAs fit on an SM, and a grid of about 1.4 CTAs per SM measured
 // fastest (more loads in flight; beyond that the clusters no longer all become resident at once):
 // the largest S <= 8 with tiles * S <= 1.4 SMs, each split at least `min_k` K steps.  7 is skipped:
 // clusters of 7 did not all become resident at sizes where 6 and 8 did.
-static inline int fewtok_ntok(int64_t M) { return M <= 16 ? 16 : (M <= 32 ? 32 : 64); }
-static inline int fewtok_cluster(int64_t tiles, int64_t k_steps, int min_k, int sm_count) {
-  int64_t s = (int64_t)sm_count * 14 / 10 / (tiles > 0 ? tiles : 1);
+static inline int fewtok_ntok(int64_t M) { return M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : (M <= 128 ? 128 : 256))); }
+static inline int fewtok_cluster(int64_t tiles, int64_t k_steps, int min_k, int sm_count, int ctas_per_sm) {
+  // two CTAs fit on an SM: 1.4 per SM on average keeps the most bytes in flight; one: one wave
+  int64_t s = (int64_t)sm_count * (ctas_per_sm >= 2 ? 14 : 10) / 10 / (tiles > 0 ? tiles : 1);
   if (s > 8) s = 8;
   if (s > k_steps / min_k) s = k_steps / min_k;
   if (s == 7) s = 6;
@@ -396,12 +400,12 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
     return launch_status();
   }
   CUtensorMap tmX, tmR;
-  if (M <= RotFewCfg::MAX_TOK && d % 128 == 0 && x_terms == 1 && fmt != FMT_F32OUT) {
+  if (M <= kRotFewMaxTokens && d % 128 == 0 && x_terms == 1 && fmt != FMT_F32OUT) {
     // Few tokens: 128 features x all tokens per CTA, K split over a cluster, reduced through
     // distributed shared memory; one launch, no scratch.
     const int ntok = fewtok_ntok(M);
     const int tiles = (int)(d / 128);
-    const int S = fewtok_cluster(tiles, d / 64, 2, st->sm_count);
+    const int S = fewtok_cluster(tiles, d / 64, 2, st->sm_count, RotFewCfg::ctas_per_sm(ntok));
     if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d, (uint32_t)ntok, 64) ||
         !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
       return TORQ_ERR_LAUNCH;
@@ -575,13 +579,13 @@ static torq_status gemm_impl(const void* Aq, const void* As, const void* Wq, con
   constexpr int BN = 256;
   const uint64_t krow = (uint64_t)(FMT == FMT_MXINT4 ? K : K / 2);   // operand bytes per row
   CUtensorMap tmA, tmB;
-  if (M <= RotFewCfg::MAX_TOK) {
+  if (M <= kGemmFewMaxTokens) {
     // Few tokens: 128 output features x all tokens per CTA, K split over a cluster, reduced through
     // distributed shared memory.
     using FC = GemmFewCfg<FMT>;
     const int ntok = fewtok_ntok(M);
     const int tiles = (int)((N + 127) / 128);
-    const int S = fewtok_cluster(tiles, (K + FC::BK - 1) / FC::BK, 1, st->sm_count);
+    const int S = fewtok_cluster(tiles, (K + FC::BK - 1) / FC::BK, 1, st->sm_count, FC::ctas_per_sm(ntok));
     if (!encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, krow, 128, 128) ||
         !encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, krow, (uint32_t)ntok, 128))
       return TORQ_ERR_LAUNCH;

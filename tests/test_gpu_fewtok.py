@@ -1,5 +1,5 @@
-"""GPU parity of the few-token kernels (up to 64 tokens; the regime where the layer streams R_inter
-and W from HBM once): the rotation that splits its contraction over a cluster and reduces the
+"""GPU parity of the few-token kernels (rotation up to 256 tokens, GEMM up to 128; the regime where the layer
+streams R_inter and W from HBM once): the rotation that splits its contraction over a cluster and reduces the
 partial sums through distributed shared memory, and the GEMM built the same way, against the oracle.
 Same bounds as everywhere else: rotate + quantize at most 1e-4 of the elements one lattice step off
 and 1e-4 of the block scales one step off (one element / block at sizes where 1e-4 is less than
@@ -26,7 +26,9 @@ def _rand_rotation(d, seed):
 
 # cluster sizes reached on 148 SMs: d = 128 -> 1, 256 -> 2, 640 -> 5, 1536 -> 8, 2560 -> 7, 4096 -> 4, 5120 -> 3
 @pytest.mark.parametrize("M,d", [(1, 128), (16, 256), (17, 256), (32, 640), (33, 640), (64, 1536), (5, 2560),
-                                 (48, 4096), (1, 5120), (64, 5120)])
+                                 (48, 4096), (1, 5120), (64, 5120),
+                                 # 128 and 256 tokens per instruction (one CTA per SM), two row tiles of scales
+                                 (65, 256), (100, 1536), (128, 640), (129, 256), (200, 5120), (256, 2560), (130, 4096)])
 def test_rotation_alone_without_any_workspace(M, d):
     g = np.random.default_rng(1000 * M + d)
     xb = I.to_bf16_bits(g.standard_t(3.0, size=(M, d)))
@@ -96,7 +98,8 @@ def _gpu_gemm(ac, asb, wc, wsb, out_dtype):
 # K = 128 (one half stage), 384 (a half last stage), 640 and 5120 (several stages per split); N ragged in the
 # last 128-row tile; cluster sizes 1 .. 8
 @pytest.mark.parametrize("M,N,K", [(1, 8, 128), (16, 136, 384), (17, 640, 640), (33, 2560, 1024), (64, 5120, 5120),
-                                   (5, 4096, 4096), (64, 264, 2048), (40, 1000, 896)])
+                                   (5, 4096, 4096), (64, 264, 2048), (40, 1000, 896),
+                                   (65, 136, 384), (100, 2560, 1024), (128, 5120, 5120), (97, 1000, 896)])
 def test_gemm_random_operands(M, N, K):
     ac, asb = _rand_operand(M, K, 1)
     wc, wsb = _rand_operand(N, K, 2)
