@@ -108,11 +108,12 @@ torq_status torq_mxfp4_gemm(const void* Aq, const void* As, const void* Wq, cons
 /* Algorithm 3 steps 1-5 in one call: rotate, quantize, multiply.  The quantized activations live
  * in `workspace` (>= torq_workspace_bytes(M, d, N) bytes, 256-byte aligned), laid out as codes
  * [M, d/2] followed (256-byte aligned) by the tiled scales; pass dbg_codes / dbg_scales non-NULL
- * to also receive copies of them.  When the rotation has few output tiles (128 rows x 256 columns
- * each) relative to the number of SMs -- few tokens, or a narrow layer -- the workspace also holds
- * fp32 partial tiles: the rotation is then split along its contraction so that every SM streams a
- * share of R_inter, and a second kernel adds the partials in a fixed order before the intra-block
- * step and Eq. 1.
+ * to also receive copies of them.  Up to 256 tokens the rotation is one kernel that splits its
+ * contraction over thread-block clusters and adds the partial sums on chip, in a fixed order.
+ * Beyond that, when the rotation has few output tiles (128 rows x 256 columns each) relative to
+ * the number of SMs -- a narrow layer -- the workspace also holds fp32 partial tiles: the rotation
+ * is then split along its contraction so that every SM streams a share of R_inter, and a second
+ * kernel adds the partials in a fixed order before the intra-block step and Eq. 1.
  * Requires d % 128 == 0 and N % 8 == 0. */
 torq_status torq_rotated_linear(const void* X, const void* R_inter, const void* R_intra,
                                 const void* Wq, const void* Ws, int64_t M, int64_t d, int64_t N,
