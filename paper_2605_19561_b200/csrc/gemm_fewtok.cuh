@@ -33,6 +33,9 @@ struct GemmFewCfg {
   static constexpr int CH = FMT == FMT_NVFP4 ? 4 : (FMT == FMT_MXINT4 ? 1 : 2);   // scale chunks per stage and 128 rows
   static constexpr int SF_BYTES = CH * 512;
   static constexpr int STAGES = 4;
+  // the same for every token count: three stages at 128 tokens would let two CTAs share an SM (clusters of 5
+  // instead of 3), which measured 4 - 10 % slower than four stages and one CTA per SM
+  __host__ __device__ static constexpr int stages(int) { return STAGES; }
   static constexpr int BAR_BYTES = 256;
   static constexpr int THREADS = 192;
   static constexpr int MAX_CLUSTER = 8;
@@ -40,8 +43,11 @@ struct GemmFewCfg {
   __host__ __device__ static constexpr int stage_bytes(int ntok) {
     return (A_BYTES + ntok * 128 + 2 * SF_BYTES + 1023) / 1024 * 1024;
   }
-  __host__ __device__ static constexpr int smem_bytes(int ntok) { return STAGES * stage_bytes(ntok) + BAR_BYTES + 1024; }
+  __host__ __device__ static constexpr int smem_bytes(int ntok) { return stages(ntok) * stage_bytes(ntok) + BAR_BYTES + 1024; }
   __host__ __device__ static constexpr int ctas_per_sm(int ntok) { return smem_bytes(ntok) <= 113 * 1024 ? 2 : 1; }
+  __host__ __device__ static constexpr int max_smem_bytes() {                  // over the token counts in use
+    return smem_bytes(64) > smem_bytes(128) ? smem_bytes(64) : smem_bytes(128);
+  }
   __host__ __device__ static constexpr uint32_t tmem_cols(int ntok) {
     return ntok + 8 * CH <= 32 ? 32u : (ntok + 8 * CH <= 64 ? 64u : (ntok + 8 * CH <= 128 ? 128u : 256u));
   }
@@ -61,7 +67,8 @@ gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const int stage_bytes = C::stage_bytes(ntok);
   const int b_bytes = ntok * 128;
-  const uint32_t bar_off = C::STAGES * stage_bytes;
+  const int nst = C::stages(ntok);
+  const uint32_t bar_off = nst * stage_bytes;
   const uint32_t bar_base = smem_base + bar_off;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };
@@ -81,10 +88,10 @@ gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   // just before this one: the thread that initialises the barriers sends their loads for the first
   // stages right behind the initialisation (the kernel's time starts with an HBM round trip; tensor-
   // memory allocation and the block-wide barrier come after it instead of before); the activations wait.
-  const int pre = (kt1 - kt0) < C::STAGES ? (kt1 - kt0) : C::STAGES;
+  const int pre = (kt1 - kt0) < nst ? (kt1 - kt0) : nst;
   auto stage_tx = [&](int kt) { return (uint32_t)(C::A_BYTES + b_bytes) + 2u * 512u * (uint32_t)min(CH, kb4 - CH * kt); };
   if (threadIdx.x == 0) {
-    for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < nst; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(accf_bar, 1);
     *cta_abort = 0;
     fence_mbar_init();
@@ -112,8 +119,8 @@ gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     // ------------------------------------------------------------------ TMA producer
     bool ok = true;
     for (int kt = kt0, it = 0; kt < kt1 && ok; ++kt, ++it) {
-      const int s = it % C::STAGES;
-      if (!mbar_wait_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word, SITE_PRODUCER_EMPTY)) {
+      const int s = it % nst;
+      if (!mbar_wait_warp(empty_bar(s), ((it / nst) & 1) ^ 1, cta_abort, err_word, SITE_PRODUCER_EMPTY)) {
         ok = false; break;
       }
       const uint32_t st = smem_base + s * stage_bytes;
@@ -137,8 +144,8 @@ gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     const uint32_t idesc2 = FMT == FMT_NVFP4 ? idesc_nvf4(128, ntok) : idesc_mxf4(128, ntok, 2, 2);
     const uint32_t sfa_t = tmem_base + ntok, sfb_t = tmem_base + ntok + 4 * CH;     // 4 columns per chunk each
     for (int kt = kt0, it = 0; kt < kt1 && ok; ++kt, ++it) {
-      const int s = it % C::STAGES;
-      if (!mbar_wait_warp(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
+      const int s = it % nst;
+      if (!mbar_wait_warp(full_bar(s), (it / nst) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
         ok = false; break;
       }
       tc_fence_after_sync();

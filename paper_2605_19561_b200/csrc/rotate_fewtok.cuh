@@ -37,6 +37,9 @@ struct RotFewCfg {
   static constexpr int A_BYTES = BK * BF * 2;          // 16 KiB: two boxes of 64 (k) x 64 (j)
   static constexpr int A_BOX_BYTES = 64 * 64 * 2;
   static constexpr int STAGES = 4;
+  // the same for every token count: three stages at 128 tokens would let two CTAs share an SM (clusters of 5
+  // instead of 3), which measured 4 - 10 % slower than four stages and one CTA per SM
+  __host__ __device__ static constexpr int stages(int) { return STAGES; }
   static constexpr int MAX_TOK = 256;                  // N of the instruction; 16, 32, 64, 128 or 256 are used
   static constexpr int Y_BYTES = 16 * 33 * 4;          // per epilogue warp: 16 tokens x 32 features, row stride 33
   static constexpr int RI_BYTES = 32 * 80;             // per epilogue warp: R_intra[block] as bf16 rows of 80 bytes
@@ -45,13 +48,19 @@ struct RotFewCfg {
   static constexpr int MAX_CLUSTER = 8;
   __host__ __device__ static constexpr int stage_bytes(int ntok) { return A_BYTES + ntok * BK * 2; }
   __host__ __device__ static constexpr int smem_bytes(int ntok) {
-    return STAGES * stage_bytes(ntok) + BAR_BYTES + 4 * RI_BYTES + 1024;
+    return stages(ntok) * stage_bytes(ntok) + BAR_BYTES + 4 * RI_BYTES + 1024;
   }
   // the partial tile (ntok x 512 B) and the warps' y tiles must fit inside the stages they reuse
-  // (4 x (16 KiB + ntok x 128 B)): true for every ntok
-  static_assert(4 * Y_BYTES <= STAGES * A_BYTES && BF * 4 <= STAGES * BK * 2, "reduction buffers");
+  __host__ __device__ static constexpr bool reduction_fits(int ntok) {
+    return ntok * BF * 4 + 4 * Y_BYTES <= stages(ntok) * stage_bytes(ntok);
+  }
   __host__ __device__ static constexpr int ctas_per_sm(int ntok) { return smem_bytes(ntok) <= 113 * 1024 ? 2 : 1; }
+  __host__ __device__ static constexpr int max_smem_bytes() {                  // over the token counts in use
+    return smem_bytes(256) > smem_bytes(64) ? smem_bytes(256) : smem_bytes(64);
+  }
 };
+static_assert(RotFewCfg::reduction_fits(16) && RotFewCfg::reduction_fits(32) && RotFewCfg::reduction_fits(64) &&
+              RotFewCfg::reduction_fits(128) && RotFewCfg::reduction_fits(256), "reduction buffers");
 
 // grid = (d / 128) * S CTAs in clusters of S along x: CTA b works feature tile b / S, k split b % S.
 // tmX: X [M, d] bf16, box [ntok rows x 64]; tmR: R_inter [d, d] bf16, box [64 x 64].  ntok = 16, 32, 64, 128 or 256
@@ -67,7 +76,8 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const int stage_bytes = C::stage_bytes(ntok);
-  const uint32_t bar_off = C::STAGES * stage_bytes;
+  const int nst = C::stages(ntok);
+  const uint32_t bar_off = nst * stage_bytes;
   const uint32_t bar_base = smem_base + bar_off;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };
@@ -89,9 +99,9 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   // one: the thread that initialises the barriers sends the loads of the first stages' R_inter tiles
   // right behind the initialisation (the kernel's time starts with an HBM round trip; tensor-memory
   // allocation and the block-wide barrier come after it instead of before).  X waits for that kernel.
-  const int pre = (kt1 - kt0) < C::STAGES ? (kt1 - kt0) : C::STAGES;
+  const int pre = (kt1 - kt0) < nst ? (kt1 - kt0) : nst;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < nst; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(accf_bar, 1);
     *cta_abort = 0;
     fence_mbar_init();
@@ -128,8 +138,8 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     // ------------------------------------------------------------------ TMA producer
     bool ok = true;
     for (int kt = kt0, it = 0; kt < kt1 && ok; ++kt, ++it) {
-      const int s = it % C::STAGES;
-      if (!mbar_wait_warp(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, cta_abort, err_word, SITE_PRODUCER_EMPTY)) {
+      const int s = it % nst;
+      if (!mbar_wait_warp(empty_bar(s), ((it / nst) & 1) ^ 1, cta_abort, err_word, SITE_PRODUCER_EMPTY)) {
         ok = false; break;
       }
       const uint32_t st = smem_base + s * stage_bytes;
@@ -149,8 +159,8 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const uint32_t idesc = idesc_bf16(128, ntok, /*A MN-major*/ true, /*B MN-major*/ false);
     bool ok = true;
     for (int kt = kt0, it = 0; kt < kt1 && ok; ++kt, ++it) {
-      const int s = it % C::STAGES;
-      if (!mbar_wait_warp(full_bar(s), (it / C::STAGES) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
+      const int s = it % nst;
+      if (!mbar_wait_warp(full_bar(s), (it / nst) & 1, cta_abort, err_word, SITE_MMA_FULL)) {
         ok = false; break;
       }
       tc_fence_after_sync();

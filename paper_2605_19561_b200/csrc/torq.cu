@@ -117,12 +117,12 @@ static DeviceState* device_state() {
               opt_in_smem(rotate_quantize_kernel<256, FMT_MXINT4>, RotCfg<256>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_pair_kernel<FMT_MXINT4>, RotPairCfg::SMEM_BYTES) &&
               opt_in_smem(rotate_structured_kernel<FMT_MXINT4>, RotStructCfg::SMEM_BYTES) &&
-              opt_in_smem(rotate_fewtok_kernel<FMT_MXFP4>, RotFewCfg::smem_bytes(RotFewCfg::MAX_TOK)) &&
-              opt_in_smem(rotate_fewtok_kernel<FMT_NVFP4>, RotFewCfg::smem_bytes(RotFewCfg::MAX_TOK)) &&
-              opt_in_smem(rotate_fewtok_kernel<FMT_MXINT4>, RotFewCfg::smem_bytes(RotFewCfg::MAX_TOK)) &&
-              opt_in_smem(gemm_fewtok_kernel<FMT_MXFP4>, GemmFewCfg<FMT_MXFP4>::smem_bytes(GemmFewCfg<FMT_MXFP4>::MAX_TOK)) &&
-              opt_in_smem(gemm_fewtok_kernel<FMT_NVFP4>, GemmFewCfg<FMT_NVFP4>::smem_bytes(GemmFewCfg<FMT_NVFP4>::MAX_TOK)) &&
-              opt_in_smem(gemm_fewtok_kernel<FMT_MXINT4>, GemmFewCfg<FMT_MXINT4>::smem_bytes(GemmFewCfg<FMT_MXINT4>::MAX_TOK)) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_MXFP4>, RotFewCfg::max_smem_bytes()) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_NVFP4>, RotFewCfg::max_smem_bytes()) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_MXINT4>, RotFewCfg::max_smem_bytes()) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_MXFP4>, GemmFewCfg<FMT_MXFP4>::max_smem_bytes()) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_NVFP4>, GemmFewCfg<FMT_NVFP4>::max_smem_bytes()) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_MXINT4>, GemmFewCfg<FMT_MXINT4>::max_smem_bytes()) &&
               opt_in_smem(rotate_quantize_kernel<256, FMT_F32OUT>, RotCfg<256>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_pair_kernel<FMT_F32OUT>, RotPairCfg::SMEM_BYTES);
     if (!ok) return nullptr;
