@@ -52,7 +52,7 @@ struct RotFewCfg {
   }
   // the partial tile (ntok x 512 B) and the warps' y tiles must fit inside the stages they reuse
   __host__ __device__ static constexpr bool reduction_fits(int ntok) {
-    return ntok * BF * 4 + 4 * Y_BYTES <= stages(ntok) * stage_bytes(ntok);
+    return ntok * BF * 4 + 8 * Y_BYTES <= stages(ntok) * stage_bytes(ntok);   // up to eight epilogue warps
   }
   __host__ __device__ static constexpr int ctas_per_sm(int ntok) { return smem_bytes(ntok) <= 113 * 1024 ? 2 : 1; }
   __host__ __device__ static constexpr int max_smem_bytes() {                  // over the token counts in use
@@ -65,8 +65,11 @@ static_assert(RotFewCfg::reduction_fits(16) && RotFewCfg::reduction_fits(32) && 
 // grid = (d / 128) * S CTAs in clusters of S along x: CTA b works feature tile b / S, k split b % S.
 // tmX: X [M, d] bf16, box [ntok rows x 64]; tmR: R_inter [d, d] bf16, box [64 x 64].  ntok = 16, 32, 64, 128 or 256
 // >= M.  d % 128 == 0.  `codes` / `scales` / `tensor_scale` as in rotate_quantize_kernel for FMT.
-template <int FMT = FMT_MXFP4>
-__global__ void __launch_bounds__(192, 2)
+// ESETS: sets of four epilogue warps (threads = 64 + 128 ESETS).  One set and two CTAs per SM up to 64
+// tokens; with 128 or 256 tokens a CTA fills an SM by itself and has several token groups to reduce, rotate
+// and quantize, each a dependent chain of about a microsecond for one warp: two sets take them in turn.
+template <int FMT = FMT_MXFP4, int ESETS = 1>
+__global__ void __launch_bounds__(64 + 128 * ESETS, ESETS == 1 ? 2 : 1)
 rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
                      const __nv_bfloat16* __restrict__ R_intra, uint8_t* __restrict__ codes,
                      uint8_t* __restrict__ scales, int M, int d, int ntok, int S, float tensor_scale,
@@ -121,7 +124,7 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   const uint32_t tmem_base = *tmem_slot;
   griddep_launch_dependents();
   const int groups = ntok / 16;                          // token groups of 16; group g belongs to CTA g % S
-  if (warp >= 2 && R_intra != nullptr && rank < groups) {
+  if (warp >= 2 && warp < 6 && R_intra != nullptr && rank < groups) {
     // this warp's R_intra block (a constant of the layer as well), 128 pieces of 16 B: row piece / 4
     uint8_t* r_s = ri_tiles + (warp - 2) * C::RI_BYTES;
     const uint4* src = reinterpret_cast<const uint4*>(R_intra + (size_t)(ft * 4 + (warp - 2)) * 1024);
@@ -188,10 +191,11 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     // that code cost about 2.5 us of instruction fetches -- a fifth of the kernel.  Pass 1 is the
     // real one: accumulator -> own shared memory, cluster barrier, then the units of this warp.
     const int q = warp & 3;
-    const int ew = warp - 2;                             // 0..3 = 32-block of the tile
+    const int ew = (warp - 2) & 3;                       // 0..3 = 32-block of the tile
+    const int es = (warp - 2) >> 2;                      // set of epilogue warps
     const int nblocks = d / 32;
     const int blk = ft * 4 + ew;
-    float* y_s = reinterpret_cast<float*>(y_tiles + ew * C::Y_BYTES);
+    float* y_s = reinterpret_cast<float*>(y_tiles + (es * 4 + ew) * C::Y_BYTES);
     const uint32_t r_saddr = smem_u32(ri_tiles + ew * C::RI_BYTES);
     const uint32_t p_saddr = smem_u32(P);
     // lane l adds tokens (l / 8) + 4 j, j = 0..3, features 4 (l % 8) .. + 3 of the block, two tokens at a
@@ -210,7 +214,7 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
           // every load into the stages has landed and every instruction that read them has completed
           const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
           float* prow = P + q * 32 + lane;               // feature 32 q + lane of token 0
-          for (int c0 = 0; c0 < ntok; c0 += 16) {
+          for (int c0 = 16 * es; c0 < ntok; c0 += 16 * ESETS) {
             uint32_t v[16];
             tmem_ld_32x32_x16(tacc + c0, v);
             tmem_ld_wait();
@@ -226,7 +230,7 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 #pragma unroll
       for (int s = 0; s < C::MAX_CLUSTER; ++s)
         p_rank[s] = s < S ? map_to_cta(p_saddr, live ? (uint32_t)s : (uint32_t)rank) : 0u;
-      for (int g = rank; g < groups; g += S) {
+      for (int g = rank + es * S; g < groups; g += S * ESETS) {
 #pragma unroll
         for (int jh = 0; jh < 2; ++jh) {
           if (16 * g + 8 * jh >= M) break;               // rows 8 jh .. 8 jh + 7 of the group hold no token
@@ -260,7 +264,7 @@ rotate_fewtok_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
       }
     }
     // scale bytes of the rows no unit covers (ntok .. 127 of the single 128-row scale tile): zero
-    if (rank == 0) {
+    if (rank == 0 && es == 0) {
       const int row = ew * 32 + lane;
       if (row >= ntok) {
         if constexpr (FMT == FMT_NVFP4) {

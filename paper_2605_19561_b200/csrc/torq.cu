@@ -117,9 +117,12 @@ static DeviceState* device_state() {
               opt_in_smem(rotate_quantize_kernel<256, FMT_MXINT4>, RotCfg<256>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_pair_kernel<FMT_MXINT4>, RotPairCfg::SMEM_BYTES) &&
               opt_in_smem(rotate_structured_kernel<FMT_MXINT4>, RotStructCfg::SMEM_BYTES) &&
-              opt_in_smem(rotate_fewtok_kernel<FMT_MXFP4>, RotFewCfg::max_smem_bytes()) &&
-              opt_in_smem(rotate_fewtok_kernel<FMT_NVFP4>, RotFewCfg::max_smem_bytes()) &&
-              opt_in_smem(rotate_fewtok_kernel<FMT_MXINT4>, RotFewCfg::max_smem_bytes()) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_MXFP4, 1>, RotFewCfg::max_smem_bytes()) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_MXFP4, 2>, RotFewCfg::max_smem_bytes()) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_NVFP4, 1>, RotFewCfg::max_smem_bytes()) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_NVFP4, 2>, RotFewCfg::max_smem_bytes()) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_MXINT4, 1>, RotFewCfg::max_smem_bytes()) &&
+              opt_in_smem(rotate_fewtok_kernel<FMT_MXINT4, 2>, RotFewCfg::max_smem_bytes()) &&
               opt_in_smem(gemm_fewtok_kernel<FMT_MXFP4>, GemmFewCfg<FMT_MXFP4>::max_smem_bytes()) &&
               opt_in_smem(gemm_fewtok_kernel<FMT_NVFP4>, GemmFewCfg<FMT_NVFP4>::max_smem_bytes()) &&
               opt_in_smem(gemm_fewtok_kernel<FMT_MXINT4>, GemmFewCfg<FMT_MXINT4>::max_smem_bytes()) &&
@@ -410,16 +413,29 @@ static torq_status rotate_quantize_impl(const void* X, const void* R_inter, cons
         !encode_2d(&tmR, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, R_inter, (uint64_t)d, (uint64_t)d, 64, 64))
       return TORQ_ERR_LAUNCH;
     const int smem = RotFewCfg::smem_bytes(ntok);
-    if (fmt == FMT_MXINT4)
-      launch_tc(rotate_fewtok_kernel<FMT_MXINT4>, S, tiles * S, RotFewCfg::THREADS, smem, s, tmX, tmR,
-                static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, ntok, S, 0.0f, st->err_word);
-    else if (fmt == FMT_NVFP4)
-      launch_tc(rotate_fewtok_kernel<FMT_NVFP4>, S, tiles * S, RotFewCfg::THREADS, smem, s, tmX, tmR,
-                static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, ntok, S, tensor_scale,
-                st->err_word);
-    else
-      launch_tc(rotate_fewtok_kernel<FMT_MXFP4>, S, tiles * S, RotFewCfg::THREADS, smem, s, tmX, tmR,
-                static_cast<const __nv_bfloat16*>(R_intra), codes, scales, (int)M, (int)d, ntok, S, 0.0f, st->err_word);
+    const float ts = fmt == FMT_NVFP4 ? tensor_scale : 0.0f;
+    const __nv_bfloat16* ri = static_cast<const __nv_bfloat16*>(R_intra);
+    if (RotFewCfg::ctas_per_sm(ntok) >= 2) {             // up to 64 tokens: one set of epilogue warps, two CTAs per SM
+      if (fmt == FMT_MXINT4)
+        launch_tc(rotate_fewtok_kernel<FMT_MXINT4, 1>, S, tiles * S, 192, smem, s, tmX, tmR, ri, codes, scales, (int)M,
+                  (int)d, ntok, S, ts, st->err_word);
+      else if (fmt == FMT_NVFP4)
+        launch_tc(rotate_fewtok_kernel<FMT_NVFP4, 1>, S, tiles * S, 192, smem, s, tmX, tmR, ri, codes, scales, (int)M,
+                  (int)d, ntok, S, ts, st->err_word);
+      else
+        launch_tc(rotate_fewtok_kernel<FMT_MXFP4, 1>, S, tiles * S, 192, smem, s, tmX, tmR, ri, codes, scales, (int)M,
+                  (int)d, ntok, S, ts, st->err_word);
+    } else {                                             // 128 or 256 tokens: two sets
+      if (fmt == FMT_MXINT4)
+        launch_tc(rotate_fewtok_kernel<FMT_MXINT4, 2>, S, tiles * S, 320, smem, s, tmX, tmR, ri, codes, scales, (int)M,
+                  (int)d, ntok, S, ts, st->err_word);
+      else if (fmt == FMT_NVFP4)
+        launch_tc(rotate_fewtok_kernel<FMT_NVFP4, 2>, S, tiles * S, 320, smem, s, tmX, tmR, ri, codes, scales, (int)M,
+                  (int)d, ntok, S, ts, st->err_word);
+      else
+        launch_tc(rotate_fewtok_kernel<FMT_MXFP4, 2>, S, tiles * S, 320, smem, s, tmX, tmR, ri, codes, scales, (int)M,
+                  (int)d, ntok, S, ts, st->err_word);
+    }
     return launch_status();
   }
   if (!encode_2d(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)d * x_terms, 128, 64) ||
