@@ -55,8 +55,10 @@ struct GemmFewCfg {
 
 // grid = ceil(N / 128) * S CTAs in clusters of S along x: CTA b works feature tile b / S, k split b % S.
 // tmW: Wq [N, K bytes] box [128 x 128]; tmA: Aq [M, K bytes] box [ntok x 128]; As / Ws: tiled scales.
-template <int FMT = FMT_MXFP4>
-__global__ void __launch_bounds__(192, 2)
+// ESETS: sets of four epilogue warps (threads = 64 + 128 ESETS): one set and two CTAs per SM up to 64 tokens;
+// two sets at 128 tokens, where a CTA fills an SM by itself and has some forty tokens to add up and store.
+template <int FMT = FMT_MXFP4, int ESETS = 1>
+__global__ void __launch_bounds__(64 + 128 * ESETS, ESETS == 1 ? 2 : 1)
 gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA,
                    const uint8_t* __restrict__ As, const uint8_t* __restrict__ Ws, void* __restrict__ Y,
                    int y_is_bf16, int M, int N, int K, int ntok, int S, float alpha, int* err_word) {
@@ -197,7 +199,8 @@ gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     // bytes per warp and partial) and stores 8 or 16 bytes of the token's row of Y.  Two tokens per
     // iteration, all their loads issued before the first add: few round trips through the cluster.
     const int q = warp & 3;
-    const int ew = warp - 2;
+    const int ew = warp - 2;                             // 0 .. 4 ESETS - 1
+    constexpr int NW = 4 * ESETS;
     const int64_t n = (int64_t)nt * C::BF + 4 * lane;
     const uint32_t p_saddr = smem_u32(P);
 #pragma unroll 1
@@ -211,7 +214,7 @@ gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
           tc_fence_after_sync();
           const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
           float* prow = P + q * 32 + lane;               // feature 32 q + lane of token 0
-          for (int c0 = 0; c0 < ntok; c0 += 16) {
+          for (int c0 = 16 * (ew >> 2); c0 < ntok; c0 += 16 * ESETS) {
             uint32_t v[16];
             tmem_ld_32x32_x16(tacc + c0, v);
             tmem_ld_wait();
@@ -227,11 +230,11 @@ gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 #pragma unroll
       for (int s = 0; s < C::MAX_CLUSTER; ++s)
         p_rank[s] = s < S ? map_to_cta(p_saddr, live ? (uint32_t)s : (uint32_t)rank) : 0u;
-      for (int m0 = rank + S * ew; m0 < M; m0 += 8 * S) {
+      for (int m0 = rank + S * ew; m0 < M; m0 += 2 * NW * S) {
         float4 part[2][C::MAX_CLUSTER];
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
-          const int m = m0 + 4 * S * j;
+          const int m = m0 + NW * S * j;
           if (m < M) {
             const uint32_t off = (uint32_t)((m * C::BF + 4 * lane) * 4);
 #pragma unroll
@@ -244,7 +247,7 @@ gemm_fewtok_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         }
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
-          const int m = m0 + 4 * S * j;
+          const int m = m0 + NW * S * j;
           if (m < M) {
             float4 y = make_float4(0.f, 0.f, 0.f, 0.f);  // rank order: the result does not depend on timing
 #pragma unroll

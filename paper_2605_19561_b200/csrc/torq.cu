@@ -123,9 +123,12 @@ static DeviceState* device_state() {
               opt_in_smem(rotate_fewtok_kernel<FMT_NVFP4, 2>, RotFewCfg::max_smem_bytes()) &&
               opt_in_smem(rotate_fewtok_kernel<FMT_MXINT4, 1>, RotFewCfg::max_smem_bytes()) &&
               opt_in_smem(rotate_fewtok_kernel<FMT_MXINT4, 2>, RotFewCfg::max_smem_bytes()) &&
-              opt_in_smem(gemm_fewtok_kernel<FMT_MXFP4>, GemmFewCfg<FMT_MXFP4>::max_smem_bytes()) &&
-              opt_in_smem(gemm_fewtok_kernel<FMT_NVFP4>, GemmFewCfg<FMT_NVFP4>::max_smem_bytes()) &&
-              opt_in_smem(gemm_fewtok_kernel<FMT_MXINT4>, GemmFewCfg<FMT_MXINT4>::max_smem_bytes()) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_MXFP4, 1>, GemmFewCfg<FMT_MXFP4>::max_smem_bytes()) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_MXFP4, 2>, GemmFewCfg<FMT_MXFP4>::max_smem_bytes()) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_NVFP4, 1>, GemmFewCfg<FMT_NVFP4>::max_smem_bytes()) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_NVFP4, 2>, GemmFewCfg<FMT_NVFP4>::max_smem_bytes()) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_MXINT4, 1>, GemmFewCfg<FMT_MXINT4>::max_smem_bytes()) &&
+              opt_in_smem(gemm_fewtok_kernel<FMT_MXINT4, 2>, GemmFewCfg<FMT_MXINT4>::max_smem_bytes()) &&
               opt_in_smem(rotate_quantize_kernel<256, FMT_F32OUT>, RotCfg<256>::SMEM_BYTES) &&
               opt_in_smem(rotate_quantize_pair_kernel<FMT_F32OUT>, RotPairCfg::SMEM_BYTES);
     if (!ok) return nullptr;
@@ -605,9 +608,14 @@ static torq_status gemm_impl(const void* Aq, const void* As, const void* Wq, con
     if (!encode_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (uint64_t)N, krow, 128, 128) ||
         !encode_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Aq, (uint64_t)M, krow, (uint32_t)ntok, 128))
       return TORQ_ERR_LAUNCH;
-    launch_tc(gemm_fewtok_kernel<FMT>, S, tiles * S, FC::THREADS, FC::smem_bytes(ntok), s, tmB, tmA,
-              static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y, y_dtype == TORQ_BF16 ? 1 : 0, (int)M,
-              (int)N, (int)K, ntok, S, alpha, st->err_word);
+    if (FC::ctas_per_sm(ntok) >= 2)                      // up to 64 tokens: one set of epilogue warps, two CTAs per SM
+      launch_tc(gemm_fewtok_kernel<FMT, 1>, S, tiles * S, 192, FC::smem_bytes(ntok), s, tmB, tmA,
+                static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y, y_dtype == TORQ_BF16 ? 1 : 0, (int)M,
+                (int)N, (int)K, ntok, S, alpha, st->err_word);
+    else                                                 // 128 tokens: two sets
+      launch_tc(gemm_fewtok_kernel<FMT, 2>, S, tiles * S, 320, FC::smem_bytes(ntok), s, tmB, tmA,
+                static_cast<const uint8_t*>(As), static_cast<const uint8_t*>(Ws), Y, y_dtype == TORQ_BF16 ? 1 : 0, (int)M,
+                (int)N, (int)K, ntok, S, alpha, st->err_word);
     return launch_status();
   }
   // CTA pairs from two row tiles on -- except for exactly two row tiles with so few 256-column tiles
