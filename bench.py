@@ -2,7 +2,7 @@
 """Benchmark of the rotated-MXFP4 linear hot path (rotate -> MXFP4 quantize -> block-scaled FP4
 GEMM).  The timed K steps run the LLaMA3-8B QKV-projection shape (M=2048 tokens, d=4096, N=6144,
 bf16 output); the same line also carries the second 8B shape (down-projection, 2048 x 14336 ->
-4096) and a token sweep at d = N = 5120 (M = 1, 64, 256, 1024, 16384), each with per-kernel times,
+4096) and a token sweep at d = N = 5120 (M = 1, 4, 16, 64, 256, 1024, 4096, 16384), each with per-kernel times,
 both roofline fractions and the SM clock sampled inside its own loop.
 
 One step = one pass of the whole path over one batch of seeded synthetic activations.  Prints ONE
@@ -548,7 +548,7 @@ def measure_e2e(torq, layer, stream, steps, barrier):
     barrier()
     return e0.elapsed_time(e1) / n, Xh.numel() * 2, Yh[0].numel() * 2
 
-SWEEP_M = (1, 64, 256, 1024, 16384)
+SWEEP_M = (1, 4, 16, 64, 256, 1024, 4096, 16384)
 
 
 def main():
