@@ -29,8 +29,8 @@ def _narrow_starts(rows, cols):
 
 # (rows, cols) with both kinds of narrow tiles on 74 pairs: 3840 x 1280 -> 72 wide + 4 narrow (columns 512, 704,
 # 896, 1088), 4864 x 1024 -> 73 + 4 (one row tile: 256, 448, 640, 832), 2500 x 2048 -> 74 + 8 with a ragged last
-# row tile
-SHAPES = [(3840, 1280), (4864, 1024), (2500, 2048)]
+# row tile; 6400 x 768 -> 72 + 4, where the one row tile that trades has no 256-column tile left at all
+SHAPES = [(3840, 1280), (4864, 1024), (2500, 2048), (6400, 768)]
 
 
 def _rand_rotation(d, seed):
@@ -129,7 +129,7 @@ def _gpu_gemm(ac, asb, wc, wsb, out_dtype):
     return y.float().cpu().numpy().astype(np.float64)
 
 
-@pytest.mark.parametrize("M,N,K", [(3840, 1280, 512), (4864, 1024, 384), (2500, 2048, 256)])
+@pytest.mark.parametrize("M,N,K", [(3840, 1280, 512), (4864, 1024, 384), (2500, 2048, 256), (6400, 768, 256)])
 def test_gemm_mxfp4(M, N, K):
     if _pairs() == 74:
         assert _narrow_starts(M, N) == [0, 64]
